@@ -1,0 +1,215 @@
+/*
+ * pq.h -- C ABI of the B200 (sm_100a) PermuQuant quantized-linear library.
+ *
+ * The library implements the per-group quantized linear layer of the PermuQuant method:
+ *   offline : channel statistics -> joint second-moment sort candidates (Eq. 9, Prop. 3.2)
+ *             -> calibration error of every candidate (Eq. 3) -> acceptance rule (Eq. 10)
+ *             -> permuted, quantized weight (Eq. 8, P^T W);
+ *   runtime : bf16 activations (already in permuted channel order) -> NVFP4 -> W4A4
+ *             block-scaled GEMM with fp32 accumulation and bf16 output (Eq. 8, Q(XP) Q(P^T W)).
+ *
+ * General rules for every entry point
+ *   - Every tensor pointer is a DEVICE pointer owned by the caller, 16-byte aligned unless
+ *     stated otherwise.  The library allocates nothing and frees nothing (scratch memory is a
+ *     caller-provided workspace sized by pq_workspace_bytes).
+ *   - Work is enqueued on `stream` (a cudaStream_t passed as void*; NULL = default stream)
+ *     and the call returns without synchronising.  Device scalars (tensor scales, best, accept)
+ *     are read and written by kernels, so a whole pipeline can be enqueued back to back.
+ *   - Errors are reported by return code only; argument errors are detected on the host before
+ *     anything is launched.  Nothing aborts, throws or prints.
+ *   - bf16 tensors are row-major [rows, K] with leading dimension `ld` (elements, multiple of 8),
+ *     K contiguous.  Activations are X[M,K]; weights are stored transposed, Wt[N,K] (the
+ *     nn.Linear convention), so "input channel i of W" is column i of Wt.
+ *   - Permutations use the gather convention of App. C: position j of the reordered tensor
+ *     reads channel perm[j] of the original one.
+ *   - Inputs must be finite.  Tensor scales must lie in [2^-100, 2^100].
+ *
+ * NVFP4 storage
+ *   codes : uint8 [rows, K/2], channel 2j in the low nibble and 2j+1 in the high nibble;
+ *           nibble = sign bit (8) | E2M1 magnitude code 0..7 = {0, .5, 1, 1.5, 2, 3, 4, 6}.
+ *   sf    : one unsigned E4M3 byte per 16 channels.  PQ_SF_LINEAR: [rows, K/16] row-major.
+ *           PQ_SF_TCGEN05: the tensor-core layout -- rows padded to a multiple of 128 and K/16
+ *           padded to a multiple of 4; the tensor is tiled in blocks of 128 rows x 4 scale
+ *           columns, blocks ordered [row block][column block], 512 bytes each; inside a block the
+ *           byte of (row r, column c) sits at (r % 32) * 16 + (r / 32) * 4 + c.
+ *           Size in bytes: pq_sf_bytes(rows, K, layout).
+ *   ts    : one fp32 tensor scale; value = E2M1 value * E4M3 scale * ts.
+ */
+#ifndef PQ_H
+#define PQ_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    PQ_OK = 0,
+    PQ_ERR_NULL = 1,      /* a required pointer is NULL */
+    PQ_ERR_SHAPE = 2,     /* a size is out of range or not divisible as required */
+    PQ_ERR_ALIGN = 3,     /* a pointer or leading dimension is misaligned */
+    PQ_ERR_FORMAT = 4,    /* unsupported pq_format / scale layout */
+    PQ_ERR_WORKSPACE = 5, /* workspace missing or too small */
+    PQ_ERR_CUDA = 6,      /* the CUDA runtime reported an error (launch, attribute, driver) */
+    PQ_ERR_TIMEOUT = 7    /* a bounded device-side wait expired (see pq_device_status) */
+} pq_status;
+
+/* Quantization format of the error / fake-quant entry points.
+ *   kind 0: NVFP4 (bits and group ignored: 4 bits, groups of 16).
+ *   kind 1: symmetric integer, Eq. 1-2, Q = 2^(bits-1) - 1; bits in 2..8, group in {16,32,64,128}. */
+typedef struct {
+    int kind;
+    int bits;
+    int group;
+} pq_format;
+
+enum { PQ_SF_LINEAR = 0, PQ_SF_TCGEN05 = 1 };
+
+/* Which entry point a workspace is for (argument `op` of pq_workspace_bytes). */
+enum {
+    PQ_OP_CALIB_STATS = 1,
+    PQ_OP_SELECT_PERM = 2,
+    PQ_OP_GROUP_ERROR = 3,
+    PQ_OP_QUANT_WEIGHT = 4,
+    PQ_OP_GEMM = 5
+};
+
+/* Rows per fp32 partial sum in pq_calib_stats and pq_group_error (part of the arithmetic
+ * definition: results depend on it). */
+#define PQ_CHUNK_ROWS 64
+
+const char *pq_status_string(pq_status s);
+
+/* Library version as major*100 + minor. */
+int pq_version(void);
+
+/* Bytes of scratch the given entry point needs for these sizes (rows = M / T / N as the entry
+ * point calls it, P = number of candidate orders, ignored elsewhere).  Never fails; unknown op
+ * returns 0.  The workspace must be 256-byte aligned. */
+size_t pq_workspace_bytes(int op, int64_t rows, int64_t K, int64_t N, int P);
+
+/* Bytes of the scale tensor of a [rows, K] NVFP4 tensor in the given layout (0 on bad input). */
+size_t pq_sf_bytes(int64_t rows, int64_t K, int sf_layout);
+
+/* Channel statistics (second moment of Assumption 3.1 / Sec. 3.3 before the division by the
+ * row count, and the absmax used for the tensor scale).  For every channel i:
+ *     sumsq[i] += sum_t T[t,i]^2        amax[i] = max(amax[i], |T[t,i]|)
+ * Rows are cut into chunks of PQ_CHUNK_ROWS; squares are accumulated in fp32 (fused
+ * multiply-add, row order) inside a chunk, chunk partials are added to the fp64 total in
+ * ascending order.  Call once per calibration batch (and once on Wt for the weight side);
+ * the caller zeroes sumsq / amax before the first batch.
+ *   T     : bf16 [rows, K], ld.  K % 8 == 0.
+ *   sumsq : fp64 [K] in/out.  amax : fp32 [K] in/out.
+ *   ws    : pq_workspace_bytes(PQ_OP_CALIB_STATS, rows, K, 0, 0). */
+pq_status pq_calib_stats(const void *T, int64_t rows, int64_t K, int64_t ld, double *sumsq,
+                         float *amax, void *ws, size_t ws_bytes, void *stream);
+
+/* fp32 tensor scale from per-channel absmax: *ts = max_i amax[i] / 2688 (= 6 * 448), or 1 if
+ * the maximum is 0.  ts is a device scalar. */
+pq_status pq_tensor_scale(const float *amax, int64_t K, float *ts, void *stream);
+
+/* Sort candidates of the joint second-moment criterion, Eq. 9, for alpha = j/J, j = 0..J.
+ * With a_i = sumsq_a[i]/rows_a and w_i = sumsq_w[i]/rows_w the key of channel i is the
+ * left-to-right fp64 product of j factors a_i and J-j factors w_i (ordered like
+ * (a_i)^alpha (w_i)^(1-alpha)).  perms[j*K + pos] = channel with the pos-th largest key; equal
+ * keys keep ascending channel order.  j = J is the activation-only sort of Prop. 3.2, j = 0 the
+ * weight-only sort.
+ *   K <= 16384, 1 <= J <= 16.  perms : int32 [J+1, K] out.  ws: unused (may be NULL). */
+pq_status pq_select_perm(const double *sumsq_a, int64_t rows_a, const double *sumsq_w,
+                         int64_t rows_w, int64_t K, int J, int32_t *perms, void *ws,
+                         size_t ws_bytes, void *stream);
+
+/* Calibration quantization error, Eq. 3, per candidate order p and group column k:
+ *     err[p*(K/g) + k] += sum_t sum_{j<g} (e_j - ehat_j)^2,   e_j = T[t, perms[p*K + k*g + j]]
+ * where ehat is the per-group quantize-dequantize of e in format `fmt` (NVFP4 with tensor scale
+ * *ts, or Eq. 1-2 integers).  perms == NULL means P == 1 and the original order.  fp32
+ * arithmetic: residual by one fused multiply-add, squares summed in runs of 8 channels, runs
+ * combined pairwise; rows chunked as in pq_calib_stats; fp64 across chunks and calls.
+ *   T : bf16 [rows, K], ld.  K % group == 0, K <= 16384, 1 <= P <= 8.
+ *   ts: device fp32 scalar (NVFP4 only, else may be NULL).
+ *   err : fp64 [P, K/g] in/out (caller zeroes before the first batch).
+ *   ws : pq_workspace_bytes(PQ_OP_GROUP_ERROR, rows, K, 0, P). */
+pq_status pq_group_error(const void *T, int64_t rows, int64_t K, int64_t ld, pq_format fmt,
+                         const float *ts, const int32_t *perms, int P, double *err, void *ws,
+                         size_t ws_bytes, void *stream);
+
+/* Relative-error weights for pq_accept: lambda[0] = 1 / sum_i sumsq_a[i], lambda[1] =
+ * 1 / sum_i sumsq_w[i] (sequential fp64 sums in channel order).  lambda: device fp64 [2]. */
+pq_status pq_error_weights(const double *sumsq_a, const double *sumsq_w, int64_t K, double *lambda,
+                           void *stream);
+
+/* Candidate selection and the acceptance rule, Eq. 10.  Row 0 of err_x / err_w is the original
+ * order, rows 1..P the candidates.
+ *     E[p] = lambda[0] * sum_k err_x[p,k] + lambda[1] * sum_k err_w[p,k]      (fp64, in k order)
+ *     best = argmin_{p in 1..P} E[p] (first on ties);   accept = (E[0] - E[best] > tau * E[0]).
+ * tau is a fraction (the paper's 2.5 means 0.025); tau = 0 is the paper's default.
+ *   lambda : device fp64 [2], or NULL for (1, 1).  best, accept : device int32 scalars out.
+ *   E : device fp64 [P+1] out, or NULL. */
+pq_status pq_accept(const double *err_x, const double *err_w, const double *lambda, int P,
+                    int64_t Kg, double tau, int32_t *best, int32_t *accept, double *E,
+                    void *stream);
+
+/* Offline weight path of Eq. 8: gather the input channels by perm (P^T W), compute the weight
+ * tensor scale *ts_w = max|Wt| / 2688 and quantize to NVFP4.
+ *   Wt : bf16 [N, K], ld.  K % 16 == 0 (K % 64 == 0 for PQ_SF_TCGEN05), K <= 16384.
+ *   perm : int32 [K] or NULL (original order).
+ *   perm_select : device int32 [2] = {best, accept} as written by pq_accept, or NULL.  When
+ *       given, `perm` must be the [J+1, K] candidate table and the row best-1 is used if
+ *       accept != 0, the original order otherwise -- so the decision never visits the host.
+ *   codes : uint8 [N, K/2] out.  sf : pq_sf_bytes(N, K, sf_layout) bytes out.  ts_w : device out.
+ *   ws : pq_workspace_bytes(PQ_OP_QUANT_WEIGHT, N, K, 0, 0). */
+pq_status pq_quant_weight(const void *Wt, int64_t N, int64_t K, int64_t ld, const int32_t *perm,
+                          const int32_t *perm_select, uint8_t *codes, uint8_t *sf, int sf_layout,
+                          float *ts_w, void *ws, size_t ws_bytes, void *stream);
+
+/* Runtime activation quantizer (dynamic per-group scales, static tensor scale *ts_x from
+ * calibration).  Per row and 16-channel group: absmax -> E4M3(absmax / (6 ts)) -> 16 E2M1 codes
+ * of x / (scale * ts), round to nearest even, saturating.  Channels arrive already permuted.
+ *   X : bf16 [M, K], ld.  K % 16 == 0 (K % 64 == 0 for PQ_SF_TCGEN05).
+ *   codes : uint8 [M, K/2] out.  sf : pq_sf_bytes(M, K, sf_layout) bytes out (padding bytes of
+ *   the tensor-core layout are written as 0). */
+pq_status pq_quant_act_nvfp4(const void *X, int64_t M, int64_t K, int64_t ld, const float *ts_x,
+                             uint8_t *codes, uint8_t *sf, int sf_layout, void *stream);
+
+/* W4A4 block-scaled GEMM, right-hand side of Eq. 8:
+ *     Y[m,n] = bf16( ts_x*ts_w * sum_kb sfx[m,kb]*sfw[n,kb] * sum_{j<16} qx[m,16kb+j]*qw[n,16kb+j] )
+ * on the tcgen05 tensor cores (E2M1 operands, UE4M3 block scales in tensor memory, fp32
+ * accumulation).  Both scale tensors must be in PQ_SF_TCGEN05 layout.
+ *   xq [M,K/2], wq [N,K/2] codes;  K % 64 == 0, K >= 64;  N % 8 == 0;  M, N >= 1.
+ *   Y : bf16 [M, N], ldy (multiple of 8).
+ *   ws : pq_workspace_bytes(PQ_OP_GEMM, M, K, N, 0) (holds the device status word).
+ * Every device-side wait is bounded; if one expires the kernel records PQ_ERR_TIMEOUT in the
+ * status word (read it with pq_device_status) and returns. */
+pq_status pq_gemm_w4a4(const uint8_t *xq, const uint8_t *sfx, const float *ts_x, const uint8_t *wq,
+                       const uint8_t *sfw, const float *ts_w, int64_t M, int64_t N, int64_t K,
+                       void *Y, int64_t ldy, void *ws, size_t ws_bytes, void *stream);
+
+/* The timed runtime path: pq_quant_act_nvfp4 (tensor-core scale layout) followed by
+ * pq_gemm_w4a4.  xq / sfx are caller-provided intermediates of the sizes above. */
+pq_status pq_linear_w4a4(const void *X, int64_t M, int64_t K, int64_t ld, const float *ts_x,
+                         uint8_t *xq, uint8_t *sfx, const uint8_t *wq, const uint8_t *sfw,
+                         const float *ts_w, int64_t N, void *Y, int64_t ldy, void *ws,
+                         size_t ws_bytes, void *stream);
+
+/* Integer fake-quant of Eq. 1-2 (quantize, dequantize, round to bf16), optional gather.
+ *   T : bf16 [rows, K], ld.  out : bf16 [rows, K], ldo.  perm : int32 [K] or NULL.
+ *   fmt.kind must be 1; K % fmt.group == 0; K <= 16384 when perm != NULL. */
+pq_status pq_fakequant_int(const void *T, int64_t rows, int64_t K, int64_t ld, pq_format fmt,
+                           const int32_t *perm, void *out, int64_t ldo, void *stream);
+
+/* Rearrange scale bytes from the tensor-core layout into [rows, K/16] row-major (for tests and
+ * debugging). */
+pq_status pq_sf_to_linear(const uint8_t *sf_tc, int64_t rows, int64_t K, uint8_t *sf_linear,
+                          void *stream);
+
+/* Synchronises `stream`, then reads the status word a GEMM workspace holds: PQ_OK, or
+ * PQ_ERR_TIMEOUT if a bounded wait inside the kernel expired, PQ_ERR_CUDA if the stream reports
+ * an asynchronous error.  HOST call; `ws` is the device workspace passed to pq_gemm_w4a4. */
+pq_status pq_device_status(const void *ws, void *stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* PQ_H */

@@ -1,0 +1,35 @@
+// Entry points that launch no kernel: status strings, version, workspace sizing.
+#include "pq_common.cuh"
+
+extern "C" const char *pq_status_string(pq_status s) {
+    switch (s) {
+        case PQ_OK: return "ok";
+        case PQ_ERR_NULL: return "a required pointer is NULL";
+        case PQ_ERR_SHAPE: return "size out of range or not divisible as required";
+        case PQ_ERR_ALIGN: return "pointer or leading dimension misaligned";
+        case PQ_ERR_FORMAT: return "unsupported quantization format or scale layout";
+        case PQ_ERR_WORKSPACE: return "workspace missing or too small";
+        case PQ_ERR_CUDA: return "CUDA runtime error";
+        case PQ_ERR_TIMEOUT: return "a bounded device-side wait expired";
+    }
+    return "unknown status";
+}
+
+extern "C" int pq_version(void) { return 1; }
+
+static size_t round256(size_t b) { return (b + 255) / 256 * 256; }
+
+extern "C" size_t pq_workspace_bytes(int op, int64_t rows, int64_t K, int64_t N, int P) {
+    (void)N;
+    if (K <= 0) return 0;
+    const int64_t chunks = rows > 0 ? pq_ceil_div(rows, PQ_CHUNK_ROWS) : 0;
+    switch (op) {
+        case PQ_OP_CALIB_STATS: return round256(static_cast<size_t>(chunks) * K * sizeof(float));
+        case PQ_OP_SELECT_PERM: return round256(static_cast<size_t>(P > 0 ? P : 1) * K * sizeof(uint64_t));
+        case PQ_OP_GROUP_ERROR:
+            return round256(static_cast<size_t>(chunks) * (P > 0 ? P : 1) * (K / 16 + 1) * sizeof(float));
+        case PQ_OP_QUANT_WEIGHT: return 256;
+        case PQ_OP_GEMM: return 256;
+        default: return 0;
+    }
+}

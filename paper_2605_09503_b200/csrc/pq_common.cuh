@@ -1,0 +1,169 @@
+// Shared device/host helpers of the CUDA library: argument checks, bf16 unpacking and the
+// NVFP4 / integer group arithmetic used by the quantize, fake-quant and error kernels.
+//
+// Arithmetic contract (bit-exactness with the CPU definition depends on it): no fast-math,
+// denormals kept, IEEE division and reciprocal, fused multiply-add only where written.
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_fp16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/pq.h"
+
+#define PQ_REQUIRE(cond, code) \
+    do {                       \
+        if (!(cond)) return (code); \
+    } while (0)
+
+#define PQ_CUDA_OK(expr)                          \
+    do {                                          \
+        if ((expr) != cudaSuccess) {              \
+            (void)cudaGetLastError();             \
+            return PQ_ERR_CUDA;                   \
+        }                                         \
+    } while (0)
+
+static inline bool pq_aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+static inline bool pq_aligned256(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 255u) == 0; }
+
+static inline pq_status pq_launch_status() {
+    return cudaGetLastError() == cudaSuccess ? PQ_OK : PQ_ERR_CUDA;
+}
+
+static inline int64_t pq_ceil_div(int64_t a, int64_t b) { return (a + b - 1) / b; }
+
+#ifdef __CUDACC__
+
+namespace pq {
+
+// Eight consecutive bf16 values (one 16-byte load) widened to fp32 (exact).
+__device__ __forceinline__ void unpack8(const uint4 &v, float (&x)[8]) {
+    const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        x[2 * i] = __uint_as_float(w[i] << 16);
+        x[2 * i + 1] = __uint_as_float(w[i] & 0xFFFF0000u);
+    }
+}
+
+__device__ __forceinline__ float bf16_bits_to_f32(uint16_t h) {
+    return __uint_as_float(static_cast<uint32_t>(h) << 16);
+}
+
+__device__ __forceinline__ float absmax8(const float (&x)[8]) {
+    float a = 0.0f;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) a = fmaxf(a, fabsf(x[i]));
+    return a;
+}
+
+// Maximum over the TEAM consecutive lanes (TEAM = channels per group / 8) a group spans.
+template <int TEAM>
+__device__ __forceinline__ float team_max(float a) {
+#pragma unroll
+    for (int m = 1; m < TEAM; m <<= 1) a = fmaxf(a, __shfl_xor_sync(0xFFFFFFFFu, a, m));
+    return a;
+}
+
+// Balanced adjacent-pair tree over the team's run sums; every lane ends with the same value
+// because fp32 addition is commutative.
+template <int TEAM>
+__device__ __forceinline__ float team_sum(float o) {
+#pragma unroll
+    for (int m = 1; m < TEAM; m <<= 1) o = __fadd_rn(o, __shfl_xor_sync(0xFFFFFFFFu, o, m));
+    return o;
+}
+
+// fp32 -> unsigned E4M3 byte, round to nearest even, saturating at 448 (hardware convert).
+__device__ __forceinline__ uint32_t f32_to_e4m3(float u) {
+    uint16_t r;
+    asm("cvt.rn.satfinite.e4m3x2.f32 %0, %1, %2;" : "=h"(r) : "f"(0.0f), "f"(u));
+    return r & 0xFFu;
+}
+
+// E4M3 byte -> fp32 (exact: through the hardware e4m3 -> f16 convert).
+__device__ __forceinline__ float e4m3_to_f32(uint32_t b) {
+    uint32_t h2;
+    asm("cvt.rn.f16x2.e4m3x2 %0, %1;" : "=r"(h2) : "h"(static_cast<uint16_t>(b)));
+    return __half2float(__ushort_as_half(static_cast<uint16_t>(h2 & 0xFFFFu)));
+}
+
+// Eight fp32 -> eight E2M1 nibbles (element i in bits 4i..4i+3), RNE, saturating, sign kept.
+__device__ __forceinline__ uint32_t f32x8_to_e2m1(const float (&y)[8]) {
+    uint32_t out;
+    asm("{\n"
+        ".reg .b8 b0, b1, b2, b3;\n"
+        "cvt.rn.satfinite.e2m1x2.f32 b0, %2, %1;\n"
+        "cvt.rn.satfinite.e2m1x2.f32 b1, %4, %3;\n"
+        "cvt.rn.satfinite.e2m1x2.f32 b2, %6, %5;\n"
+        "cvt.rn.satfinite.e2m1x2.f32 b3, %8, %7;\n"
+        "mov.b32 %0, {b0, b1, b2, b3};\n"
+        "}\n"
+        : "=r"(out)
+        : "f"(y[0]), "f"(y[1]), "f"(y[2]), "f"(y[3]), "f"(y[4]), "f"(y[5]), "f"(y[6]), "f"(y[7]));
+    return out;
+}
+
+// Eight E2M1 nibbles -> their fp32 values.  Twice the magnitude of code m is the m-th nibble of
+// 0xC8643210 (0, 1, 2, 3, 4, 6, 8, 12); the int -> float conversion and the halving are exact.
+__device__ __forceinline__ void e2m1x8_to_f32(uint32_t codes, float (&q)[8]) {
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        const uint32_t c = (codes >> (4 * i)) & 0xFu;
+        const uint32_t twice = (0xC8643210u >> ((c & 7u) * 4)) & 0xFu;
+        const float mag = __fmul_rn(static_cast<float>(twice), 0.5f);
+        q[i] = __uint_as_float(__float_as_uint(mag) | ((c & 8u) << 28));
+    }
+}
+
+// NVFP4 scale of one group from its absmax: E4M3 byte and fp32 decode scale d = sf * ts.
+__device__ __forceinline__ void nvfp4_scale(float amax, float ts, uint32_t &sf8, float &d, float &r) {
+    const float c = __fmul_rn(6.0f, ts);
+    const float u = __fdiv_rn(amax, c);
+    sf8 = f32_to_e4m3(u);
+    d = __fmul_rn(e4m3_to_f32(sf8), ts);
+    r = (d > 0.0f) ? __frcp_rn(d) : 0.0f;
+}
+
+// NVFP4 codes of this lane's eight values given the group's reciprocal decode scale.
+__device__ __forceinline__ uint32_t nvfp4_codes(const float (&x)[8], float r) {
+    float y[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) y[i] = __fmul_rn(x[i], r);
+    return f32x8_to_e2m1(y);
+}
+
+// Integer quantizer of Eq. 1-2: s = amax / Q, z = clamp(rint(x * (1/s)), -Q, Q).
+__device__ __forceinline__ void int_scale(float amax, float Qf, float &s, float &r) {
+    s = __fdiv_rn(amax, Qf);
+    r = (s > 0.0f) ? __frcp_rn(s) : 0.0f;
+}
+
+__device__ __forceinline__ void int_levels(const float (&x)[8], float r, float Qf, float (&z)[8]) {
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        float q = rintf(__fmul_rn(x[i], r));
+        z[i] = fminf(fmaxf(q, -Qf), Qf);
+    }
+}
+
+// Sum of squared residuals of eight values: delta = fma(-q, d, x); acc = fma(delta, delta, acc).
+__device__ __forceinline__ float run_sse(const float (&x)[8], const float (&q)[8], float d) {
+    float acc = 0.0f;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        const float delta = __fmaf_rn(-q[i], d, x[i]);
+        acc = __fmaf_rn(delta, delta, acc);
+    }
+    return acc;
+}
+
+// Byte offset of scale (row, col) in the tensor-core layout; kb4 = number of 4-column blocks.
+__device__ __host__ __forceinline__ int64_t sf_tc_offset(int64_t row, int64_t col, int64_t kb4) {
+    return ((row >> 7) * kb4 + (col >> 2)) * 512 + (row & 31) * 16 + ((row >> 5) & 3) * 4 + (col & 3);
+}
+
+}  // namespace pq
+#endif  // __CUDACC__
