@@ -179,7 +179,9 @@ pq_status pq_quant_act_nvfp4(const void *X, int64_t M, int64_t K, int64_t ld, co
  * accumulation).  Both scale tensors must be in PQ_SF_TCGEN05 layout.
  *   xq [M,K/2], wq [N,K/2] codes;  K % 64 == 0, K >= 64;  N % 8 == 0;  M, N >= 1.
  *   Y : bf16 [M, N], ldy (multiple of 8).
- *   ws : pq_workspace_bytes(PQ_OP_GEMM, M, K, N, 0) (holds the device status word).
+ *   ws : pq_workspace_bytes(PQ_OP_GEMM, M, K, N, 0) bytes holding the device status word.  The
+ *        caller zeroes it once (cudaMemset) before the first GEMM that uses it; the kernel only
+ *        ever writes a non-zero code there.
  * Every device-side wait is bounded; if one expires the kernel records PQ_ERR_TIMEOUT in the
  * status word (read it with pq_device_status) and returns. */
 pq_status pq_gemm_w4a4(const uint8_t *xq, const uint8_t *sfx, const float *ts_x, const uint8_t *wq,

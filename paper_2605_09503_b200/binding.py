@@ -107,7 +107,7 @@ def sf_bytes(rows, K, layout):
 
 def workspace(op, rows, K, N=0, P=0, device="cuda"):
     """Allocate (through torch) a workspace big enough for the given call."""
-    return torch.empty(max(workspace_bytes(op, rows, K, N, P), 256), dtype=torch.uint8, device=device)
+    return torch.zeros(max(workspace_bytes(op, rows, K, N, P), 256), dtype=torch.uint8, device=device)
 
 
 def _ws(ws):

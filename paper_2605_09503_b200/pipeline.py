@@ -1,0 +1,116 @@
+"""Sequencing of the C-ABI calls into the two halves of the method.  No arithmetic happens
+here: every step is one entry point of libpq.so, all enqueued on the current stream without a
+host round trip (the accept decision stays on the device and is consumed by pq_quant_weight).
+
+  calibrate()  offline: statistics -> Eq. 9 candidates -> Eq. 3 errors -> Eq. 10 -> P^T W quantized
+  QuantLinear  runtime: bf16 activations (already permuted) -> NVFP4 -> W4A4 GEMM -> bf16
+"""
+from dataclasses import dataclass
+
+import torch
+
+from . import binding as B
+
+NVFP4 = (B.KIND_NVFP4, 4, 16)
+
+
+@dataclass
+class Calibration:
+    """Everything the offline pass produces, all on the device."""
+    sumsq_a: torch.Tensor      # fp64 [K]
+    sumsq_w: torch.Tensor      # fp64 [K]
+    amax_a: torch.Tensor       # fp32 [K]
+    ts_x: torch.Tensor         # fp32 [1] static activation tensor scale
+    ts_w: torch.Tensor         # fp32 [1]
+    perms: torch.Tensor        # int32 [J+1, K] candidates, row j <-> alpha = j/J
+    err_x: torch.Tensor        # fp64 [J+2, K/g], row 0 = original order
+    err_w: torch.Tensor        # fp64 [J+2, K/g]
+    lam: torch.Tensor          # fp64 [2]
+    E: torch.Tensor            # fp64 [J+2]
+    select: torch.Tensor       # int32 [2] = {best, accept}
+    wq: torch.Tensor           # uint8 [N, K/2]
+    sfw: torch.Tensor          # uint8, tensor-core layout
+    rows_a: int
+
+    def chosen_perm(self) -> torch.Tensor:
+        """The order the acceptance rule kept (identity if rejected), as int64 indices."""
+        best, accept = self.select.tolist()
+        K = self.perms.shape[1]
+        if accept:
+            return self.perms[best - 1].long()
+        return torch.arange(K, device=self.perms.device)
+
+
+def calibrate(batches, Wt, fmt=NVFP4, J=5, tau=0.0, sf_layout=B.PQ_SF_TCGEN05) -> Calibration:
+    """Offline pass over calibration batches (list of bf16 [T, K] device tensors) and the weight
+    Wt (bf16 [N, K] device tensor).  `fmt` is the format whose error drives the acceptance rule."""
+    dev = Wt.device
+    N, K = Wt.shape
+    group = 16 if fmt[0] == B.KIND_NVFP4 else fmt[2]
+    Kg = K // group
+    sumsq_a = torch.zeros(K, dtype=torch.float64, device=dev)
+    sumsq_w = torch.zeros(K, dtype=torch.float64, device=dev)
+    amax_a = torch.zeros(K, dtype=torch.float32, device=dev)
+    amax_w = torch.zeros(K, dtype=torch.float32, device=dev)
+    rows_a = 0
+    max_rows = max([b.shape[0] for b in batches] + [N])
+    ws = B.workspace(B.OP_GROUP_ERROR, max_rows, K, 0, J + 1)     # large enough for every step below
+    ws_stats = B.workspace(B.OP_CALIB_STATS, max_rows, K)
+    for x in batches:
+        B.pq_calib_stats(x, sumsq_a, amax_a, ws_stats)
+        rows_a += x.shape[0]
+    B.pq_calib_stats(Wt, sumsq_w, amax_w, ws_stats)
+    ts_x = torch.empty(1, dtype=torch.float32, device=dev)
+    ts_w_err = torch.empty(1, dtype=torch.float32, device=dev)
+    B.pq_tensor_scale(amax_a, ts_x)
+    B.pq_tensor_scale(amax_w, ts_w_err)
+
+    perms = torch.empty(J + 1, K, dtype=torch.int32, device=dev)
+    B.pq_select_perm(sumsq_a, rows_a, sumsq_w, N, J, perms, B.workspace(B.OP_SELECT_PERM, 0, K, 0, J + 1))
+
+    err_x = torch.zeros(J + 2, Kg, dtype=torch.float64, device=dev)
+    err_w = torch.zeros(J + 2, Kg, dtype=torch.float64, device=dev)
+    for x in batches:
+        B.pq_group_error(x, fmt, ts_x, None, err_x[0:1], ws)
+        B.pq_group_error(x, fmt, ts_x, perms, err_x[1:], ws)
+    B.pq_group_error(Wt, fmt, ts_w_err, None, err_w[0:1], ws)
+    B.pq_group_error(Wt, fmt, ts_w_err, perms, err_w[1:], ws)
+
+    lam = torch.empty(2, dtype=torch.float64, device=dev)
+    B.pq_error_weights(sumsq_a, sumsq_w, lam)
+    select = torch.zeros(2, dtype=torch.int32, device=dev)
+    E = torch.empty(J + 2, dtype=torch.float64, device=dev)
+    B.pq_accept(err_x, err_w, lam, tau, select[0:1], select[1:2], E)
+
+    wq = torch.empty(N, K // 2, dtype=torch.uint8, device=dev)
+    sfw = torch.empty(B.sf_bytes(N, K, sf_layout), dtype=torch.uint8, device=dev)
+    ts_w = torch.empty(1, dtype=torch.float32, device=dev)
+    B.pq_quant_weight(Wt, perms, select, wq, sfw, sf_layout, ts_w, B.workspace(B.OP_QUANT_WEIGHT, N, K))
+    return Calibration(sumsq_a, sumsq_w, amax_a, ts_x, ts_w, perms, err_x, err_w, lam, E, select, wq, sfw, rows_a)
+
+
+class QuantLinear:
+    """Runtime half: holds the quantized weight and the intermediates of one layer."""
+
+    def __init__(self, wq, sfw, ts_w, ts_x, M_max):
+        self.wq, self.sfw, self.ts_w, self.ts_x = wq, sfw, ts_w, ts_x
+        self.N, self.K = wq.shape[0], wq.shape[1] * 2
+        dev = wq.device
+        self.xq = torch.empty(M_max, self.K // 2, dtype=torch.uint8, device=dev)
+        self.sfx = torch.empty(B.sf_bytes(M_max, self.K, B.PQ_SF_TCGEN05), dtype=torch.uint8, device=dev)
+        self.ws = B.workspace(B.OP_GEMM, M_max, self.K, self.N)
+        self.M_max = M_max
+
+    def __call__(self, X, Y=None):
+        M = X.shape[0]
+        assert M <= self.M_max and X.shape[1] == self.K
+        if Y is None:
+            Y = torch.empty(M, self.N, dtype=torch.bfloat16, device=X.device)
+        B.pq_linear_w4a4(X, self.ts_x, self.xq[:M], self.sfx, self.wq, self.sfw, self.ts_w, Y, self.ws)
+        return Y
+
+    def check(self):
+        """Synchronise and raise if a bounded device-side wait expired."""
+        code = B.pq_device_status(self.ws)
+        if code != B.PQ_OK:
+            raise B.PqError("pq_gemm_w4a4 (device)", code, B.status_string(code))
