@@ -195,6 +195,19 @@ pq_status pq_linear_w4a4(const void *X, int64_t M, int64_t K, int64_t ld, const 
                          const float *ts_w, int64_t N, void *Y, int64_t ldy, void *ws,
                          size_t ws_bytes, void *stream);
 
+/* The same runtime path for a caller whose tensors live in HOST memory (the end-to-end
+ * measurement): copies X_host -> X_dev on `stream`, runs pq_linear_w4a4, copies Y_dev -> Y_host,
+ * all asynchronously on `stream` (the caller synchronises the stream before reading Y_host).
+ *   X_host : bf16 [M, K] contiguous HOST memory (pinned for the copy to be asynchronous).
+ *   Y_host : bf16 [M, N] contiguous HOST memory, out.
+ *   X_dev  : bf16 [M, K] contiguous device staging buffer;  Y_dev : bf16 [M, N] contiguous device
+ *            staging buffer;  everything else as in pq_linear_w4a4.
+ * Returns PQ_ERR_CUDA if a copy cannot be enqueued. */
+pq_status pq_linear_w4a4_host(const void *X_host, int64_t M, int64_t K, const float *ts_x,
+                              void *X_dev, uint8_t *xq, uint8_t *sfx, const uint8_t *wq,
+                              const uint8_t *sfw, const float *ts_w, int64_t N, void *Y_dev,
+                              void *Y_host, void *ws, size_t ws_bytes, void *stream);
+
 /* Integer fake-quant of Eq. 1-2 (quantize, dequantize, round to bf16), optional gather.
  *   T : bf16 [rows, K], ld.  out : bf16 [rows, K], ldo.  perm : int32 [K] or NULL.
  *   fmt.kind must be 1; K % fmt.group == 0; K <= 16384 when perm != NULL. */

@@ -49,6 +49,8 @@ _SIGNATURES = {
     "pq_gemm_w4a4": (_int, [_vp, _vp, _vp, _vp, _vp, _vp, _i64, _i64, _i64, _vp, _i64, _vp, _sz, _vp]),
     "pq_linear_w4a4": (_int, [_vp, _i64, _i64, _i64, _vp, _vp, _vp, _vp, _vp, _vp, _i64, _vp, _i64,
                               _vp, _sz, _vp]),
+    "pq_linear_w4a4_host": (_int, [_vp, _i64, _i64, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _i64, _vp, _vp,
+                                   _vp, _sz, _vp]),
     "pq_fakequant_int": (_int, [_vp, _i64, _i64, _i64, pq_format, _vp, _vp, _i64, _vp]),
     "pq_sf_to_linear": (_int, [_vp, _i64, _i64, _vp, _vp]),
     "pq_device_status": (_int, [_vp, _vp]),
@@ -198,6 +200,22 @@ def pq_linear_w4a4(X, ts_x, xq, sfx, wq, sfw, ts_w, Y, ws):
     w, wb = _ws(ws)
     _check("pq_linear_w4a4", lib().pq_linear_w4a4(_p(X), M, K, X.stride(0), _p(ts_x), _p(xq), _p(sfx), _p(wq),
                                                   _p(sfw), _p(ts_w), N, _p(Y), Y.stride(0), w, wb, _stream()))
+
+
+def pq_linear_w4a4_host(X_host, ts_x, X_dev, xq, sfx, wq, sfw, ts_w, Y_dev, Y_host, ws):
+    """Host tensors in, host tensor out (pinned CPU tensors); copies and kernels are enqueued on
+    the current stream, the caller synchronises before reading Y_host."""
+    assert not X_host.is_cuda and not Y_host.is_cuda and X_host.is_contiguous() and Y_host.is_contiguous()
+    assert X_host.dtype == torch.bfloat16 and Y_host.dtype == torch.bfloat16
+    _bf16(X_dev)
+    M, K = X_host.shape
+    N = wq.shape[0]
+    assert X_dev.shape == (M, K) and X_dev.is_contiguous() and Y_dev.shape == (M, N) and Y_dev.is_contiguous()
+    assert Y_host.shape == (M, N)
+    w, wb = _ws(ws)
+    _check("pq_linear_w4a4_host", lib().pq_linear_w4a4_host(
+        C.c_void_p(X_host.data_ptr()), M, K, _p(ts_x), _p(X_dev), _p(xq), _p(sfx), _p(wq), _p(sfw), _p(ts_w), N,
+        _p(Y_dev), C.c_void_p(Y_host.data_ptr()), w, wb, _stream()))
 
 
 def pq_fakequant_int(T, fmt, perm, out):

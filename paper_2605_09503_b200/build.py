@@ -38,7 +38,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
             cmd.insert(1, "-Xptxas=-v")
         subprocess.run(cmd, check=True)
         objs.append(obj)
-    subprocess.run(["nvcc", "-shared", "-cudart", "static", "-o", LIB, *objs, "-ldl", "-lpthread", "-lrt"], check=True)
+    subprocess.run(["nvcc", "-Wno-deprecated-gpu-targets", "-shared", "-cudart", "static", "-o", LIB, *objs, "-ldl", "-lpthread", "-lrt"], check=True)
     return LIB
 
 

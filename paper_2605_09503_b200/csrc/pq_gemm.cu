@@ -466,6 +466,20 @@ extern "C" pq_status pq_linear_w4a4(const void *X, int64_t M, int64_t K, int64_t
     return pq_gemm_w4a4(xq, sfx, ts_x, wq, sfw, ts_w, M, N, K, Y, ldy, ws, ws_bytes, stream);
 }
 
+extern "C" pq_status pq_linear_w4a4_host(const void *X_host, int64_t M, int64_t K, const float *ts_x, void *X_dev,
+                                         uint8_t *xq, uint8_t *sfx, const uint8_t *wq, const uint8_t *sfw,
+                                         const float *ts_w, int64_t N, void *Y_dev, void *Y_host, void *ws,
+                                         size_t ws_bytes, void *stream) {
+    PQ_REQUIRE(X_host && X_dev && Y_dev && Y_host, PQ_ERR_NULL);
+    PQ_REQUIRE(M > 0 && K > 0 && N > 0, PQ_ERR_SHAPE);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    PQ_CUDA_OK(cudaMemcpyAsync(X_dev, X_host, static_cast<size_t>(M) * K * 2, cudaMemcpyHostToDevice, st));
+    const pq_status rc = pq_linear_w4a4(X_dev, M, K, K, ts_x, xq, sfx, wq, sfw, ts_w, N, Y_dev, N, ws, ws_bytes, stream);
+    if (rc != PQ_OK) return rc;
+    PQ_CUDA_OK(cudaMemcpyAsync(Y_host, Y_dev, static_cast<size_t>(M) * N * 2, cudaMemcpyDeviceToHost, st));
+    return PQ_OK;
+}
+
 extern "C" pq_status pq_device_status(const void *ws, void *stream) {
     PQ_REQUIRE(ws, PQ_ERR_NULL);
     int word = 0;
