@@ -5,19 +5,23 @@
 // Design (one CTA per SM, persistent over output tiles of 128 x 192):
 //   warp 0      producer: TMA loads of the packed E2M1 operand tiles (128-byte swizzle) and bulk
 //               copies of the scale-factor blocks into a 4-stage shared-memory ring;
-//   warp 1      issues tcgen05.cp (scale factors: shared -> tensor memory) and
-//               tcgen05.mma.kind::mxf4nvf4.block_scale (K = 64 per instruction, 4 per stage) into one
-//               of two 128 x 192 fp32 accumulators in tensor memory;
+//   warp 1      issues tcgen05.mma.kind::mxf4nvf4.block_scale (K = 64 per instruction, 4 per stage)
+//               into one of two 128 x 192 fp32 accumulators in tensor memory;
 //   warps 2..5  epilogue: tcgen05.ld the finished accumulator, scale by ts_x*ts_w, round to bf16,
-//               store -- overlapping the next tile's main loop through the second accumulator.
+//               store -- overlapping the next tile's main loop through the second accumulator;
+//   warps 6..9  scale-factor stagers: read the stage's scale blocks from shared memory and write
+//               them into one of two scale slots in tensor memory with tcgen05.st (one warp per
+//               lane quadrant).  Measured on B200: a tcgen05.cp of one 512-byte block costs about
+//               80 cycles of the tensor pipe and twelve are needed per stage, more than the stage's
+//               four MMAs (384 cycles); the register path costs the pipe nothing.
 // K is consumed 256 channels (128 bytes of codes per row) per stage.  192 divides every FLUX
 // output width (3072, 9216, 12288) and leaves room in the 512 tensor-memory columns for two
 // accumulators plus the scale factors.
 //
-// Scale factors live in global memory in 512-byte blocks of 128 rows x 4 groups (see pq.h); one
-// tcgen05.cp.32x128b.warpx4 moves a block to 4 tensor-memory columns (row r of the block ->
-// lane r%32, column r/32, replicated over the four lane quadrants), which is the layout the MMA
-// reads.  A 192-wide tile that starts in the middle of a 128-row block (n0 % 128 == 64) loads
+// Scale factors live in global memory in 512-byte blocks of 128 rows x 4 groups (see pq.h); a
+// block occupies 4 tensor-memory columns (row r of the block -> lane r%32, column r/32, the same
+// in all four lane quadrants), which is the layout the MMA reads: lane l of every stager warp
+// loads the 16 bytes at offset 16 l of the block and stores them as 4 columns of its quadrant.  A 192-wide tile that starts in the middle of a 128-row block (n0 % 128 == 64) loads
 // the two blocks it touches and offsets the B scale address by two columns.
 //
 // Every wait on an mbarrier is bounded.  If one expires the CTA records PQ_ERR_TIMEOUT in the
@@ -37,12 +41,15 @@ constexpr int kSfBlock = 512;              // 128 rows x 4 groups
 constexpr int kSfaBytes = 4 * kSfBlock;    // 4 K-blocks of one 128-row block
 constexpr int kSfbBytes = 2 * kSfaBytes;   // two 128-row blocks
 constexpr int kStageBytes = kABytes + kBBytes + kSfaBytes + kSfbBytes;  // 47104 = 46 * 1024
-constexpr int kThreads = 192;
+constexpr int kThreads = 320;
 constexpr int kTmemCols = 512;
 constexpr uint32_t kAccStride = 256;  // accumulator b starts at column b * 256
-constexpr uint32_t kSfaCol = 192, kSfbCol = 208;
+// two scale slots in the columns the accumulators leave free: 16 columns of A scales, 32 of B scales
+__device__ __forceinline__ uint32_t sf_slot_col(uint32_t t) { return t ? 448u : 192u; }
+constexpr uint32_t kSfbOfs = 16;
 constexpr long long kWaitCycles = 4000000000ll;  // about two seconds of SM clock per wait
 constexpr size_t kSmemBytes = kStages * kStageBytes + 1024 /*alignment slack*/ + 256 /*barriers*/;
+constexpr int kNumBars = 2 * kStages + 6;  // full[S] empty[S] acc_full[2] acc_empty[2] sf_full[2]
 
 struct GemmParams {
     const uint8_t *sfx, *sfw;
@@ -113,8 +120,21 @@ __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::
 __device__ __forceinline__ void tc_commit(uint32_t bar) {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
-__device__ __forceinline__ void tc_cp_sf(uint32_t tmem_col, uint64_t desc) {
-    asm volatile("tcgen05.cp.cta_group::1.32x128b.warpx4 [%0], %1;" ::"r"(tmem_col), "l"(desc) : "memory");
+__device__ __forceinline__ void tc_st4(uint32_t taddr, const uint4 &v) {
+    asm volatile("tcgen05.st.sync.aligned.32x32b.x4.b32 [%0], {%1, %2, %3, %4};" ::"r"(taddr), "r"(v.x), "r"(v.y),
+                 "r"(v.z), "r"(v.w)
+                 : "memory");
+}
+__device__ __forceinline__ void tc_st8(uint32_t taddr, const uint4 &a, const uint4 &b) {
+    asm volatile("tcgen05.st.sync.aligned.32x32b.x8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"r"(taddr),
+                 "r"(a.x), "r"(a.y), "r"(a.z), "r"(a.w), "r"(b.x), "r"(b.y), "r"(b.z), "r"(b.w)
+                 : "memory");
+}
+__device__ __forceinline__ void tc_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ uint4 lds128(uint32_t addr) {
+    uint4 v;
+    asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
+    return v;
 }
 __device__ __forceinline__ void tc_mma(uint32_t d_tmem, uint64_t da, uint64_t db, uint32_t idesc, uint32_t sfa,
                                        uint32_t sfb, uint32_t accumulate) {
@@ -147,10 +167,6 @@ __device__ __forceinline__ uint64_t operand_desc(uint32_t smem_addr) {
     return static_cast<uint64_t>((smem_addr & 0x3FFFFu) >> 4) | (1ull << 16) | (64ull << 32) | (1ull << 46) |
            (2ull << 61);
 }
-// Descriptor of one 512-byte scale block: 32 rows of 16 bytes, no swizzle, 8-row groups 128 bytes apart.
-__device__ __forceinline__ uint64_t sf_desc(uint32_t smem_addr) {
-    return static_cast<uint64_t>((smem_addr & 0x3FFFFu) >> 4) | (8ull << 32) | (1ull << 46);
-}
 // Instruction descriptor: E2M1 x E2M1, UE4M3 scales, both K-major, M = 128, N = BN, K = 64.
 constexpr uint32_t kIdesc = (1u << 7) | (1u << 10) | (static_cast<uint32_t>(BN >> 3) << 17) | (0u << 23) |
                             (static_cast<uint32_t>(BM >> 4) << 24);
@@ -165,13 +181,14 @@ gemm_w4a4_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
     uint8_t *base_ptr = smem_raw + (base - raw);
     const uint32_t bars = base + kStages * kStageBytes;
     uint8_t *bars_ptr = base_ptr + kStages * kStageBytes;
-    // barrier block: full[S] | empty[S] | acc_full[2] | acc_empty[2] | tmem base | abort flag
+    // barrier block: full[S] | empty[S] | acc_full[2] | acc_empty[2] | sf_full[2] | tmem base | abort flag
     auto full_bar = [&](int s) { return bars + 8u * s; };
     auto empty_bar = [&](int s) { return bars + 8u * (kStages + s); };
     auto acc_full_bar = [&](int b) { return bars + 8u * (2 * kStages + b); };
     auto acc_empty_bar = [&](int b) { return bars + 8u * (2 * kStages + 2 + b); };
-    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars_ptr + 8 * (2 * kStages + 4));
-    volatile int *abort_flag = reinterpret_cast<volatile int *>(bars_ptr + 8 * (2 * kStages + 4) + 8);
+    auto sf_full_bar = [&](int t) { return bars + 8u * (2 * kStages + 4 + t); };
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars_ptr + 8 * kNumBars);
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(bars_ptr + 8 * kNumBars + 8);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
@@ -183,6 +200,7 @@ gemm_w4a4_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
         for (int b = 0; b < 2; ++b) {
             mbar_init(acc_full_bar(b), 1);
             mbar_init(acc_empty_bar(b), 4);
+            mbar_init(sf_full_bar(b), 4);
         }
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -255,41 +273,30 @@ gemm_w4a4_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
             if (!mbar_wait(acc_empty_bar(b), accpar ^ 1u, abort_flag, p.status)) break;
             tc_fence_after();
             const uint32_t d_tmem = tmem_base + b * kAccStride;
-            const uint32_t sfa_t = tmem_base + kSfaCol, sfb_t = tmem_base + kSfbCol;
             for (int kt = 0; kt < p.k_tiles; ++kt, ++it) {
                 const int s = it % kStages;
                 const uint32_t par = (it / kStages) & 1u;
-                if (!mbar_wait(full_bar(s), par, abort_flag, p.status)) {
+                const uint32_t t = it & 1u;
+                if (!mbar_wait(full_bar(s), par, abort_flag, p.status) ||
+                    !mbar_wait(sf_full_bar(t), (it >> 1) & 1u, abort_flag, p.status)) {
                     ok = false;
                     break;
                 }
+                tc_fence_after();
                 const int kb_valid = min(4, p.kb_total - kt * 4);
                 const uint32_t stage = base + s * kStageBytes;
                 const uint64_t da = operand_desc(stage), db = operand_desc(stage + kABytes);
-                const uint64_t dsa = sf_desc(stage + kABytes + kBBytes);
-                const uint64_t dsb0 = sf_desc(stage + kABytes + kBBytes + kSfaBytes);
-                const uint64_t dsb1 = sf_desc(stage + kABytes + kBBytes + 2 * kSfaBytes);
+                const uint32_t sfa_t = tmem_base + sf_slot_col(t), sfb_t = sfa_t + kSfbOfs + sfb_shift;
                 if (lane == 0) {
                     if (kb_valid == 4) {
 #pragma unroll
-                        for (int kk = 0; kk < 4; ++kk) {
-                            tc_cp_sf(sfa_t + 4 * kk, dsa + kk * (kSfBlock >> 4));
-                            tc_cp_sf(sfb_t + 8 * kk, dsb0 + kk * (kSfBlock >> 4));
-                            tc_cp_sf(sfb_t + 8 * kk + 4, dsb1 + kk * (kSfBlock >> 4));
-                        }
-#pragma unroll
                         for (int kk = 0; kk < 4; ++kk)
-                            tc_mma(d_tmem, da + 2 * kk, db + 2 * kk, kIdesc, sfa_t + 4 * kk,
-                                   sfb_t + 8 * kk + sfb_shift, (kt | kk) ? 1u : 0u);
+                            tc_mma(d_tmem, da + 2 * kk, db + 2 * kk, kIdesc, sfa_t + 4 * kk, sfb_t + 8 * kk,
+                                   (kt | kk) ? 1u : 0u);
                     } else {
-                        for (int kk = 0; kk < kb_valid; ++kk) {
-                            tc_cp_sf(sfa_t + 4 * kk, dsa + kk * (kSfBlock >> 4));
-                            tc_cp_sf(sfb_t + 8 * kk, dsb0 + kk * (kSfBlock >> 4));
-                            tc_cp_sf(sfb_t + 8 * kk + 4, dsb1 + kk * (kSfBlock >> 4));
-                        }
                         for (int kk = 0; kk < kb_valid; ++kk)
-                            tc_mma(d_tmem, da + 2 * kk, db + 2 * kk, kIdesc, sfa_t + 4 * kk,
-                                   sfb_t + 8 * kk + sfb_shift, (kt | kk) ? 1u : 0u);
+                            tc_mma(d_tmem, da + 2 * kk, db + 2 * kk, kIdesc, sfa_t + 4 * kk, sfb_t + 8 * kk,
+                                   (kt | kk) ? 1u : 0u);
                     }
                     tc_commit(empty_bar(s));
                 }
@@ -297,6 +304,41 @@ gemm_w4a4_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
             }
             if (ok && lane == 0) tc_commit(acc_full_bar(b));
             __syncwarp();
+        }
+    } else if (warp >= 6) {
+        // ------------------------------------------------------------ scale-factor stagers
+        const uint32_t q = warp & 3;  // tensor-memory lane quadrant this warp may write
+        const uint32_t lane_ofs = (q * 32u) << 16;
+        uint32_t it = 0;
+        bool ok = true;
+        for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
+            for (int kt = 0; kt < p.k_tiles; ++kt, ++it) {
+                const int s = it % kStages;
+                const uint32_t t = it & 1u;
+                // the stage's scale blocks have landed, and the MMAs that read this slot two
+                // iterations ago have completed (their commit released that iteration's stage)
+                if (!mbar_wait(full_bar(s), (it / kStages) & 1u, abort_flag, p.status) ||
+                    (it >= 2 && !mbar_wait(empty_bar((it - 2) % kStages), ((it - 2) / kStages) & 1u, abort_flag,
+                                           p.status))) {
+                    ok = false;
+                    break;
+                }
+                tc_fence_after();
+                const int kb_valid = min(4, p.kb_total - kt * 4);
+                const uint32_t sf_s = base + s * kStageBytes + kABytes + kBBytes + lane * 16u;
+                const uint32_t sf_t = tmem_base + lane_ofs + sf_slot_col(t);
+                for (int kk = 0; kk < kb_valid; ++kk) {
+                    const uint4 a = lds128(sf_s + kk * kSfBlock);
+                    const uint4 b0 = lds128(sf_s + kSfaBytes + kk * kSfBlock);
+                    const uint4 b1 = lds128(sf_s + 2 * kSfaBytes + kk * kSfBlock);
+                    tc_st4(sf_t + 4 * kk, a);
+                    tc_st8(sf_t + kSfbOfs + 8 * kk, b0, b1);
+                }
+                tc_wait_st();
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(sf_full_bar(t));
+            }
         }
     } else {
         // ------------------------------------------------------------ epilogue
