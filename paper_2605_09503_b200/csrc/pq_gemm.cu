@@ -2,69 +2,121 @@
 //
 //   Y[m,n] = bf16( ts_x*ts_w * sum_k (qx[m,k]*sfx[m,k/16]) * (qw[n,k]*sfw[n,k/16]) )
 //
-// Design (one CTA per SM, persistent over output tiles of 128 x 192):
-//   warp 0      producer: TMA loads of the packed E2M1 operand tiles (128-byte swizzle) and bulk
-//               copies of the scale-factor blocks into a 4-stage shared-memory ring;
-//   warp 1      issues tcgen05.mma.kind::mxf4nvf4.block_scale (K = 64 per instruction, 4 per stage)
-//               into one of two 128 x 192 fp32 accumulators in tensor memory;
-//   warps 2..5  epilogue: tcgen05.ld the finished accumulator, scale by ts_x*ts_w, round to bf16,
-//               store -- overlapping the next tile's main loop through the second accumulator;
-//   warps 6..9  scale-factor stagers: read the stage's scale blocks from shared memory and write
-//               them into one of two scale slots in tensor memory with tcgen05.st (one warp per
-//               lane quadrant).  Measured on B200: a tcgen05.cp of one 512-byte block costs about
-//               80 cycles of the tensor pipe and twelve are needed per stage, more than the stage's
-//               four MMAs (384 cycles); the register path costs the pipe nothing.
-// K is consumed 256 channels (128 bytes of codes per row) per stage.  192 divides every FLUX
-// output width (3072, 9216, 12288) and leaves room in the 512 tensor-memory columns for two
-// accumulators plus the scale factors.
+// Design.  Thread-block clusters of two CTAs (one per SM) work as a pair on output tiles of
+// 256 x 192, persistent over the tile list: tcgen05.mma.cta_group::2 lets each CTA hold 128 rows
+// of the accumulator while the B operand is split between the two shared memories, so a CTA
+// fetches 128 rows of X codes and only 96 rows of W codes per 256-channel K step -- a quarter
+// less L2->SM traffic than two independent 128 x 192 tiles.  Roles of the 14 warps of a CTA:
+//   warp 0       producer: TMA loads of the packed E2M1 operand tiles (128-byte swizzle) and bulk
+//                copies of the scale-factor blocks into a 5-stage shared-memory ring.  Operand
+//                loads of both CTAs signal the pair leader's barrier (cp.async.bulk.tensor with
+//                .cta_group::2).
+//   warp 1       (leader CTA) issues tcgen05.mma.kind::mxf4nvf4.block_scale, K = 64 per instruction,
+//                4 per stage, into one of two 192-column fp32 accumulators in tensor memory.
+//   warps 2..5   epilogue: tcgen05.ld the finished accumulator (own CTA's 128 rows), scale by
+//                ts_x*ts_w, round to bf16, stage 32 x 64 boxes in swizzled shared memory and write
+//                them with TMA stores (full 128-byte lines) -- overlapping the next tile's main
+//                loop through the second accumulator.
+//   warps 6..13  scale-factor stagers: read the stage's scale blocks from shared memory and write
+//                them into one of three scale slots in tensor memory with tcgen05.st (one warp per
+//                lane quadrant; two sets of four warps take alternate K iterations).
+// 192 divides every FLUX output width (3072, 9216, 12288) and leaves room in the 512 tensor-memory
+// columns for two accumulators (384) plus three scale slots (3 x 40).
+//
+// Measurements on B200 behind these choices:
+//   - a tcgen05.cp of one 512-byte scale block occupies the tensor pipe for about 80 cycles and
+//     twelve are needed per stage, more than the stage's four MMAs (384 cycles); the register path
+//     (ld.shared + tcgen05.st, 7 to 16 cycles per store) costs the pipe nothing;
+//   - TMA and tcgen05 instructions take their operands from uniform registers.  Issued from a
+//     divergent single-lane loop (`if (lane == 0) for (...)`) every operand is moved there one by
+//     one and an MMA costs about 190 cycles of issue time instead of 96; the producer and the MMA
+//     issuer therefore run their loops with the whole warp and single out one lane with
+//     elect.sync only around those instructions;
+//   - a remote mbarrier arrive with cluster-scope release semantics costs 500 to 2500 cycles;
+//     what the arrivals here publish has already completed (tcgen05.wait) when they are issued,
+//     so the default semantics are used.
 //
 // Scale factors live in global memory in 512-byte blocks of 128 rows x 4 groups (see pq.h); a
 // block occupies 4 tensor-memory columns (row r of the block -> lane r%32, column r/32, the same
 // in all four lane quadrants), which is the layout the MMA reads: lane l of every stager warp
-// loads the 16 bytes at offset 16 l of the block and stores them as 4 columns of its quadrant.  A 192-wide tile that starts in the middle of a 128-row block (n0 % 128 == 64) loads
-// the two blocks it touches and offsets the B scale address by two columns.
+// loads the 16 bytes at offset 16 l of the block and stores them as columns of its quadrant.
+// The 192 B-scale rows of a tile span two blocks; the stagers pick the six 32-row words that
+// belong to the tile (it may start in the middle of a block) and store them as 6 columns.
 //
-// Every wait on an mbarrier is bounded.  If one expires the CTA records PQ_ERR_TIMEOUT in the
-// status word, raises a shared abort flag that every role polls, drains its outstanding loads
-// (bounded), frees its tensor memory and returns.
+// Cross-CTA signalling uses plain remote mbarrier arrives: the MMA issuer commits to barriers of
+// its own CTA only, and the leader's producer (stages) and epilogue (accumulators) pass each
+// completion on to the peer.  Every wait on an mbarrier is bounded.  If one expires the CTA
+// records PQ_ERR_TIMEOUT in the status word, raises a shared abort flag that every role polls,
+// and falls through to the common teardown (cluster barrier, tensor-memory release).
 #include <cuda.h>
 
 #include "pq_common.cuh"
 
 namespace {
 
-constexpr int BM = 128, BN = 192, BK = 256;
-constexpr int kStages = 4;
-constexpr int kABytes = BM * BK / 2;       // 16384
-constexpr int kBBytes = BN * BK / 2;       // 24576
+constexpr int BM = 256, BM_CTA = 128, BN = 192, BN_CTA = BN / 2, BK = 256;
+constexpr int kStages = 5;
+constexpr int kABytes = BM_CTA * BK / 2;   // 16384
+constexpr int kBBytes = BN_CTA * BK / 2;   // 12288
 constexpr int kSfBlock = 512;              // 128 rows x 4 groups
 constexpr int kSfaBytes = 4 * kSfBlock;    // 4 K-blocks of one 128-row block
 constexpr int kSfbBytes = 2 * kSfaBytes;   // two 128-row blocks
-constexpr int kStageBytes = kABytes + kBBytes + kSfaBytes + kSfbBytes;  // 47104 = 46 * 1024
-constexpr int kThreads = 320;
+constexpr int kStageBytes = kABytes + kBBytes + kSfaBytes + kSfbBytes;  // 34816 = 34 * 1024
+constexpr int kEpiBox = 32 * 128;          // 32 rows x 64 bf16, one TMA store
+constexpr int kEpiBytes = 4 * 2 * kEpiBox; // two boxes per epilogue warp
+constexpr int kThreads = 448;              // producer, MMA issuer, 4 epilogue and 8 stager warps
 constexpr int kTmemCols = 512;
-constexpr uint32_t kAccStride = 256;  // accumulator b starts at column b * 256
-// two scale slots in the columns the accumulators leave free: 16 columns of A scales, 32 of B scales
-__device__ __forceinline__ uint32_t sf_slot_col(uint32_t t) { return t ? 448u : 192u; }
-constexpr uint32_t kSfbOfs = 16;
+constexpr uint32_t kAccStride = BN;        // accumulator b starts at column b * 192
+// Three scale slots follow the accumulators.  A slot holds the scales of one stage: per 64-channel
+// K block 4 columns of A scales (128 rows) and 6 columns of B scales (192 rows).
+constexpr int kSfSlots = 3;
+constexpr uint32_t kSfSlotCol0 = 2 * BN, kSfSlotCols = 4 * (4 + 6), kSfbOfs = 16;
+static_assert(kSfSlotCol0 + kSfSlots * kSfSlotCols <= 512, "tensor memory columns");
 constexpr long long kWaitCycles = 4000000000ll;  // about two seconds of SM clock per wait
-constexpr size_t kSmemBytes = kStages * kStageBytes + 1024 /*alignment slack*/ + 256 /*barriers*/;
-constexpr int kNumBars = 2 * kStages + 6;  // full[S] empty[S] acc_full[2] acc_empty[2] sf_full[2]
+// barriers: stage_full[S] sf_ready[S] stage_free[S] acc_full[2] acc_empty[2]
+constexpr int kNumBars = 3 * kStages + 4;
+constexpr size_t kSmemBytes = kStages * kStageBytes + kEpiBytes + 1024 /*alignment slack*/ + 8 * kNumBars + 64;
 
 struct GemmParams {
     const uint8_t *sfx, *sfw;
     const float *ts_x, *ts_w;
-    uint16_t *Y;
-    int64_t ldy;
     int M, N, K;
     int m_tiles, n_tiles, k_tiles, kb_total, kb4;
-    int n_rowblocks;
+    int m_rowblocks, n_rowblocks;
     int *status;
 };
 
 // ---------------------------------------------------------------- PTX wrappers
 __device__ __forceinline__ uint32_t smem_u32(const void *p) {
     return static_cast<uint32_t>(__cvta_generic_to_shared(p));
+}
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+// Address of the same shared-memory location in CTA `rank` of the cluster.
+__device__ __forceinline__ uint32_t mapa(uint32_t addr, uint32_t rank) {
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
+    return r;
+}
+// One lane of a converged warp; the branch on it stays friendly to uniform registers.
+__device__ __forceinline__ bool elect_one() {
+    uint32_t pred = 0;
+    asm volatile(
+        "{\n"
+        ".reg .b32 rx;\n"
+        ".reg .pred px;\n"
+        "elect.sync rx|px, %1;\n"
+        "@px mov.s32 %0, 1;\n"
+        "}\n"
+        : "+r"(pred)
+        : "r"(0xFFFFFFFFu));
+    return pred != 0;
+}
+__device__ __forceinline__ void cluster_sync() {
+    asm volatile("barrier.cluster.arrive.release.aligned;\nbarrier.cluster.wait.acquire.aligned;" ::: "memory");
 }
 __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
     asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
@@ -74,6 +126,21 @@ __device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
 }
 __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+// Arrive on the copy of a barrier in CTA `rank` of the pair.
+__device__ __forceinline__ void mbar_arrive_remote(uint32_t bar, uint32_t rank) {
+    asm volatile(
+        "{\n"
+        ".reg .b32 remote;\n"
+        "mapa.shared::cluster.u32 remote, %0, %1;\n"
+        "mbarrier.arrive.shared::cluster.b64 _, [remote];\n"
+        "}\n" ::"r"(bar), "r"(rank)
+        : "memory");
+}
+// Arrive on the pair leader's copy of a barrier.
+__device__ __forceinline__ void mbar_arrive_leader(uint32_t bar, uint32_t rank) {
+    if (rank == 0) mbar_arrive(bar);
+    else mbar_arrive_remote(bar, 0);
 }
 __device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
     uint32_t ok;
@@ -90,8 +157,7 @@ __device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
 }
 // Bounded wait: polls until the phase completes, the abort flag goes up, or kWaitCycles SM
 // clock cycles have passed (then it raises the flag and records the timeout).
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag, int *status) {
-    if (mbar_try(bar, parity)) return true;
+__device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volatile int *abort_flag, int *status) {
     const long long t0 = clock64();
     for (uint32_t spins = 1;; ++spins) {
         if (mbar_try(bar, parity)) return true;
@@ -104,10 +170,17 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
     atomicExch(status, static_cast<int>(PQ_ERR_TIMEOUT));
     return false;
 }
-__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map, int x, int y, uint32_t bar) {
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag, int *status) {
+    if (mbar_try(bar, parity)) return true;
+    return mbar_wait_slow(bar, parity, abort_flag, status);
+}
+// Operand tile load of a CTA pair: data lands in this CTA's shared memory, the byte count is
+// credited to the barrier at `bar_cluster` (the pair leader's).
+__device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap *map, int x, int y,
+                                                 uint32_t bar_cluster) {
     asm volatile(
-        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
-        ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar)
+        "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+        ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar_cluster)
         : "memory");
 }
 __device__ __forceinline__ void bulk_load(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar) {
@@ -115,34 +188,32 @@ __device__ __forceinline__ void bulk_load(uint32_t dst, const void *src, uint32_
                  ::"r"(dst), "l"(src), "r"(bytes), "r"(bar)
                  : "memory");
 }
+__device__ __forceinline__ void tma_store_2d(const CUtensorMap *map, int x, int y, uint32_t src) {
+    asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%1, %2}], [%3];"
+                 ::"l"(map), "r"(x), "r"(y), "r"(src)
+                 : "memory");
+}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void bulk_wait_read() {
+    asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory");
+}
+__device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_commit(uint32_t bar) {
-    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+// Arrive on `bar` (this CTA's) once every tcgen05 operation issued so far by this thread has
+// completed in both CTAs of the pair.
+__device__ __forceinline__ void tc_commit_pair(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
-__device__ __forceinline__ void tc_st4(uint32_t taddr, const uint4 &v) {
-    asm volatile("tcgen05.st.sync.aligned.32x32b.x4.b32 [%0], {%1, %2, %3, %4};" ::"r"(taddr), "r"(v.x), "r"(v.y),
-                 "r"(v.z), "r"(v.w)
-                 : "memory");
-}
-__device__ __forceinline__ void tc_st8(uint32_t taddr, const uint4 &a, const uint4 &b) {
-    asm volatile("tcgen05.st.sync.aligned.32x32b.x8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"r"(taddr),
-                 "r"(a.x), "r"(a.y), "r"(a.z), "r"(a.w), "r"(b.x), "r"(b.y), "r"(b.z), "r"(b.w)
-                 : "memory");
-}
-__device__ __forceinline__ void tc_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
-__device__ __forceinline__ uint4 lds128(uint32_t addr) {
-    uint4 v;
-    asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
-    return v;
-}
-__device__ __forceinline__ void tc_mma(uint32_t d_tmem, uint64_t da, uint64_t db, uint32_t idesc, uint32_t sfa,
-                                       uint32_t sfb, uint32_t accumulate) {
+__device__ __forceinline__ void tc_mma_pair(uint32_t d_tmem, uint64_t da, uint64_t db, uint32_t idesc, uint32_t sfa,
+                                            uint32_t sfb, uint32_t accumulate) {
     asm volatile(
         "{\n"
         ".reg .pred p;\n"
         "setp.ne.b32 p, %4, 0;\n"
-        "tcgen05.mma.cta_group::1.kind::mxf4nvf4.block_scale.block16 [%0], %1, %2, %3, [%5], [%6], p;\n"
+        "tcgen05.mma.cta_group::2.kind::mxf4nvf4.block_scale.block16 [%0], %1, %2, %3, [%5], [%6], p;\n"
         "}\n"
         ::"r"(d_tmem), "l"(da), "l"(db), "r"(idesc), "r"(accumulate), "r"(sfa), "r"(sfb)
         : "memory");
@@ -160,6 +231,34 @@ __device__ __forceinline__ void tc_ld32(uint32_t taddr, uint32_t (&v)[32]) {
         : "memory");
 }
 __device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void tc_st4(uint32_t taddr, const uint4 &v) {
+    asm volatile("tcgen05.st.sync.aligned.32x32b.x4.b32 [%0], {%1, %2, %3, %4};" ::"r"(taddr), "r"(v.x), "r"(v.y),
+                 "r"(v.z), "r"(v.w)
+                 : "memory");
+}
+__device__ __forceinline__ void tc_st2(uint32_t taddr, uint32_t a, uint32_t b) {
+    asm volatile("tcgen05.st.sync.aligned.32x32b.x2.b32 [%0], {%1, %2};" ::"r"(taddr), "r"(a), "r"(b) : "memory");
+}
+// Six columns of B scales of one K block: the 32-row words of the tile's 192 rows, picked from the
+// two 128-row blocks the tile touches (`mid`: the tile starts in the middle of the first block).
+__device__ __forceinline__ void stage_b_scales(uint32_t taddr, const uint4 &b0, const uint4 &b1, bool mid) {
+    if (mid) {
+        tc_st4(taddr, make_uint4(b0.z, b0.w, b1.x, b1.y));
+        tc_st2(taddr + 4, b1.z, b1.w);
+    } else {
+        tc_st4(taddr, b0);
+        tc_st2(taddr + 4, b1.x, b1.y);
+    }
+}
+__device__ __forceinline__ void tc_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ uint4 lds128(uint32_t addr) {
+    uint4 v;
+    asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
+    return v;
+}
+__device__ __forceinline__ void sts128(uint32_t addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
+    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
+}
 
 // Shared-memory matrix descriptor of a K-major operand tile with 128-byte swizzle: rows of
 // 128 bytes, 8-row groups 1024 bytes apart.
@@ -167,52 +266,68 @@ __device__ __forceinline__ uint64_t operand_desc(uint32_t smem_addr) {
     return static_cast<uint64_t>((smem_addr & 0x3FFFFu) >> 4) | (1ull << 16) | (64ull << 32) | (1ull << 46) |
            (2ull << 61);
 }
-// Instruction descriptor: E2M1 x E2M1, UE4M3 scales, both K-major, M = 128, N = BN, K = 64.
+// Instruction descriptor: E2M1 x E2M1, UE4M3 scales, both K-major, M = 256 (pair), N = BN, K = 64.
 constexpr uint32_t kIdesc = (1u << 7) | (1u << 10) | (static_cast<uint32_t>(BN >> 3) << 17) | (0u << 23) |
                             (static_cast<uint32_t>(BM >> 4) << 24);
 
+__device__ __forceinline__ uint32_t sf_slot_col(uint32_t t) { return kSfSlotCol0 + t * kSfSlotCols; }
+
+// Two accumulator values times alpha, each rounded to bf16 (nearest even), packed low | high.
+__device__ __forceinline__ uint32_t pack_bf16(uint32_t lo_bits, uint32_t hi_bits, float alpha) {
+    const float lo = __fmul_rn(__uint_as_float(lo_bits), alpha);
+    const float hi = __fmul_rn(__uint_as_float(hi_bits), alpha);
+    uint32_t r;
+    asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+    return r;
+}
+
 // ---------------------------------------------------------------- kernel
-__global__ void __launch_bounds__(kThreads, 1)
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
 gemm_w4a4_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
-                 const GemmParams p) {
+                 const __grid_constant__ CUtensorMap map_y, const GemmParams p) {
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
-    const uint32_t base = (raw + 1023u) & ~1023u;
+    const uint32_t base = (raw + 1023u) & ~1023u;  // identical in both CTAs of the pair
     uint8_t *base_ptr = smem_raw + (base - raw);
-    const uint32_t bars = base + kStages * kStageBytes;
-    uint8_t *bars_ptr = base_ptr + kStages * kStageBytes;
-    // barrier block: full[S] | empty[S] | acc_full[2] | acc_empty[2] | sf_full[2] | tmem base | abort flag
-    auto full_bar = [&](int s) { return bars + 8u * s; };
-    auto empty_bar = [&](int s) { return bars + 8u * (kStages + s); };
-    auto acc_full_bar = [&](int b) { return bars + 8u * (2 * kStages + b); };
-    auto acc_empty_bar = [&](int b) { return bars + 8u * (2 * kStages + 2 + b); };
-    auto sf_full_bar = [&](int t) { return bars + 8u * (2 * kStages + 4 + t); };
+    const uint32_t epi = base + kStages * kStageBytes;
+    const uint32_t bars = epi + kEpiBytes;
+    uint8_t *bars_ptr = base_ptr + kStages * kStageBytes + kEpiBytes;
+    // stage_full: operand bytes of both CTAs have landed (1 arrival + transaction bytes) and the
+    // stage's scales are in tensor memory in both CTAs (8 stager-warp arrivals); leader's copy only
+    auto stage_full_bar = [&](int s) { return bars + 8u * s; };
+    auto sf_ready_bar = [&](int s) { return bars + 8u * (kStages + s); };     // scale blocks landed (own CTA)
+    auto stage_free_bar = [&](int s) { return bars + 8u * (2 * kStages + s); };  // the stage's MMAs have run
+    auto acc_full_bar = [&](int b) { return bars + 8u * (3 * kStages + b); };
+    auto acc_empty_bar = [&](int b) { return bars + 8u * (3 * kStages + 2 + b); };  // leader's copy only
     uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars_ptr + 8 * kNumBars);
     volatile int *abort_flag = reinterpret_cast<volatile int *>(bars_ptr + 8 * kNumBars + 8);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t rank = cluster_ctarank();  // 0 = pair leader
+    const int pair = blockIdx.x >> 1, num_pairs = gridDim.x >> 1;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < kStages; ++s) {
-            mbar_init(full_bar(s), 1);
-            mbar_init(empty_bar(s), 1);
+            mbar_init(stage_full_bar(s), 9);  // producer + 4 stager warps in each CTA
+            mbar_init(sf_ready_bar(s), 1);
+            mbar_init(stage_free_bar(s), 1);
         }
         for (int b = 0; b < 2; ++b) {
             mbar_init(acc_full_bar(b), 1);
-            mbar_init(acc_empty_bar(b), 4);
-            mbar_init(sf_full_bar(b), 4);
+            mbar_init(acc_empty_bar(b), 8);  // 4 epilogue warps in each CTA
         }
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == 1) {
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
+        asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
                      "r"(kTmemCols)
                      : "memory");
-        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
     }
     tc_fence_before();
     __syncthreads();
+    cluster_sync();  // both CTAs' barriers are initialised before anyone signals across
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
 
@@ -220,106 +335,123 @@ gemm_w4a4_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
 
     if (warp == 0) {
         // ------------------------------------------------------------ producer
-        if (lane == 0) {
-            uint32_t it = 0;
-            bool ok = true;
-            for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
-                const int m_blk = tile % p.m_tiles, n_blk = tile / p.m_tiles;
-                const int m0 = m_blk * BM, n0 = n_blk * BN;
-                const int nb0 = n0 >> 7;
-                const int rb0 = min(nb0, p.n_rowblocks - 1), rb1 = min(nb0 + 1, p.n_rowblocks - 1);
-                for (int kt = 0; kt < p.k_tiles; ++kt, ++it) {
-                    const int s = it % kStages;
-                    const uint32_t par = (it / kStages) & 1u;
-                    if (!mbar_wait(empty_bar(s), par ^ 1u, abort_flag, p.status)) {
-                        ok = false;
-                        break;
-                    }
-
-                    const int kb_valid = min(4, p.kb_total - kt * 4);
-                    const uint32_t sf_bytes = static_cast<uint32_t>(kb_valid) * kSfBlock;
-                    const uint32_t stage = base + s * kStageBytes;
-                    mbar_expect_tx(full_bar(s), kABytes + kBBytes + 3u * sf_bytes);
-                    tma_load_2d(stage, &map_a, kt * (BK / 2), m0, full_bar(s));
-                    tma_load_2d(stage + kABytes, &map_b, kt * (BK / 2), n0, full_bar(s));
-                    const int64_t kofs = static_cast<int64_t>(kt) * 4 * kSfBlock;
-                    bulk_load(stage + kABytes + kBBytes,
-                              p.sfx + static_cast<int64_t>(m_blk) * p.kb4 * kSfBlock + kofs, sf_bytes, full_bar(s));
-                    bulk_load(stage + kABytes + kBBytes + kSfaBytes,
-                              p.sfw + static_cast<int64_t>(rb0) * p.kb4 * kSfBlock + kofs, sf_bytes, full_bar(s));
-                    bulk_load(stage + kABytes + kBBytes + kSfaBytes + kSfaBytes,
-                              p.sfw + static_cast<int64_t>(rb1) * p.kb4 * kSfBlock + kofs, sf_bytes, full_bar(s));
-                }
-            }
-            if (!ok) {
-                // drain: give every load already issued a bounded chance to land before leaving
-                const uint32_t issued = it;
-                const uint32_t first = issued > kStages ? issued - kStages : 0;
-                for (uint32_t j = first; j < issued; ++j)
-                    for (uint32_t i = 0; i < 4096 && !mbar_try(full_bar(j % kStages), (j / kStages) & 1u); ++i) {}
-            }
-        }
-        __syncwarp();
-    } else if (warp == 1) {
-        // ------------------------------------------------------------ MMA issuer
-        // The whole warp walks the loop (uniform control flow, so descriptors live in uniform
-        // registers); lane 0 issues the tensor-core instructions.
-        uint32_t it = 0, tcount = 0;
+        uint32_t it = 0;
         bool ok = true;
-        for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++tcount) {
-            const int n_blk = tile / p.m_tiles;
-            const uint32_t sfb_shift = ((n_blk * BN) & 127) ? 2u : 0u;
-            const uint32_t b = tcount & 1u, accpar = (tcount >> 1) & 1u;
-            if (!mbar_wait(acc_empty_bar(b), accpar ^ 1u, abort_flag, p.status)) break;
-            tc_fence_after();
-            const uint32_t d_tmem = tmem_base + b * kAccStride;
+        for (int tile = pair; tile < total_tiles && ok; tile += num_pairs) {
+            const int m_blk = tile % p.m_tiles, n_blk = tile / p.m_tiles;
+            const int m0 = m_blk * BM + static_cast<int>(rank) * BM_CTA;
+            const int n0 = n_blk * BN;
+            const int ra = min(m0 >> 7, p.m_rowblocks - 1);
+            const int nb0 = n0 >> 7;
+            const int rb0 = min(nb0, p.n_rowblocks - 1), rb1 = min(nb0 + 1, p.n_rowblocks - 1);
+            const uint8_t *sfa_src = p.sfx + static_cast<int64_t>(ra) * p.kb4 * kSfBlock;
+            const uint8_t *sfb0_src = p.sfw + static_cast<int64_t>(rb0) * p.kb4 * kSfBlock;
+            const uint8_t *sfb1_src = p.sfw + static_cast<int64_t>(rb1) * p.kb4 * kSfBlock;
             for (int kt = 0; kt < p.k_tiles; ++kt, ++it) {
                 const int s = it % kStages;
                 const uint32_t par = (it / kStages) & 1u;
-                const uint32_t t = it & 1u;
-                if (!mbar_wait(full_bar(s), par, abort_flag, p.status) ||
-                    !mbar_wait(sf_full_bar(t), (it >> 1) & 1u, abort_flag, p.status)) {
-                    ok = false;
-                    break;
-                }
-                tc_fence_after();
+                ok = __all_sync(0xFFFFFFFFu, mbar_wait(stage_free_bar(s), par ^ 1u, abort_flag, p.status));
+                if (!ok) break;
                 const int kb_valid = min(4, p.kb_total - kt * 4);
+                const uint32_t sf_bytes = static_cast<uint32_t>(kb_valid) * kSfBlock;
                 const uint32_t stage = base + s * kStageBytes;
-                const uint64_t da = operand_desc(stage), db = operand_desc(stage + kABytes);
-                const uint32_t sfa_t = tmem_base + sf_slot_col(t), sfb_t = sfa_t + kSfbOfs + sfb_shift;
-                if (lane == 0) {
-                    if (kb_valid == 4) {
-#pragma unroll
-                        for (int kk = 0; kk < 4; ++kk)
-                            tc_mma(d_tmem, da + 2 * kk, db + 2 * kk, kIdesc, sfa_t + 4 * kk, sfb_t + 8 * kk,
-                                   (kt | kk) ? 1u : 0u);
-                    } else {
-                        for (int kk = 0; kk < kb_valid; ++kk)
-                            tc_mma(d_tmem, da + 2 * kk, db + 2 * kk, kIdesc, sfa_t + 4 * kk, sfb_t + 8 * kk,
-                                   (kt | kk) ? 1u : 0u);
-                    }
-                    tc_commit(empty_bar(s));
+                const uint32_t full_leader = mapa(stage_full_bar(s), 0);
+                const int64_t kofs = static_cast<int64_t>(kt) * 4 * kSfBlock;
+                if (elect_one()) {
+                    // the MMA issuer signals only its own CTA; pass each completion on to the peer
+                    if (rank == 0 && it >= kStages) mbar_arrive_remote(stage_free_bar(s), 1);
+                    if (rank == 0) mbar_expect_tx(stage_full_bar(s), 2u * (kABytes + kBBytes));
+                    mbar_expect_tx(sf_ready_bar(s), 3u * sf_bytes);
+                    bulk_load(stage + kABytes + kBBytes, sfa_src + kofs, sf_bytes, sf_ready_bar(s));
+                    bulk_load(stage + kABytes + kBBytes + kSfaBytes, sfb0_src + kofs, sf_bytes, sf_ready_bar(s));
+                    bulk_load(stage + kABytes + kBBytes + 2 * kSfaBytes, sfb1_src + kofs, sf_bytes, sf_ready_bar(s));
+                    tma_load_2d_pair(stage, &map_a, kt * (BK / 2), m0, full_leader);
+                    tma_load_2d_pair(stage + kABytes, &map_b, kt * (BK / 2), n0 + static_cast<int>(rank) * BN_CTA,
+                                     full_leader);
                 }
                 __syncwarp();
             }
-            if (ok && lane == 0) tc_commit(acc_full_bar(b));
-            __syncwarp();
+        }
+        if (ok && rank == 0) {
+            // completions of the last iterations, which no later load waited for
+            for (uint32_t j = it > kStages ? it - kStages : 0; j < it && ok; ++j) {
+                ok = __all_sync(0xFFFFFFFFu,
+                                mbar_wait(stage_free_bar(j % kStages), (j / kStages) & 1u, abort_flag, p.status));
+                if (ok && lane == 0) mbar_arrive_remote(stage_free_bar(j % kStages), 1);
+            }
+        }
+        if (!ok && lane == 0) {
+            // give the scale copies already issued a bounded chance to land before leaving
+            const uint32_t first = it > kStages ? it - kStages : 0;
+            for (uint32_t j = first; j < it; ++j)
+                for (uint32_t i = 0; i < 4096 && !mbar_try(sf_ready_bar(j % kStages), (j / kStages) & 1u); ++i) {}
+        }
+        __syncwarp();
+    } else if (warp == 1) {
+        // ------------------------------------------------------------ MMA issuer (pair leader)
+        if (rank == 0) {
+            // Ring positions are kept incrementally: operand stage s with phase ph, scale slot t.
+            uint32_t s = 0, ph = 0, t = 0, tcount = 0;
+            bool ok = true;
+            for (int tile = pair; tile < total_tiles && ok; tile += num_pairs, ++tcount) {
+                const uint32_t b = tcount & 1u, accpar = (tcount >> 1) & 1u;
+                ok = __all_sync(0xFFFFFFFFu, mbar_wait(acc_empty_bar(b), accpar ^ 1u, abort_flag, p.status));
+                if (!ok) break;
+                const uint32_t d_tmem = tmem_base + b * kAccStride;
+                uint32_t acc = 0;
+                for (int kt = 0; kt < p.k_tiles; ++kt) {
+                    ok = __all_sync(0xFFFFFFFFu, mbar_wait(stage_full_bar(s), ph, abort_flag, p.status));
+                    if (!ok) break;
+                    tc_fence_after();
+                    const uint32_t stage = base + s * kStageBytes;
+                    const uint64_t da = operand_desc(stage), db = operand_desc(stage + kABytes);
+                    const uint32_t sfa_t = tmem_base + sf_slot_col(t), sfb_t = sfa_t + kSfbOfs;
+                    const int kb_valid = min(4, p.kb_total - kt * 4);
+                    if (elect_one()) {
+                        if (kb_valid == 4) {
+                            tc_mma_pair(d_tmem, da, db, kIdesc, sfa_t, sfb_t, acc);
+                            tc_mma_pair(d_tmem, da + 2, db + 2, kIdesc, sfa_t + 4, sfb_t + 6, 1u);
+                            tc_mma_pair(d_tmem, da + 4, db + 4, kIdesc, sfa_t + 8, sfb_t + 12, 1u);
+                            tc_mma_pair(d_tmem, da + 6, db + 6, kIdesc, sfa_t + 12, sfb_t + 18, 1u);
+                        } else {
+                            for (int kk = 0; kk < kb_valid; ++kk)
+                                tc_mma_pair(d_tmem, da + 2 * kk, db + 2 * kk, kIdesc, sfa_t + 4 * kk, sfb_t + 6 * kk,
+                                            acc | static_cast<uint32_t>(kk));
+                        }
+                        // the stage (and its scale slot) is free once these MMAs have run in both
+                        // CTAs; the producer passes the signal on to the peer CTA
+                        tc_commit_pair(stage_free_bar(s));
+                    }
+                    __syncwarp();
+                    acc = 1u;
+                    s = (s + 1 == kStages) ? 0u : s + 1;
+                    ph ^= (s == 0) ? 1u : 0u;
+                    t = (t + 1 == kSfSlots) ? 0u : t + 1;
+                }
+                if (ok && elect_one()) tc_commit_pair(acc_full_bar(b));  // the leader's epilogue passes it on
+                __syncwarp();
+            }
         }
     } else if (warp >= 6) {
         // ------------------------------------------------------------ scale-factor stagers
+        // Two sets of four warps (one warp per tensor-memory lane quadrant) take alternate K
+        // iterations, so a set has two stages' worth of MMA time for one stage of scales.
         const uint32_t q = warp & 3;  // tensor-memory lane quadrant this warp may write
+        const uint32_t set = static_cast<uint32_t>(warp - 6) >> 2;
         const uint32_t lane_ofs = (q * 32u) << 16;
         uint32_t it = 0;
         bool ok = true;
-        for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
+        for (int tile = pair; tile < total_tiles && ok; tile += num_pairs) {
+            const bool mid = (((tile / p.m_tiles) * BN) & 127) != 0;
             for (int kt = 0; kt < p.k_tiles; ++kt, ++it) {
+                if ((it & 1u) != set) continue;
                 const int s = it % kStages;
-                const uint32_t t = it & 1u;
-                // the stage's scale blocks have landed, and the MMAs that read this slot two
+                const uint32_t t = it % kSfSlots;
+                // the stage's scale blocks have landed, and the MMAs that read this slot three
                 // iterations ago have completed (their commit released that iteration's stage)
-                if (!mbar_wait(full_bar(s), (it / kStages) & 1u, abort_flag, p.status) ||
-                    (it >= 2 && !mbar_wait(empty_bar((it - 2) % kStages), ((it - 2) / kStages) & 1u, abort_flag,
-                                           p.status))) {
+                if (!mbar_wait(sf_ready_bar(s), (it / kStages) & 1u, abort_flag, p.status) ||
+                    (it >= kSfSlots && !mbar_wait(stage_free_bar((it - kSfSlots) % kStages),
+                                                  ((it - kSfSlots) / kStages) & 1u, abort_flag, p.status))) {
                     ok = false;
                     break;
                 }
@@ -327,70 +459,95 @@ gemm_w4a4_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
                 const int kb_valid = min(4, p.kb_total - kt * 4);
                 const uint32_t sf_s = base + s * kStageBytes + kABytes + kBBytes + lane * 16u;
                 const uint32_t sf_t = tmem_base + lane_ofs + sf_slot_col(t);
-                for (int kk = 0; kk < kb_valid; ++kk) {
-                    const uint4 a = lds128(sf_s + kk * kSfBlock);
-                    const uint4 b0 = lds128(sf_s + kSfaBytes + kk * kSfBlock);
-                    const uint4 b1 = lds128(sf_s + 2 * kSfaBytes + kk * kSfBlock);
-                    tc_st4(sf_t + 4 * kk, a);
-                    tc_st8(sf_t + kSfbOfs + 8 * kk, b0, b1);
+                if (kb_valid == 4) {
+                    uint4 a[4], b0[4], b1[4];
+#pragma unroll
+                    for (int kk = 0; kk < 4; ++kk) {
+                        a[kk] = lds128(sf_s + kk * kSfBlock);
+                        b0[kk] = lds128(sf_s + kSfaBytes + kk * kSfBlock);
+                        b1[kk] = lds128(sf_s + 2 * kSfaBytes + kk * kSfBlock);
+                    }
+#pragma unroll
+                    for (int kk = 0; kk < 4; ++kk) {
+                        tc_st4(sf_t + 4 * kk, a[kk]);
+                        stage_b_scales(sf_t + kSfbOfs + 6 * kk, b0[kk], b1[kk], mid);
+                    }
+                } else {
+                    for (int kk = 0; kk < kb_valid; ++kk) {
+                        const uint4 a = lds128(sf_s + kk * kSfBlock);
+                        const uint4 b0 = lds128(sf_s + kSfaBytes + kk * kSfBlock);
+                        const uint4 b1 = lds128(sf_s + 2 * kSfaBytes + kk * kSfBlock);
+                        tc_st4(sf_t + 4 * kk, a);
+                        stage_b_scales(sf_t + kSfbOfs + 6 * kk, b0, b1, mid);
+                    }
                 }
                 tc_wait_st();
                 tc_fence_before();
                 __syncwarp();
-                if (lane == 0) mbar_arrive(sf_full_bar(t));
+                if (lane == 0) mbar_arrive_leader(stage_full_bar(s), rank);
             }
         }
     } else {
         // ------------------------------------------------------------ epilogue
         const int q = warp & 3;  // tensor-memory lane quadrant this warp may read
         const float alpha = __fmul_rn(__ldg(p.ts_x), __ldg(p.ts_w));
-        uint32_t tcount = 0;
-        for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x, ++tcount) {
+        const uint32_t my_epi = epi + static_cast<uint32_t>(q) * (2 * kEpiBox);
+        const uint32_t row_ofs = static_cast<uint32_t>(lane) * 128u, sw = static_cast<uint32_t>(lane & 7);
+        uint32_t tcount = 0, boxes = 0;
+        for (int tile = pair; tile < total_tiles; tile += num_pairs, ++tcount) {
             const int m_blk = tile % p.m_tiles, n_blk = tile / p.m_tiles;
-            const int m0 = m_blk * BM, n0 = n_blk * BN;
+            const int m0 = m_blk * BM + static_cast<int>(rank) * BM_CTA + q * 32, n0 = n_blk * BN;
             const uint32_t b = tcount & 1u, accpar = (tcount >> 1) & 1u;
             const bool got = mbar_wait(acc_full_bar(b), accpar, abort_flag, p.status);
             if (!__all_sync(0xFFFFFFFFu, got)) break;
+            if (rank == 0 && q == 0 && lane == 0) mbar_arrive_remote(acc_full_bar(b), 1);
             tc_fence_after();
-
-            const int row = m0 + q * 32 + lane;
-            uint16_t *yrow = p.Y + static_cast<int64_t>(row) * p.ldy;
+            const uint32_t acc = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + b * kAccStride;
 #pragma unroll 1
-            for (int c = 0; c < BN / 32; ++c) {
-                uint32_t v[32];
-                tc_ld32(tmem_base + (static_cast<uint32_t>(q * 32) << 16) + b * kAccStride + c * 32, v);
+            for (int c = 0; c < BN / 64; ++c, ++boxes) {
+                uint32_t v[32], w[32];
+                tc_ld32(acc + c * 64, v);
+                tc_ld32(acc + c * 64 + 32, w);
                 tc_wait_ld();
-                const int col0 = n0 + c * 32;
-                if (row < p.M) {
+                if (c == BN / 64 - 1) {
+                    // the whole accumulator has been read: hand it back to the MMA issuer
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive_leader(acc_empty_bar(b), rank);
+                }
+                const uint32_t buf = my_epi + (boxes & 1u) * kEpiBox;
+                // the TMA store that read this box two boxes ago must have finished reading it
+                if (lane == 0) bulk_wait_read<1>();
+                __syncwarp();
 #pragma unroll
-                    for (int j = 0; j < 4; ++j) {
-                        if (col0 + j * 8 + 8 <= p.N) {
-                            uint32_t w[4];
+                for (int i = 0; i < 4; ++i)
+                    sts128(buf + row_ofs + ((static_cast<uint32_t>(i) ^ sw) << 4), pack_bf16(v[8 * i], v[8 * i + 1], alpha),
+                           pack_bf16(v[8 * i + 2], v[8 * i + 3], alpha), pack_bf16(v[8 * i + 4], v[8 * i + 5], alpha),
+                           pack_bf16(v[8 * i + 6], v[8 * i + 7], alpha));
 #pragma unroll
-                            for (int i = 0; i < 4; ++i) {
-                                const float lo = __fmul_rn(__uint_as_float(v[j * 8 + 2 * i]), alpha);
-                                const float hi = __fmul_rn(__uint_as_float(v[j * 8 + 2 * i + 1]), alpha);
-                                w[i] = static_cast<uint32_t>(__bfloat16_as_ushort(__float2bfloat16_rn(lo))) |
-                                       (static_cast<uint32_t>(__bfloat16_as_ushort(__float2bfloat16_rn(hi))) << 16);
-                            }
-                            *reinterpret_cast<uint4 *>(yrow + col0 + j * 8) = make_uint4(w[0], w[1], w[2], w[3]);
-                        }
-                    }
+                for (int i = 0; i < 4; ++i)
+                    sts128(buf + row_ofs + ((static_cast<uint32_t>(i + 4) ^ sw) << 4),
+                           pack_bf16(w[8 * i], w[8 * i + 1], alpha), pack_bf16(w[8 * i + 2], w[8 * i + 3], alpha),
+                           pack_bf16(w[8 * i + 4], w[8 * i + 5], alpha), pack_bf16(w[8 * i + 6], w[8 * i + 7], alpha));
+                fence_async_smem();
+                __syncwarp();
+                if (lane == 0) {
+                    if (m0 < p.M && n0 + c * 64 < p.N) tma_store_2d(&map_y, n0 + c * 64, m0, buf);
+                    bulk_commit();
                 }
             }
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(acc_empty_bar(b));
         }
+        if (lane == 0) bulk_wait_all();  // shared memory must outlive the stores that read it
+        __syncwarp();
     }
 
     // ---------------------------------------------------------------- teardown
     tc_fence_before();
     __syncthreads();
-
+    cluster_sync();  // the peer may still signal this CTA's barriers or read its operands until here
     if (warp == 1) {
         tc_fence_after();
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
+        asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
     }
 }
 
@@ -411,12 +568,12 @@ EncodeTiledFn encode_tiled() {
     return fn;
 }
 
-// Packed E2M1 codes [rows, K/2] bytes, row-major: a byte tensor with 128-byte-swizzled boxes
-// of 128 bytes (256 channels) x box_rows rows.  Out-of-range rows / columns read as zero.
+// A row-major 2-D tensor [rows, row_bytes / elem] cut into 128-byte-swizzled boxes of 128 bytes x
+// box_rows rows.  Loads read out-of-range rows / columns as zero, stores skip them.
 struct MapKey {
-    const uint8_t *ptr;
-    int64_t rows, K;
-    int box_rows;
+    const void *ptr;
+    int64_t rows, row_bytes, pitch;
+    int box_rows, elem;
 };
 struct MapSlot {
     MapKey key;
@@ -424,31 +581,59 @@ struct MapSlot {
     bool used;
 };
 // Encoding a tensor map costs several microseconds of host time; a layer calls the GEMM with
-// the same operand buffers over and over, so the last few encodings are kept.
-bool make_codes_map(CUtensorMap *map, const uint8_t *ptr, int64_t rows, int64_t K, int box_rows) {
-    static thread_local MapSlot cache[8];
+// the same buffers over and over, so the last few encodings are kept.
+bool make_map(CUtensorMap *map, const void *ptr, int64_t rows, int64_t row_bytes, int64_t pitch, int box_rows,
+              int elem) {
+    constexpr int kSlots = 16;
+    static thread_local MapSlot cache[kSlots];
     static thread_local int next = 0;
     for (MapSlot &c : cache)
-        if (c.used && c.key.ptr == ptr && c.key.rows == rows && c.key.K == K && c.key.box_rows == box_rows) {
+        if (c.used && c.key.ptr == ptr && c.key.rows == rows && c.key.row_bytes == row_bytes && c.key.pitch == pitch &&
+            c.key.box_rows == box_rows && c.key.elem == elem) {
             *map = c.map;
             return true;
         }
     EncodeTiledFn enc = encode_tiled();
     if (!enc) return false;
-    const cuuint64_t dims[2] = {static_cast<cuuint64_t>(K / 2), static_cast<cuuint64_t>(rows)};
-    const cuuint64_t strides[1] = {static_cast<cuuint64_t>(K / 2)};
-    const cuuint32_t box[2] = {static_cast<cuuint32_t>(BK / 2), static_cast<cuuint32_t>(box_rows)};
+    const cuuint64_t dims[2] = {static_cast<cuuint64_t>(row_bytes / elem), static_cast<cuuint64_t>(rows)};
+    const cuuint64_t strides[1] = {static_cast<cuuint64_t>(pitch)};
+    const cuuint32_t box[2] = {static_cast<cuuint32_t>(128 / elem), static_cast<cuuint32_t>(box_rows)};
     const cuuint32_t estr[2] = {1, 1};
-    if (enc(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<uint8_t *>(ptr), dims, strides, box, estr,
-            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+    const CUtensorMapDataType dt = elem == 1 ? CU_TENSOR_MAP_DATA_TYPE_UINT8 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16;
+    if (enc(map, dt, 2, const_cast<void *>(ptr), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+            CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
         return false;
     MapSlot &slot = cache[next];
-    next = (next + 1) % 8;
-    slot.key = MapKey{ptr, rows, K, box_rows};
+    next = (next + 1) % kSlots;
+    slot.key = MapKey{ptr, rows, row_bytes, pitch, box_rows, elem};
     slot.map = *map;
     slot.used = true;
     return true;
+}
+
+// Number of CTA pairs that can be resident at once (a cluster must fit inside one GPC).
+int resident_pairs() {
+    static int pairs = 0;
+    if (pairs) return pairs;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(2, 1, 1);
+    cfg.blockDim = dim3(kThreads, 1, 1);
+    cfg.dynamicSmemBytes = kSmemBytes;
+    cudaLaunchAttribute attr;
+    attr.id = cudaLaunchAttributeClusterDimension;
+    attr.val.clusterDim.x = 2;
+    attr.val.clusterDim.y = 1;
+    attr.val.clusterDim.z = 1;
+    cfg.attrs = &attr;
+    cfg.numAttrs = 1;
+    int n = 0;
+    if (cudaOccupancyMaxActiveClusters(&n, gemm_w4a4_kernel, &cfg) != cudaSuccess || n <= 0) {
+        (void)cudaGetLastError();
+        return 0;
+    }
+    pairs = n;
+    return pairs;
 }
 
 }  // namespace
@@ -466,8 +651,10 @@ extern "C" pq_status pq_gemm_w4a4(const uint8_t *xq, const uint8_t *sfx, const f
     PQ_REQUIRE(pq_aligned256(ws), PQ_ERR_ALIGN);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
 
-    CUtensorMap map_a, map_b;
-    if (!make_codes_map(&map_a, xq, M, K, BM) || !make_codes_map(&map_b, wq, N, K, BN)) return PQ_ERR_CUDA;
+    CUtensorMap map_a, map_b, map_y;
+    if (!make_map(&map_a, xq, M, K / 2, K / 2, BM_CTA, 1) || !make_map(&map_b, wq, N, K / 2, K / 2, BN_CTA, 1) ||
+        !make_map(&map_y, Y, M, N * 2, ldy * 2, 32, 2))
+        return PQ_ERR_CUDA;
 
     static bool attr_set = false;
     if (!attr_set) {
@@ -475,28 +662,23 @@ extern "C" pq_status pq_gemm_w4a4(const uint8_t *xq, const uint8_t *sfx, const f
                                         static_cast<int>(kSmemBytes)));
         attr_set = true;
     }
-    static int sms = 0;
-    if (sms == 0) {
-        int dev = 0;
-        PQ_CUDA_OK(cudaGetDevice(&dev));
-        PQ_CUDA_OK(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
-    }
+    const int pairs_max = resident_pairs();
+    if (pairs_max <= 0) return PQ_ERR_CUDA;
 
     GemmParams p;
     p.sfx = sfx, p.sfw = sfw, p.ts_x = ts_x, p.ts_w = ts_w;
-    p.Y = static_cast<uint16_t *>(Y);
-    p.ldy = ldy;
     p.M = static_cast<int>(M), p.N = static_cast<int>(N), p.K = static_cast<int>(K);
     p.m_tiles = static_cast<int>(pq_ceil_div(M, BM));
     p.n_tiles = static_cast<int>(pq_ceil_div(N, BN));
     p.k_tiles = static_cast<int>(pq_ceil_div(K, BK));
     p.kb_total = static_cast<int>(K / 64);
     p.kb4 = p.kb_total;
+    p.m_rowblocks = static_cast<int>(pq_ceil_div(M, 128));
     p.n_rowblocks = static_cast<int>(pq_ceil_div(N, 128));
     p.status = static_cast<int *>(ws);
     const int64_t tiles = static_cast<int64_t>(p.m_tiles) * p.n_tiles;
-    const int grid = static_cast<int>(tiles < sms ? tiles : sms);
-    gemm_w4a4_kernel<<<grid, kThreads, kSmemBytes, st>>>(map_a, map_b, p);
+    const int pairs = static_cast<int>(tiles < pairs_max ? tiles : pairs_max);
+    gemm_w4a4_kernel<<<2 * pairs, kThreads, kSmemBytes, st>>>(map_a, map_b, map_y, p);
     return pq_launch_status();
 }
 
