@@ -43,9 +43,8 @@
 // The 192 B-scale rows of a tile span two blocks; the stagers pick the six 32-row words that
 // belong to the tile (it may start in the middle of a block) and store them as 6 columns.
 //
-// Cross-CTA signalling uses plain remote mbarrier arrives: the MMA issuer commits to barriers of
-// its own CTA only, and the leader's producer (stages) and epilogue (accumulators) pass each
-// completion on to the peer.  Every wait on an mbarrier is bounded.  If one expires the CTA
+// Cross-CTA signalling uses plain remote mbarrier arrives and, for the completion of a stage's
+// MMAs, one tcgen05.commit per CTA (the leader's epilogue passes accumulator completions on).  Every wait on an mbarrier is bounded.  If one expires the CTA
 // records PQ_ERR_TIMEOUT in the status word, raises a shared abort flag that every role polls,
 // and falls through to the common teardown (cluster barrier, tensor-memory release).
 #include <cuda.h>
@@ -202,8 +201,8 @@ __device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wa
 __device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-// Arrive on `bar` (this CTA's) once every tcgen05 operation issued so far by this thread has
-// completed in both CTAs of the pair.
+// Arrive on `bar` (cluster-window address: this CTA's or the peer's) once every tcgen05 operation
+// issued so far by this thread has completed in both CTAs of the pair.
 __device__ __forceinline__ void tc_commit_pair(uint32_t bar) {
     asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
@@ -358,8 +357,6 @@ gemm_w4a4_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
                 const uint32_t full_leader = mapa(stage_full_bar(s), 0);
                 const int64_t kofs = static_cast<int64_t>(kt) * 4 * kSfBlock;
                 if (elect_one()) {
-                    // the MMA issuer signals only its own CTA; pass each completion on to the peer
-                    if (rank == 0 && it >= kStages) mbar_arrive_remote(stage_free_bar(s), 1);
                     if (rank == 0) mbar_expect_tx(stage_full_bar(s), 2u * (kABytes + kBBytes));
                     mbar_expect_tx(sf_ready_bar(s), 3u * sf_bytes);
                     bulk_load(stage + kABytes + kBBytes, sfa_src + kofs, sf_bytes, sf_ready_bar(s));
@@ -370,14 +367,6 @@ gemm_w4a4_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
                                      full_leader);
                 }
                 __syncwarp();
-            }
-        }
-        if (ok && rank == 0) {
-            // completions of the last iterations, which no later load waited for
-            for (uint32_t j = it > kStages ? it - kStages : 0; j < it && ok; ++j) {
-                ok = __all_sync(0xFFFFFFFFu,
-                                mbar_wait(stage_free_bar(j % kStages), (j / kStages) & 1u, abort_flag, p.status));
-                if (ok && lane == 0) mbar_arrive_remote(stage_free_bar(j % kStages), 1);
             }
         }
         if (!ok && lane == 0) {
@@ -391,6 +380,7 @@ gemm_w4a4_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
         // ------------------------------------------------------------ MMA issuer (pair leader)
         if (rank == 0) {
             // Ring positions are kept incrementally: operand stage s with phase ph, scale slot t.
+            const uint32_t peer = mapa(bars, 1) - bars;  // cluster-window offset of the peer's shared memory
             uint32_t s = 0, ph = 0, t = 0, tcount = 0;
             bool ok = true;
             for (int tile = pair; tile < total_tiles && ok; tile += num_pairs, ++tcount) {
@@ -418,9 +408,9 @@ gemm_w4a4_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
                                 tc_mma_pair(d_tmem, da + 2 * kk, db + 2 * kk, kIdesc, sfa_t + 4 * kk, sfb_t + 6 * kk,
                                             acc | static_cast<uint32_t>(kk));
                         }
-                        // the stage (and its scale slot) is free once these MMAs have run in both
-                        // CTAs; the producer passes the signal on to the peer CTA
+                        // the stage (and its scale slot) is free in both CTAs once these MMAs have run
                         tc_commit_pair(stage_free_bar(s));
+                        tc_commit_pair(stage_free_bar(s) + peer);
                     }
                     __syncwarp();
                     acc = 1u;
@@ -449,24 +439,30 @@ gemm_w4a4_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
                 const uint32_t t = it % kSfSlots;
                 // the stage's scale blocks have landed, and the MMAs that read this slot three
                 // iterations ago have completed (their commit released that iteration's stage)
-                if (!mbar_wait(sf_ready_bar(s), (it / kStages) & 1u, abort_flag, p.status) ||
-                    (it >= kSfSlots && !mbar_wait(stage_free_bar((it - kSfSlots) % kStages),
-                                                  ((it - kSfSlots) / kStages) & 1u, abort_flag, p.status))) {
+                if (!mbar_wait(sf_ready_bar(s), (it / kStages) & 1u, abort_flag, p.status)) {
                     ok = false;
                     break;
                 }
-                tc_fence_after();
                 const int kb_valid = min(4, p.kb_total - kt * 4);
                 const uint32_t sf_s = base + s * kStageBytes + kABytes + kBBytes + lane * 16u;
                 const uint32_t sf_t = tmem_base + lane_ofs + sf_slot_col(t);
+                // the shared-memory reads do not depend on the slot: start them before waiting for it
+                uint4 a[4], b0[4], b1[4];
                 if (kb_valid == 4) {
-                    uint4 a[4], b0[4], b1[4];
 #pragma unroll
                     for (int kk = 0; kk < 4; ++kk) {
                         a[kk] = lds128(sf_s + kk * kSfBlock);
                         b0[kk] = lds128(sf_s + kSfaBytes + kk * kSfBlock);
                         b1[kk] = lds128(sf_s + 2 * kSfaBytes + kk * kSfBlock);
                     }
+                }
+                if (it >= kSfSlots && !mbar_wait(stage_free_bar((it - kSfSlots) % kStages),
+                                                 ((it - kSfSlots) / kStages) & 1u, abort_flag, p.status)) {
+                    ok = false;
+                    break;
+                }
+                tc_fence_after();
+                if (kb_valid == 4) {
 #pragma unroll
                     for (int kk = 0; kk < 4; ++kk) {
                         tc_st4(sf_t + 4 * kk, a[kk]);
