@@ -173,6 +173,18 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
     if (mbar_try(bar, parity)) return true;
     return mbar_wait_slow(bar, parity, abort_flag, status);
 }
+// The same for a converged warp: every lane gets the same answer (the vote is only taken on the
+// slow path; a vote per K iteration costs the MMA issuer 20 of its 384 cycles).
+__device__ __noinline__ bool mbar_wait_slow_warp(uint32_t bar, uint32_t parity, volatile int *abort_flag, int *status) {
+    return __all_sync(0xFFFFFFFFu, mbar_wait_slow(bar, parity, abort_flag, status));
+}
+__device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, volatile int *abort_flag, int *status) {
+    if (mbar_try(bar, parity)) return true;
+    return mbar_wait_slow_warp(bar, parity, abort_flag, status);
+}
+__device__ __forceinline__ void prefetch_tensormap(const CUtensorMap *map) {
+    asm volatile("prefetch.tensormap [%0];" ::"l"(map) : "memory");
+}
 // Operand tile load of a CTA pair: data lands in this CTA's shared memory, the byte count is
 // credited to the barrier at `bar_cluster` (the pair leader's).
 __device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap *map, int x, int y,
@@ -317,6 +329,9 @@ gemm_w4a4_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
         }
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        prefetch_tensormap(&map_a);
+        prefetch_tensormap(&map_b);
+        prefetch_tensormap(&map_y);
     }
     if (warp == 1) {
         asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
@@ -349,7 +364,7 @@ gemm_w4a4_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
             for (int kt = 0; kt < p.k_tiles; ++kt, ++it) {
                 const int s = it % kStages;
                 const uint32_t par = (it / kStages) & 1u;
-                ok = __all_sync(0xFFFFFFFFu, mbar_wait(stage_free_bar(s), par ^ 1u, abort_flag, p.status));
+                ok = mbar_wait_warp(stage_free_bar(s), par ^ 1u, abort_flag, p.status);
                 if (!ok) break;
                 const int kb_valid = min(4, p.kb_total - kt * 4);
                 const uint32_t sf_bytes = static_cast<uint32_t>(kb_valid) * kSfBlock;
@@ -385,12 +400,12 @@ gemm_w4a4_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
             bool ok = true;
             for (int tile = pair; tile < total_tiles && ok; tile += num_pairs, ++tcount) {
                 const uint32_t b = tcount & 1u, accpar = (tcount >> 1) & 1u;
-                ok = __all_sync(0xFFFFFFFFu, mbar_wait(acc_empty_bar(b), accpar ^ 1u, abort_flag, p.status));
+                ok = mbar_wait_warp(acc_empty_bar(b), accpar ^ 1u, abort_flag, p.status);
                 if (!ok) break;
                 const uint32_t d_tmem = tmem_base + b * kAccStride;
                 uint32_t acc = 0;
                 for (int kt = 0; kt < p.k_tiles; ++kt) {
-                    ok = __all_sync(0xFFFFFFFFu, mbar_wait(stage_full_bar(s), ph, abort_flag, p.status));
+                    ok = mbar_wait_warp(stage_full_bar(s), ph, abort_flag, p.status);
                     if (!ok) break;
                     tc_fence_after();
                     const uint32_t stage = base + s * kStageBytes;
