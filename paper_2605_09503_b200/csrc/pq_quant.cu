@@ -17,88 +17,65 @@ namespace {
 constexpr int kQuantThreads = 256;
 
 // ---------------------------------------------------------------- activations (no gather)
-// Index space: octets (8 channels) of the tensor padded to rows_pad rows; padding rows only
-// write zero scale bytes (tensor-core layout), never codes.  Each warp walks the index space in
-// steps of 32 octets; two independent steps are in flight per iteration (loads issued first).
-struct OctetRef {
-    int64_t row, oct;
-    bool in_range, live;
-};
-
-__device__ __forceinline__ OctetRef locate(int64_t idx, int64_t total, int64_t oct_per_row, int64_t rows,
-                                           bool small) {
-    OctetRef o;
-    o.in_range = idx < total;
-    if (!o.in_range) {
-        o.row = 0, o.oct = 0, o.live = false;
-        return o;
-    }
-    if (small) {  // 32-bit division when the index space allows it
-        const uint32_t r = static_cast<uint32_t>(idx) / static_cast<uint32_t>(oct_per_row);
-        o.row = r;
-        o.oct = static_cast<uint32_t>(idx) - r * static_cast<uint32_t>(oct_per_row);
+// One thread per 16-channel group: a 32-byte load (one 256-bit instruction when the tensor is
+// 32-byte aligned), the group's absmax, scale and codes in registers, an 8-byte store of codes.
+// The scale bytes of four adjacent groups are collected with shuffles into one 32-bit store
+// (adjacent in both scale layouts).  The index space covers the rows padded to a multiple of 128
+// in the tensor-core layout; padding rows only write zero scale bytes.  A block owns 256
+// consecutive groups of the flat (row, group) space, so its starting row and group need one
+// 64-bit division per block and each thread a 32-bit one.
+template <bool WIDE>
+__device__ __forceinline__ void load_group(const uint16_t *p, uint4 &lo, uint4 &hi) {
+    if (WIDE) {
+        asm volatile("ld.global.nc.L1::no_allocate.v8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+                     : "=r"(lo.x), "=r"(lo.y), "=r"(lo.z), "=r"(lo.w), "=r"(hi.x), "=r"(hi.y), "=r"(hi.z), "=r"(hi.w)
+                     : "l"(p));
     } else {
-        o.row = idx / oct_per_row;
-        o.oct = idx - o.row * oct_per_row;
-    }
-    o.live = o.row < rows;
-    return o;
-}
-
-template <int SF_LAYOUT>
-__device__ __forceinline__ void quant_octet(const OctetRef &o, const uint4 &v, float ts, int64_t K,
-                                            int64_t kb4, bool words, uint8_t *__restrict__ codes,
-                                            uint8_t *__restrict__ sf) {
-    float x[8];
-    pq::unpack8(v, x);
-    const float amax = pq::team_max<2>(pq::absmax8(x));
-    uint32_t sf8;
-    float d, r;
-    pq::nvfp4_scale(amax, ts, sf8, d, r);
-    const uint32_t c = pq::nvfp4_codes(x, r);
-    if (o.live) __stcs(reinterpret_cast<uint32_t *>(codes + o.row * (K >> 1) + o.oct * 4), c);
-    // collect the scale bytes of 4 adjacent groups (lanes l, l+2, l+4, l+6) into lane l
-    uint32_t word = sf8;
-    word |= __shfl_down_sync(0xFFFFFFFFu, sf8, 2) << 8;
-    word |= __shfl_down_sync(0xFFFFFFFFu, sf8, 4) << 16;
-    word |= __shfl_down_sync(0xFFFFFFFFu, sf8, 6) << 24;
-    if (!o.in_range) return;
-    const int64_t g = o.oct >> 1;
-    if (SF_LAYOUT == PQ_SF_TCGEN05) {
-        if ((threadIdx.x & 7) == 0)
-            *reinterpret_cast<uint32_t *>(sf + pq::sf_tc_offset(o.row, g, kb4)) = word;
-    } else if (o.live) {
-        if (words) {
-            if ((threadIdx.x & 7) == 0) *reinterpret_cast<uint32_t *>(sf + o.row * (K >> 4) + g) = word;
-        } else if ((o.oct & 1) == 0) {
-            sf[o.row * (K >> 4) + g] = static_cast<uint8_t>(sf8);
-        }
+        lo = __ldcs(reinterpret_cast<const uint4 *>(p));
+        hi = __ldcs(reinterpret_cast<const uint4 *>(p) + 1);
     }
 }
 
-template <int SF_LAYOUT>
+template <int SF_LAYOUT, bool WIDE>
 __global__ void __launch_bounds__(kQuantThreads)
 quant_nvfp4_kernel(const uint16_t *__restrict__ X, int64_t rows, int64_t rows_pad, int64_t K,
                    int64_t ld, const float *__restrict__ ts_ptr, uint8_t *__restrict__ codes,
                    uint8_t *__restrict__ sf) {
+    const uint32_t gpr = static_cast<uint32_t>(K >> 4);  // groups per row
+    const int64_t first = static_cast<int64_t>(blockIdx.x) * kQuantThreads;
+    const int64_t row0 = first / gpr;
+    const uint32_t g0 = static_cast<uint32_t>(first - row0 * gpr) + threadIdx.x;
+    const uint32_t dr = g0 / gpr;
+    const int64_t row = row0 + dr;
+    const uint32_t g = g0 - dr * gpr;
+    const bool in_range = row < rows_pad, live = row < rows;
     const float ts = __ldg(ts_ptr);
-    const int64_t oct_per_row = K >> 3;
-    const int64_t total = rows_pad * oct_per_row;
-    const bool small = total < (1ll << 31);
-    const int64_t kb4 = (K + 63) >> 6;
-    const bool words = (K & 63) == 0;  // four groups per 32-bit scale store
-    const int64_t stride = static_cast<int64_t>(gridDim.x) * kQuantThreads;
-    // every lane of a warp iterates the same number of times so the shuffles stay convergent
-    const int64_t warp_first = (static_cast<int64_t>(blockIdx.x) * kQuantThreads + threadIdx.x) & ~31ll;
-    const int lane = threadIdx.x & 31;
-    const uint4 zero = make_uint4(0, 0, 0, 0);
-    for (int64_t base = warp_first; base < total; base += 2 * stride) {
-        const OctetRef a = locate(base + lane, total, oct_per_row, rows, small);
-        const OctetRef b = locate(base + stride + lane, total, oct_per_row, rows, small);
-        const uint4 va = a.live ? __ldcs(reinterpret_cast<const uint4 *>(X + a.row * ld + a.oct * 8)) : zero;
-        const uint4 vb = b.live ? __ldcs(reinterpret_cast<const uint4 *>(X + b.row * ld + b.oct * 8)) : zero;
-        quant_octet<SF_LAYOUT>(a, va, ts, K, kb4, words, codes, sf);
-        if (base + stride < total) quant_octet<SF_LAYOUT>(b, vb, ts, K, kb4, words, codes, sf);
+
+    uint4 lo = make_uint4(0, 0, 0, 0), hi = lo;
+    if (live) load_group<WIDE>(X + row * ld + static_cast<int64_t>(g) * 16, lo, hi);
+    float x[8], y[8];
+    pq::unpack8(lo, x);
+    pq::unpack8(hi, y);
+    const float amax = fmaxf(pq::absmax8(x), pq::absmax8(y));
+    uint32_t sf8;
+    float d, r;
+    pq::nvfp4_scale(amax, ts, sf8, d, r);
+    const uint32_t c0 = pq::nvfp4_codes(x, r), c1 = pq::nvfp4_codes(y, r);
+    if (live) __stcs(reinterpret_cast<uint2 *>(codes + row * (K >> 1) + static_cast<int64_t>(g) * 8), make_uint2(c0, c1));
+    // scale bytes of groups g .. g+3 (same row when the row holds a multiple of 4 groups)
+    uint32_t word = sf8;
+    word |= __shfl_down_sync(0xFFFFFFFFu, sf8, 1) << 8;
+    word |= __shfl_down_sync(0xFFFFFFFFu, sf8, 2) << 16;
+    word |= __shfl_down_sync(0xFFFFFFFFu, sf8, 3) << 24;
+    if (!in_range) return;
+    if (SF_LAYOUT == PQ_SF_TCGEN05) {
+        if ((g & 3u) == 0) *reinterpret_cast<uint32_t *>(sf + pq::sf_tc_offset(row, g, gpr >> 2)) = word;
+    } else if (live) {
+        if ((gpr & 3u) == 0) {
+            if ((g & 3u) == 0) *reinterpret_cast<uint32_t *>(sf + row * gpr + g) = word;
+        } else {
+            sf[row * gpr + g] = static_cast<uint8_t>(sf8);
+        }
     }
 }
 
@@ -297,13 +274,18 @@ extern "C" pq_status pq_quant_act_nvfp4(const void *X, int64_t M, int64_t K, int
     PQ_REQUIRE(pq_aligned16(X) && ld % 8 == 0 && pq_aligned16(codes) && pq_aligned16(sf), PQ_ERR_ALIGN);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const uint16_t *x = static_cast<const uint16_t *>(X);
+    // 256-bit loads need 32-byte aligned groups
+    const bool wide = (reinterpret_cast<uintptr_t>(X) & 31u) == 0 && ld % 16 == 0;
+    const int64_t rows_idx = sf_layout == PQ_SF_TCGEN05 ? pq_ceil_div(M, 128) * 128 : M;
+    const int64_t blocks = pq_ceil_div(rows_idx * (K / 16), kQuantThreads);
+    PQ_REQUIRE(blocks < (1ll << 31), PQ_ERR_SHAPE);
+    const unsigned grid = static_cast<unsigned>(blocks);
     if (sf_layout == PQ_SF_TCGEN05) {
-        const int64_t rows_pad = pq_ceil_div(M, 128) * 128;
-        const int grid = grid_for(rows_pad * (K / 8), kQuantThreads, 16);
-        quant_nvfp4_kernel<PQ_SF_TCGEN05><<<grid, kQuantThreads, 0, st>>>(x, M, rows_pad, K, ld, ts_x, codes, sf);
+        if (wide) quant_nvfp4_kernel<PQ_SF_TCGEN05, true><<<grid, kQuantThreads, 0, st>>>(x, M, rows_idx, K, ld, ts_x, codes, sf);
+        else quant_nvfp4_kernel<PQ_SF_TCGEN05, false><<<grid, kQuantThreads, 0, st>>>(x, M, rows_idx, K, ld, ts_x, codes, sf);
     } else {
-        const int grid = grid_for(M * (K / 8), kQuantThreads, 16);
-        quant_nvfp4_kernel<PQ_SF_LINEAR><<<grid, kQuantThreads, 0, st>>>(x, M, M, K, ld, ts_x, codes, sf);
+        if (wide) quant_nvfp4_kernel<PQ_SF_LINEAR, true><<<grid, kQuantThreads, 0, st>>>(x, M, rows_idx, K, ld, ts_x, codes, sf);
+        else quant_nvfp4_kernel<PQ_SF_LINEAR, false><<<grid, kQuantThreads, 0, st>>>(x, M, rows_idx, K, ld, ts_x, codes, sf);
     }
     return pq_launch_status();
 }
