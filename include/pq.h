@@ -78,7 +78,7 @@ enum {
 
 /* Rows per fp32 partial sum in pq_calib_stats and pq_group_error (part of the arithmetic
  * definition: results depend on it). */
-#define PQ_CHUNK_ROWS 64
+#define PQ_CHUNK_ROWS 16
 
 const char *pq_status_string(pq_status s);
 

@@ -27,7 +27,7 @@
 #include <stdlib.h>
 #include <string.h>
 
-#define PQO_CHUNK 64 /* rows per fp32 partial before it is folded into the fp64 total */
+#define PQO_CHUNK 16 /* rows per fp32 partial before it is folded into the fp64 total */
 
 /* ------------------------------------------------------------------ scalar formats */
 

@@ -16,7 +16,7 @@ LIB_PATH = os.path.join(_HERE, "libpq.so")
 PQ_OK = 0
 PQ_SF_LINEAR, PQ_SF_TCGEN05 = 0, 1
 OP_CALIB_STATS, OP_SELECT_PERM, OP_GROUP_ERROR, OP_QUANT_WEIGHT, OP_GEMM = 1, 2, 3, 4, 5
-CHUNK_ROWS = 64
+CHUNK_ROWS = 16
 KIND_NVFP4, KIND_INT = 0, 1
 
 

@@ -165,5 +165,49 @@ __device__ __host__ __forceinline__ int64_t sf_tc_offset(int64_t row, int64_t co
     return ((row >> 7) * kb4 + (col >> 2)) * 512 + (row & 31) * 16 + ((row >> 5) & 3) * 4 + (col & 3);
 }
 
+// total[i] += sum over chunks (ascending) of (double) part[chunk * n + i], and, WITH_MAX,
+// vmax[i] = max(vmax[i], part_max[chunk * n + i]).  The fp64 additions are sequential per output
+// (the order is part of the arithmetic definition) but the loads are not: a block owns 32
+// consecutive outputs, all its threads stage 128 chunks of partials in shared memory with
+// coalesced loads, then one warp adds them in order.
+constexpr int kFoldThreads = 256, kFoldChunks = 128;
+
+template <bool WITH_MAX>
+__global__ void __launch_bounds__(kFoldThreads)
+fold_partials(const float *__restrict__ part, const float *__restrict__ part_max, int64_t chunks, int64_t n,
+              double *__restrict__ total, float *__restrict__ vmax) {
+    __shared__ float tile[kFoldChunks * 32];
+    __shared__ float tile_max[WITH_MAX ? kFoldChunks * 32 : 1];
+    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+    const int64_t i = static_cast<int64_t>(blockIdx.x) * 32 + lane;
+    const bool live = i < n;
+    double s = 0.0;
+    float a = 0.0f;
+    if (w == 0 && live) {
+        s = total[i];
+        if (WITH_MAX) a = vmax[i];
+    }
+    for (int64_t c0 = 0; c0 < chunks; c0 += kFoldChunks) {
+        const int nc = static_cast<int>(min(static_cast<int64_t>(kFoldChunks), chunks - c0));
+        __syncthreads();
+        for (int c = w; c < nc; c += kFoldThreads / 32) {
+            tile[c * 32 + lane] = live ? __ldcs(part + (c0 + c) * n + i) : 0.0f;
+            if (WITH_MAX) tile_max[c * 32 + lane] = live ? __ldcs(part_max + (c0 + c) * n + i) : 0.0f;
+        }
+        __syncthreads();
+        if (w == 0) {
+#pragma unroll 8
+            for (int c = 0; c < nc; ++c) {
+                s = __dadd_rn(s, static_cast<double>(tile[c * 32 + lane]));
+                if (WITH_MAX) a = fmaxf(a, tile_max[c * 32 + lane]);
+            }
+        }
+    }
+    if (w == 0 && live) {
+        total[i] = s;
+        if (WITH_MAX) vmax[i] = a;
+    }
+}
+
 }  // namespace pq
 #endif  // __CUDACC__

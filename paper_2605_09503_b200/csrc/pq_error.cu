@@ -2,7 +2,7 @@
 // the candidate selection (Sec. 3.3) and the acceptance rule (Eq. 10) compare.
 //
 // Work decomposition mirrors the arithmetic definition: a TEAM of group/8 adjacent lanes owns
-// one (order, group column) pair for one 64-row chunk and walks the chunk's rows in order,
+// one (order, group column) pair for one 16-row chunk and walks the chunk's rows in order,
 // adding each row's group error to an fp32 partial.  Partials go to the workspace
 // [chunk][order][group column]; a second kernel folds them into the fp64 totals in ascending
 // chunk order.  No floating-point atomics.
@@ -36,36 +36,43 @@ __device__ __forceinline__ float group_sse_lane(const float (&x)[8], float ts, f
 }
 
 // ---------------------------------------------------------------- original order
+constexpr int kDirectThreads = 128;
+
 template <int KIND, int TEAM>
-__global__ void __launch_bounds__(kErrThreads)
+__global__ void __launch_bounds__(kDirectThreads)
 group_error_direct(const uint16_t *__restrict__ T, int64_t rows, int64_t K, int64_t ld,
                    const float *__restrict__ ts_ptr, float Qf, float *__restrict__ part /*[chunks, K/g]*/) {
-    const int64_t oct = static_cast<int64_t>(blockIdx.x) * kErrThreads + threadIdx.x;
+    const int64_t oct = static_cast<int64_t>(blockIdx.y) * kDirectThreads + threadIdx.x;
     const bool live = oct * 8 < K;  // K % (8*TEAM) == 0, so a team is live or dead as a whole
-    const int64_t chunk = blockIdx.y;
+    const int64_t chunk = blockIdx.x;
     const int64_t r0 = chunk * PQ_CHUNK_ROWS;
     const int n = static_cast<int>(min(static_cast<int64_t>(PQ_CHUNK_ROWS), rows - r0));
     const float ts = (KIND == 0) ? __ldg(ts_ptr) : 1.0f;
     const uint16_t *p = T + r0 * ld + (live ? oct * 8 : 0);
     const uint4 zero = make_uint4(0, 0, 0, 0);
     float acc = 0.0f;
-    int t = 0;
-    for (; t + 4 <= n; t += 4) {
-        uint4 v[4];
+    if (n == PQ_CHUNK_ROWS) {
+        // all of the chunk's loads first, then the per-row errors (independent of one another),
+        // then the row-ordered sum
+        uint4 v[PQ_CHUNK_ROWS];
 #pragma unroll
-        for (int u = 0; u < 4; ++u)
-            v[u] = live ? __ldg(reinterpret_cast<const uint4 *>(p + static_cast<int64_t>(t + u) * ld)) : zero;
+        for (int u = 0; u < PQ_CHUNK_ROWS; ++u)
+            v[u] = live ? __ldcs(reinterpret_cast<const uint4 *>(p + static_cast<int64_t>(u) * ld)) : zero;
+        float e[PQ_CHUNK_ROWS];
 #pragma unroll
-        for (int u = 0; u < 4; ++u) {
+        for (int u = 0; u < PQ_CHUNK_ROWS; ++u) {
             float x[8];
             pq::unpack8(v[u], x);
+            e[u] = group_sse_lane<KIND, TEAM>(x, ts, Qf);
+        }
+#pragma unroll
+        for (int u = 0; u < PQ_CHUNK_ROWS; ++u) acc = __fadd_rn(acc, e[u]);
+    } else {
+        for (int t = 0; t < n; ++t) {
+            float x[8];
+            pq::unpack8(live ? __ldcs(reinterpret_cast<const uint4 *>(p + static_cast<int64_t>(t) * ld)) : zero, x);
             acc = __fadd_rn(acc, group_sse_lane<KIND, TEAM>(x, ts, Qf));
         }
-    }
-    for (; t < n; ++t) {
-        float x[8];
-        pq::unpack8(live ? __ldg(reinterpret_cast<const uint4 *>(p + static_cast<int64_t>(t) * ld)) : zero, x);
-        acc = __fadd_rn(acc, group_sse_lane<KIND, TEAM>(x, ts, Qf));
     }
     if (live && (oct % TEAM) == 0) part[chunk * (K / (8 * TEAM)) + oct / TEAM] = acc;
 }
@@ -138,23 +145,13 @@ group_error_gather(const uint16_t *__restrict__ T, int64_t rows, int64_t K, int6
     }
 }
 
-// err[i] += sum over chunks (ascending) of (double) part[chunk][i]
-__global__ void group_error_fold(const float *__restrict__ part, int64_t chunks, int64_t n,
-                                 double *__restrict__ err) {
-    const int64_t i = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
-    if (i >= n) return;
-    double s = err[i];
-    for (int64_t c = 0; c < chunks; ++c) s = __dadd_rn(s, static_cast<double>(part[c * n + i]));
-    err[i] = s;
-}
-
 template <int KIND, int TEAM>
 pq_status launch(const uint16_t *T, int64_t rows, int64_t K, int64_t ld, const float *ts, float Qf,
                  const int32_t *perms, int P, float *part, cudaStream_t st) {
     const int64_t chunks = pq_ceil_div(rows, PQ_CHUNK_ROWS);
     if (!perms) {
-        dim3 grid(static_cast<unsigned>(pq_ceil_div(K / 8, kErrThreads)), static_cast<unsigned>(chunks));
-        group_error_direct<KIND, TEAM><<<grid, kErrThreads, 0, st>>>(T, rows, K, ld, ts, Qf, part);
+        dim3 grid(static_cast<unsigned>(chunks), static_cast<unsigned>(pq_ceil_div(K / 8, kDirectThreads)));
+        group_error_direct<KIND, TEAM><<<grid, kDirectThreads, 0, st>>>(T, rows, K, ld, ts, Qf, part);
         return pq_launch_status();
     }
     int sub_rows = static_cast<int>((96 * 1024) / (K * 2));
@@ -187,7 +184,7 @@ extern "C" pq_status pq_group_error(const void *T, int64_t rows, int64_t K, int6
     PQ_REQUIRE(P >= 1 && P <= 8 && (perms || P == 1), PQ_ERR_SHAPE);
     PQ_REQUIRE(pq_aligned16(T) && ld % 8 == 0, PQ_ERR_ALIGN);
     const int64_t chunks = pq_ceil_div(rows, PQ_CHUNK_ROWS);
-    PQ_REQUIRE(chunks <= 65535, PQ_ERR_SHAPE);
+    PQ_REQUIRE(chunks < (1ll << 31), PQ_ERR_SHAPE);
     PQ_REQUIRE(ws && ws_bytes >= pq_workspace_bytes(PQ_OP_GROUP_ERROR, rows, K, 0, P), PQ_ERR_WORKSPACE);
     PQ_REQUIRE(pq_aligned256(ws), PQ_ERR_ALIGN);
 
@@ -208,6 +205,7 @@ extern "C" pq_status pq_group_error(const void *T, int64_t rows, int64_t K, int6
     }
     if (rc != PQ_OK) return rc;
     const int64_t n = static_cast<int64_t>(P) * (K / group);
-    group_error_fold<<<static_cast<unsigned>(pq_ceil_div(n, 128)), 128, 0, st>>>(part, chunks, n, err);
+    pq::fold_partials<false><<<static_cast<unsigned>(pq_ceil_div(n, 32)), pq::kFoldThreads, 0, st>>>(part, nullptr, chunks, n,
+                                                                                                     err, nullptr);
     return pq_launch_status();
 }

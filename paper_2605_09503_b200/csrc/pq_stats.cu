@@ -2,22 +2,32 @@
 // the absmax behind the tensor scale), plus the small reductions derived from them.
 //
 // pq_calib_stats is a streaming read of the tensor (2 bytes per element): every thread owns 8
-// adjacent channels (one 16-byte load per row) of one 64-row chunk and walks the chunk's rows
-// in order, so the fp32 partial of a (chunk, channel) pair is produced by one thread in row
-// order.  Partials go to the workspace; a second small kernel folds them into the fp64 totals
-// in ascending chunk order.  No floating-point atomics anywhere.
+// adjacent channels (one 16-byte load per row) of one 16-row chunk, issues the chunk's loads at
+// once and adds the squares in row order, so the fp32 partial of a (chunk, channel) pair is
+// produced by one thread in row order.  Partials go to the workspace; a second small kernel folds
+// them (and the per-chunk absmax) into the totals in ascending chunk order.  No atomics anywhere.
 #include "pq_common.cuh"
 
 namespace {
 
 constexpr int kStatsThreads = 128;  // 128 threads x 8 channels = 1024 channels per block
 
+__device__ __forceinline__ void stats_row(const uint4 &v, float (&s)[8], float (&a)[8]) {
+    float x[8];
+    pq::unpack8(v, x);
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        s[i] = __fmaf_rn(x[i], x[i], s[i]);
+        a[i] = fmaxf(a[i], fabsf(x[i]));
+    }
+}
+
 __global__ void __launch_bounds__(kStatsThreads)
 calib_stats_partial(const uint16_t *__restrict__ T, int64_t rows, int64_t K, int64_t ld,
-                    float *__restrict__ part /*[chunks, K]*/, float *__restrict__ amax) {
-    const int64_t col = (static_cast<int64_t>(blockIdx.x) * kStatsThreads + threadIdx.x) * 8;
+                    float *__restrict__ part /*[chunks, K]*/, float *__restrict__ part_max /*[chunks, K]*/) {
+    const int64_t col = (static_cast<int64_t>(blockIdx.y) * kStatsThreads + threadIdx.x) * 8;
     if (col >= K) return;
-    const int64_t chunk = blockIdx.y;
+    const int64_t chunk = blockIdx.x;
     const int64_t r0 = chunk * PQ_CHUNK_ROWS;
     const int n = static_cast<int>(min(static_cast<int64_t>(PQ_CHUNK_ROWS), rows - r0));
     const uint16_t *p = T + r0 * ld + col;
@@ -26,48 +36,21 @@ calib_stats_partial(const uint16_t *__restrict__ T, int64_t rows, int64_t K, int
 #pragma unroll
     for (int i = 0; i < 8; ++i) s[i] = 0.0f, a[i] = 0.0f;
 
-    int t = 0;
-    for (; t + 8 <= n; t += 8) {
-        uint4 v[8];
+    if (n == PQ_CHUNK_ROWS) {
+        uint4 v[PQ_CHUNK_ROWS];
 #pragma unroll
-        for (int u = 0; u < 8; ++u)
-            v[u] = __ldg(reinterpret_cast<const uint4 *>(p + static_cast<int64_t>(t + u) * ld));
+        for (int u = 0; u < PQ_CHUNK_ROWS; ++u) v[u] = __ldcs(reinterpret_cast<const uint4 *>(p + static_cast<int64_t>(u) * ld));
 #pragma unroll
-        for (int u = 0; u < 8; ++u) {
-            float x[8];
-            pq::unpack8(v[u], x);
-#pragma unroll
-            for (int i = 0; i < 8; ++i) {
-                s[i] = __fmaf_rn(x[i], x[i], s[i]);
-                a[i] = fmaxf(a[i], fabsf(x[i]));
-            }
-        }
-    }
-    for (; t < n; ++t) {
-        float x[8];
-        pq::unpack8(__ldg(reinterpret_cast<const uint4 *>(p + static_cast<int64_t>(t) * ld)), x);
-#pragma unroll
-        for (int i = 0; i < 8; ++i) {
-            s[i] = __fmaf_rn(x[i], x[i], s[i]);
-            a[i] = fmaxf(a[i], fabsf(x[i]));
-        }
+        for (int u = 0; u < PQ_CHUNK_ROWS; ++u) stats_row(v[u], s, a);
+    } else {
+        for (int t = 0; t < n; ++t) stats_row(__ldcs(reinterpret_cast<const uint4 *>(p + static_cast<int64_t>(t) * ld)), s, a);
     }
     float4 *dst = reinterpret_cast<float4 *>(part + chunk * K + col);
     dst[0] = make_float4(s[0], s[1], s[2], s[3]);
     dst[1] = make_float4(s[4], s[5], s[6], s[7]);
-    // max is order-independent; non-negative floats order like their bit patterns
-#pragma unroll
-    for (int i = 0; i < 8; ++i)
-        atomicMax(reinterpret_cast<unsigned int *>(amax + col + i), __float_as_uint(a[i]));
-}
-
-__global__ void calib_stats_fold(const float *__restrict__ part, int64_t chunks, int64_t K,
-                                 double *__restrict__ sumsq) {
-    const int64_t i = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
-    if (i >= K) return;
-    double s = sumsq[i];
-    for (int64_t c = 0; c < chunks; ++c) s = __dadd_rn(s, static_cast<double>(part[c * K + i]));
-    sumsq[i] = s;
+    float4 *dmax = reinterpret_cast<float4 *>(part_max + chunk * K + col);
+    dmax[0] = make_float4(a[0], a[1], a[2], a[3]);
+    dmax[1] = make_float4(a[4], a[5], a[6], a[7]);
 }
 
 __global__ void tensor_scale_kernel(const float *__restrict__ amax, int64_t K, float *ts) {
@@ -104,13 +87,13 @@ extern "C" pq_status pq_calib_stats(const void *T, int64_t rows, int64_t K, int6
     PQ_REQUIRE(ws && ws_bytes >= need, PQ_ERR_WORKSPACE);
     PQ_REQUIRE(pq_aligned256(ws), PQ_ERR_ALIGN);
     const int64_t chunks = pq_ceil_div(rows, PQ_CHUNK_ROWS);
-    PQ_REQUIRE(chunks <= 65535, PQ_ERR_SHAPE);
+    PQ_REQUIRE(chunks < (1ll << 31) && K <= 65535ll * kStatsThreads * 8, PQ_ERR_SHAPE);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    dim3 grid(static_cast<unsigned>(pq_ceil_div(K, kStatsThreads * 8)), static_cast<unsigned>(chunks));
-    calib_stats_partial<<<grid, kStatsThreads, 0, st>>>(static_cast<const uint16_t *>(T), rows, K, ld,
-                                                        static_cast<float *>(ws), amax);
-    calib_stats_fold<<<static_cast<unsigned>(pq_ceil_div(K, 128)), 128, 0, st>>>(
-        static_cast<const float *>(ws), chunks, K, sumsq);
+    dim3 grid(static_cast<unsigned>(chunks), static_cast<unsigned>(pq_ceil_div(K, kStatsThreads * 8)));
+    float *part = static_cast<float *>(ws), *part_max = part + chunks * K;
+    calib_stats_partial<<<grid, kStatsThreads, 0, st>>>(static_cast<const uint16_t *>(T), rows, K, ld, part, part_max);
+    pq::fold_partials<true><<<static_cast<unsigned>(pq_ceil_div(K, 32)), pq::kFoldThreads, 0, st>>>(part, part_max, chunks,
+                                                                                                    K, sumsq, amax);
     return pq_launch_status();
 }
 

@@ -35,15 +35,15 @@ def test_stats_against_float64_sum_and_accumulation():
 
 
 def test_stats_chunk_order_is_the_stated_one():
-    """Rows in chunks of 64: fp32 fused accumulate inside a chunk, fp64 across chunks."""
-    assert O.chunk_rows() == 64
+    """Rows in chunks of 16: fp32 fused accumulate inside a chunk, fp64 across chunks."""
+    assert O.chunk_rows() == 16
     x = inputs.bits(inputs.activations(inputs.CONFIGS["tiny"], 1, 0, rows=150))[:, :16]
     x = np.ascontiguousarray(x)
     xf = O.bf16_to_f32(x)
     want = np.zeros(16)
-    for r0 in range(0, 150, 64):
+    for r0 in range(0, 150, 16):
         p = np.zeros(16, dtype=np.float32)
-        for t in range(r0, min(r0 + 64, 150)):
+        for t in range(r0, min(r0 + 16, 150)):
             p = (p.astype(np.float64) + xf[t].astype(np.float64) ** 2).astype(np.float32)  # = fmaf
         want += p.astype(np.float64)
     S, _ = O.calib_stats(x)
