@@ -106,6 +106,33 @@ size_t pq_sf_bytes(int64_t rows, int64_t K, int sf_layout);
 pq_status pq_calib_stats(const void *T, int64_t rows, int64_t K, int64_t ld, double *sumsq,
                          float *amax, void *ws, size_t ws_bytes, void *stream);
 
+/* pq_calib_stats for callers that must not allocate device memory.  (The paper has no
+ * counterpart: this is a property of the library, not of the method.)
+ *
+ * Some users of this library run where cudaMalloc is off limits: inside a serving process whose
+ * memory pool was sized at start-up and must not grow, in a plugin that is handed tensors but no
+ * allocator, or on a path that must never hit the allocator's implicit device synchronisation.
+ * They cannot produce the workspace pq_calib_stats asks for.  This entry point computes exactly
+ * what pq_calib_stats computes (same kernels, same arithmetic, same results bit for bit) but
+ * keeps the per-chunk partial sums in a fixed array that is part of the library image:
+ * pq_calib_stats_static_max_bytes() bytes (8 MiB) on every GPU that loads the library, for the
+ * life of the process.  It calls no cudaMalloc / cudaFree and no allocating library routine.
+ *
+ *   - Limit: pq_workspace_bytes(PQ_OP_CALIB_STATS, rows, K, 0, 0) must not exceed
+ *     pq_calib_stats_static_max_bytes(); larger problems return PQ_ERR_WORKSPACE before anything
+ *     is launched (8 MiB covers e.g. 4608 x 3072 or 1536 x 9216; split bigger batches by rows,
+ *     the totals accumulate across calls anyway).
+ *   - The first call on a device looks up the array's device address (once per device, with that
+ *     device current) and remembers it; make that first call outside any stream capture.
+ *   - All calls on a device share the one array, which simply keeps what the last call left
+ *     there.  Nothing in it has to start at zero (every partial a call reads it has written
+ *     first), but two calls whose kernels overlap on the GPU (different streams, no dependency
+ *     between them) race on it: order them.
+ *   T, rows, K, ld, sumsq, amax, stream: as for pq_calib_stats. */
+pq_status pq_calib_stats_static(const void *T, int64_t rows, int64_t K, int64_t ld, double *sumsq,
+                                float *amax, void *stream);
+size_t pq_calib_stats_static_max_bytes(void);
+
 /* fp32 tensor scale from per-channel absmax: *ts = max_i amax[i] / 2688 (= 6 * 448), or 1 if
  * the maximum is 0.  ts is a device scalar. */
 pq_status pq_tensor_scale(const float *amax, int64_t K, float *ts, void *stream);

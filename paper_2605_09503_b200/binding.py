@@ -39,6 +39,8 @@ _SIGNATURES = {
     "pq_workspace_bytes": (_sz, [_int, _i64, _i64, _i64, _int]),
     "pq_sf_bytes": (_sz, [_i64, _i64, _int]),
     "pq_calib_stats": (_int, [_vp, _i64, _i64, _i64, _vp, _vp, _vp, _sz, _vp]),
+    "pq_calib_stats_static": (_int, [_vp, _i64, _i64, _i64, _vp, _vp, _vp]),
+    "pq_calib_stats_static_max_bytes": (_sz, []),
     "pq_tensor_scale": (_int, [_vp, _i64, _vp, _vp]),
     "pq_select_perm": (_int, [_vp, _i64, _vp, _i64, _i64, _int, _vp, _vp, _sz, _vp]),
     "pq_group_error": (_int, [_vp, _i64, _i64, _i64, pq_format, _vp, _vp, _int, _vp, _vp, _sz, _vp]),
@@ -123,6 +125,16 @@ def pq_calib_stats(T, sumsq, amax, ws):
     w, wb = _ws(ws)
     _check("pq_calib_stats", lib().pq_calib_stats(_p(T), T.shape[0], T.shape[1], T.stride(0), _p(sumsq),
                                                   _p(amax), w, wb, _stream()))
+
+
+def pq_calib_stats_static(T, sumsq, amax):
+    """pq_calib_stats without a workspace argument: for callers that may not allocate device
+    memory, the partial sums live in a fixed 8 MiB array inside the library (one per GPU).  Raises
+    PqError (workspace) when the problem needs more than that; calls that overlap on the GPU race."""
+    _bf16(T)
+    assert sumsq.dtype == torch.float64 and amax.dtype == torch.float32
+    _check("pq_calib_stats_static", lib().pq_calib_stats_static(_p(T), T.shape[0], T.shape[1], T.stride(0),
+                                                                _p(sumsq), _p(amax), _stream()))
 
 
 def pq_tensor_scale(amax, ts):

@@ -6,6 +6,8 @@
 // once and adds the squares in row order, so the fp32 partial of a (chunk, channel) pair is
 // produced by one thread in row order.  Partials go to the workspace; a second small kernel folds
 // them (and the per-chunk absmax) into the totals in ascending chunk order.  No atomics anywhere.
+#include <mutex>
+
 #include "pq_common.cuh"
 
 namespace {
@@ -110,4 +112,38 @@ extern "C" pq_status pq_error_weights(const double *sumsq_a, const double *sumsq
     PQ_REQUIRE(K > 0, PQ_ERR_SHAPE);
     error_weights_kernel<<<1, 2, 0, static_cast<cudaStream_t>(stream)>>>(sumsq_a, sumsq_w, K, lambda);
     return pq_launch_status();
+}
+
+// ---------------------------------------------------------------- statistics without a caller workspace
+// Scratch for pq_calib_stats_static: part of the library image, so every GPU that loads the
+// library holds these bytes until the process exits.
+constexpr size_t kStaticStatsScratchBytes = 8u << 20;
+static __device__ __align__(256) unsigned char g_static_stats_scratch[kStaticStatsScratchBytes];
+
+extern "C" size_t pq_calib_stats_static_max_bytes(void) { return kStaticStatsScratchBytes; }
+
+extern "C" pq_status pq_calib_stats_static(const void *T, int64_t rows, int64_t K, int64_t ld, double *sumsq,
+                                           float *amax, void *stream) {
+    PQ_REQUIRE(rows > 0 && K > 0, PQ_ERR_SHAPE);
+    // sizes first: this needs no CUDA call, so an oversized request fails the same way everywhere
+    PQ_REQUIRE(pq_workspace_bytes(PQ_OP_CALIB_STATS, rows, K, 0, 0) <= kStaticStatsScratchBytes, PQ_ERR_WORKSPACE);
+    // In host code the array's name is only a handle; the device address has to be asked for,
+    // once per device, with that device current.
+    constexpr int kMaxDevices = 64;
+    static std::mutex lock;
+    static void *scratch[kMaxDevices] = {};
+    int dev = -1;
+    PQ_CUDA_OK(cudaGetDevice(&dev));
+    PQ_REQUIRE(dev >= 0 && dev < kMaxDevices, PQ_ERR_CUDA);
+    void *ptr = nullptr;
+    {
+        std::lock_guard<std::mutex> guard(lock);
+        if (!scratch[dev]) {
+            void *p = nullptr;
+            PQ_CUDA_OK(cudaGetSymbolAddress(&p, g_static_stats_scratch));
+            scratch[dev] = p;
+        }
+        ptr = scratch[dev];
+    }
+    return pq_calib_stats(T, rows, K, ld, sumsq, amax, ptr, kStaticStatsScratchBytes, stream);
 }
