@@ -344,6 +344,10 @@ gemm_w4a4_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
     cluster_sync();  // both CTAs' barriers are initialised before anyone signals across
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
+    // When launched as a programmatic dependent of the activation quantizer, everything above ran
+    // while that kernel was finishing; its output (and any earlier work in the stream) is complete
+    // and visible from here on.  A no-op for an ordinary launch.
+    asm volatile("griddepcontrol.wait;" ::: "memory");
 
     const int total_tiles = p.m_tiles * p.n_tiles;
 
@@ -649,9 +653,10 @@ int resident_pairs() {
 
 }  // namespace
 
-extern "C" pq_status pq_gemm_w4a4(const uint8_t *xq, const uint8_t *sfx, const float *ts_x, const uint8_t *wq,
-                                  const uint8_t *sfw, const float *ts_w, int64_t M, int64_t N, int64_t K, void *Y,
-                                  int64_t ldy, void *ws, size_t ws_bytes, void *stream) {
+namespace {
+pq_status gemm_launch(const uint8_t *xq, const uint8_t *sfx, const float *ts_x, const uint8_t *wq, const uint8_t *sfw,
+                      const float *ts_w, int64_t M, int64_t N, int64_t K, void *Y, int64_t ldy, void *ws,
+                      size_t ws_bytes, void *stream, bool after_quantizer) {
     PQ_REQUIRE(xq && sfx && ts_x && wq && sfw && ts_w && Y, PQ_ERR_NULL);
     PQ_REQUIRE(M > 0 && N > 0 && K >= 64 && K % 64 == 0 && N % 8 == 0 && ldy >= N, PQ_ERR_SHAPE);
     PQ_REQUIRE(M < (1ll << 31) - 256 && N < (1ll << 31) - 256 && K < (1ll << 31), PQ_ERR_SHAPE);
@@ -689,8 +694,28 @@ extern "C" pq_status pq_gemm_w4a4(const uint8_t *xq, const uint8_t *sfx, const f
     p.status = static_cast<int *>(ws);
     const int64_t tiles = static_cast<int64_t>(p.m_tiles) * p.n_tiles;
     const int pairs = static_cast<int>(tiles < pairs_max ? tiles : pairs_max);
-    gemm_w4a4_kernel<<<2 * pairs, kThreads, kSmemBytes, st>>>(map_a, map_b, map_y, p);
-    return pq_launch_status();
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(2 * pairs, 1, 1);
+    cfg.blockDim = dim3(kThreads, 1, 1);
+    cfg.dynamicSmemBytes = kSmemBytes;
+    cfg.stream = st;
+    // Programmatic dependent launch: the kernel may start (barrier set-up, tensor-memory allocation,
+    // tensor-map prefetch) while the quantizer in front of it drains; it waits for that kernel's
+    // results with griddepcontrol.wait before touching global memory.
+    cudaLaunchAttribute attr;
+    attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr.val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = &attr;
+    cfg.numAttrs = after_quantizer ? 1 : 0;
+    PQ_CUDA_OK(cudaLaunchKernelEx(&cfg, gemm_w4a4_kernel, map_a, map_b, map_y, p));
+    return PQ_OK;
+}
+}  // namespace
+
+extern "C" pq_status pq_gemm_w4a4(const uint8_t *xq, const uint8_t *sfx, const float *ts_x, const uint8_t *wq,
+                                  const uint8_t *sfw, const float *ts_w, int64_t M, int64_t N, int64_t K, void *Y,
+                                  int64_t ldy, void *ws, size_t ws_bytes, void *stream) {
+    return gemm_launch(xq, sfx, ts_x, wq, sfw, ts_w, M, N, K, Y, ldy, ws, ws_bytes, stream, false);
 }
 
 extern "C" pq_status pq_linear_w4a4(const void *X, int64_t M, int64_t K, int64_t ld, const float *ts_x, uint8_t *xq,
@@ -698,7 +723,7 @@ extern "C" pq_status pq_linear_w4a4(const void *X, int64_t M, int64_t K, int64_t
                                     void *Y, int64_t ldy, void *ws, size_t ws_bytes, void *stream) {
     const pq_status rc = pq_quant_act_nvfp4(X, M, K, ld, ts_x, xq, sfx, PQ_SF_TCGEN05, stream);
     if (rc != PQ_OK) return rc;
-    return pq_gemm_w4a4(xq, sfx, ts_x, wq, sfw, ts_w, M, N, K, Y, ldy, ws, ws_bytes, stream);
+    return gemm_launch(xq, sfx, ts_x, wq, sfw, ts_w, M, N, K, Y, ldy, ws, ws_bytes, stream, true);
 }
 
 extern "C" pq_status pq_linear_w4a4_host(const void *X_host, int64_t M, int64_t K, const float *ts_x, void *X_dev,

@@ -49,6 +49,9 @@ quant_nvfp4_kernel(const uint16_t *__restrict__ X, int64_t rows, int64_t rows_pa
     const int64_t row = row0 + dr;
     const uint32_t g = g0 - dr * gpr;
     const bool in_range = row < rows_pad, live = row < rows;
+    // a kernel launched as a programmatic dependent of this one (the GEMM of pq_linear_w4a4) may
+    // begin its set-up now; it still waits for this grid to complete before reading the results
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     const float ts = __ldg(ts_ptr);
 
     uint4 lo = make_uint4(0, 0, 0, 0), hi = lo;
