@@ -28,6 +28,7 @@ WORKLOAD = "qkv"
 METRIC = "w4a4_nvfp4_linear_tflops_incl_act_quant"
 NSETS = 4          # buffer sets the timed loop rotates over (each ~137 MB; L2 is 126 MB)
 XROT = 10          # activation buffers the stand-alone streaming loops rotate over (283 MB)
+ORACLE_ROWS_MAX = 2048   # largest row sample of the workload the oracle legs use
 FP4_OVER_BF16 = 4.0  # nominal dense tensor ratio (9 vs 2.25 PFLOP/s)
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
@@ -113,7 +114,7 @@ def oracle_sample_run(rows):
         w = inputs.bits(inputs.weight(cfg, 0))
         ts_w = O.tensor_scale(O.calib_stats(w)[1])
         wq, sfw = O.quant_nvfp4(w, ts_w)
-        x = inputs.bits(inputs.activations(cfg, 0, 1000, rows=256))
+        x = inputs.bits(inputs.activations(cfg, 0, 1000, rows=ORACLE_ROWS_MAX))
         ts_x = O.tensor_scale(O.calib_stats(x)[1])
         oracle_sample_run.cache = (wq, sfw, ts_w, x, ts_x)
     wq, sfw, ts_w, x, ts_x = oracle_sample_run.cache
@@ -131,12 +132,18 @@ def oracle_threads():
         return os.cpu_count() or 1
 
 
-def cpu_baseline(target_s=12.0):
+def oracle_rows_for(seconds, cap):
+    """Rows of the sample that take the oracle about `seconds` on this host (probe, then scale)."""
+    oracle_sample_run(8)                                   # builds the cache, warms the library
+    per_row = oracle_sample_run(16) / 16.0
+    return int(max(8, min(cap, seconds / max(per_row, 1e-6))))
+
+
+def cpu_baseline(target_s=15.0):
     """Oracle throughput on a row sample sized for roughly `target_s` seconds of CPU work."""
     from paper_2605_09503_b200 import inputs
     cfg = inputs.CONFIGS[WORKLOAD]
-    t_probe = oracle_sample_run(2)
-    rows = int(max(2, min(256, 2 * target_s / max(t_probe, 1e-6))))
+    rows = oracle_rows_for(target_s, ORACLE_ROWS_MAX)
     t = oracle_sample_run(rows)
     flops = 2.0 * rows * cfg.N * cfg.K
     return {"value": flops / t / 1e12, "unit": "TFLOP/s", "cores": oracle_threads(), "kind": "oracle",
@@ -150,9 +157,8 @@ def run_reference(args):
         return
     from paper_2605_09503_b200 import inputs
     cfg = inputs.CONFIGS[WORKLOAD]
-    t_probe = oracle_sample_run(2)
     budget = 150.0 / max(1, args.steps + args.warmup)               # whole run within a few minutes
-    rows = int(max(1, min(256, 2 * budget / max(t_probe, 1e-6))))
+    rows = oracle_rows_for(budget, ORACLE_ROWS_MAX)
     for _ in range(args.warmup):
         oracle_sample_run(rows)
     t0 = time.perf_counter()
