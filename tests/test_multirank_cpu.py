@@ -1,0 +1,60 @@
+"""World-size-2 checks of the multi-GPU host logic, on CPU with the gloo backend."""
+import os
+import socket
+
+import torch
+import torch.distributed as dist
+import torch.multiprocessing as mp
+
+from paper_2605_09503_b200 import sharding
+
+
+def test_shards_partition_the_rows_on_block_boundaries():
+    for M in (4608, 4609, 130, 1, 18432, 127):
+        for world in (1, 2, 3, 8):
+            spans = [sharding.shard_rows(M, world, r) for r in range(world)]
+            assert spans[0][0] == 0 and spans[-1][1] == M
+            for (lo, hi), (lo2, _) in zip(spans, spans[1:]):
+                assert hi == lo2 and lo <= hi
+            for lo, hi in spans[:-1]:
+                assert lo % sharding.ROW_QUANTUM == 0 and (hi % sharding.ROW_QUANTUM == 0 or hi == M)
+            sizes = [hi - lo for lo, hi in spans]
+            assert max(sizes) - min(sizes) < 2 * sharding.ROW_QUANTUM
+
+
+def _free_port():
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        return s.getsockname()[1]
+
+
+def _worker(rank, world, port, out):
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK=str(rank), WORLD_SIZE=str(world))
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    try:
+        ms = 10.0 + 5.0 * rank                      # rank 1 is the slow one
+        worst = sharding.max_over_ranks(ms)
+        lo, hi = sharding.shard_rows(4608, world, rank)
+        rows = torch.tensor([hi - lo], dtype=torch.int64)
+        dist.all_reduce(rows)                        # every row is owned exactly once
+        dist.barrier()
+        out.put((rank, worst, int(rows.item()), sharding.aggregate_throughput(100.0, worst * 1e-3, world)))
+    finally:
+        dist.destroy_process_group()
+
+
+def test_timing_reduction_and_sharding_across_two_ranks():
+    ctx = mp.get_context("spawn")
+    out = ctx.Queue()
+    port = _free_port()
+    procs = [ctx.Process(target=_worker, args=(r, 2, port, out)) for r in range(2)]
+    for p in procs:
+        p.start()
+    got = sorted(out.get(timeout=120) for _ in procs)
+    for p in procs:
+        p.join(timeout=60)
+        assert p.exitcode == 0
+    for rank, worst, rows, agg in got:
+        assert worst == 15.0                         # max over ranks, seen by both
+        assert rows == 4608
+        assert abs(agg - 2 * 100.0 / 15e-3) < 1e-6
