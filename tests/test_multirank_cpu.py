@@ -17,7 +17,7 @@ def test_shards_partition_the_rows_on_block_boundaries():
             for (lo, hi), (lo2, _) in zip(spans, spans[1:]):
                 assert hi == lo2 and lo <= hi
             for lo, hi in spans[:-1]:
-                assert lo % sharding.ROW_QUANTUM == 0 and (hi % sharding.ROW_QUANTUM == 0 or hi == M)
+                assert (lo % sharding.ROW_QUANTUM == 0 or lo == M) and (hi % sharding.ROW_QUANTUM == 0 or hi == M)
             sizes = [hi - lo for lo, hi in spans]
             assert max(sizes) - min(sizes) < 2 * sharding.ROW_QUANTUM
 
