@@ -53,26 +53,23 @@
 
 namespace {
 
-constexpr int BM = 512, BM_CTA = 256, BN = 192, BN_CTA = BN / 2, BK = 256;
-constexpr int kStages = 4;
-constexpr int kAHalfBytes = 128 * BK / 2;  // 16384: one 128-row half of this CTA's 256 rows
-constexpr int kABytes = 2 * kAHalfBytes;   // 32768
+constexpr int BM = 256, BM_CTA = 128, BN = 192, BN_CTA = BN / 2, BK = 256;
+constexpr int kStages = 5;
+constexpr int kABytes = BM_CTA * BK / 2;   // 16384
 constexpr int kBBytes = BN_CTA * BK / 2;   // 12288
 constexpr int kSfBlock = 512;              // 128 rows x 4 groups
 constexpr int kSfaBytes = 4 * kSfBlock;    // 4 K-blocks of one 128-row block
-// stage: A half 0 | A half 1 | B | A scales half 0 | A scales half 1 | B scales block 0 | block 1
-constexpr int kSfaOfs = kABytes + kBBytes, kSfbOfsSmem = kSfaOfs + 2 * kSfaBytes;
-constexpr int kStageBytes = kSfbOfsSmem + 2 * kSfaBytes;  // 53248 = 52 * 1024
+constexpr int kSfbBytes = 2 * kSfaBytes;   // two 128-row blocks
+constexpr int kStageBytes = kABytes + kBBytes + kSfaBytes + kSfbBytes;  // 34816 = 34 * 1024
 constexpr int kEpiBox = 32 * 128;          // 32 rows x 64 bf16, one TMA store
-constexpr int kEpiBytes = 4 * kEpiBox;     // one staging box per epilogue warp
+constexpr int kEpiBytes = 4 * 2 * kEpiBox; // two boxes per epilogue warp
 constexpr int kThreads = 448;              // producer, MMA issuer, 4 epilogue and 8 stager warps
 constexpr int kTmemCols = 512;
-constexpr uint32_t kAccStride = BN;        // the accumulator of row half h starts at column h * 192
-// Two scale slots follow the accumulators.  A slot holds the scales of one stage: per 64-channel
-// K block 4 columns of A scales for each row half (16 + 16 columns) and 6 columns of B scales
-// (192 rows; 24 columns).
-constexpr int kSfSlots = 2;
-constexpr uint32_t kSfSlotCol0 = 2 * BN, kSfSlotCols = 16 + 16 + 24, kSfbOfs = 32;
+constexpr uint32_t kAccStride = BN;        // accumulator b starts at column b * 192
+// Three scale slots follow the accumulators.  A slot holds the scales of one stage: per 64-channel
+// K block 4 columns of A scales (128 rows) and 6 columns of B scales (192 rows).
+constexpr int kSfSlots = 3;
+constexpr uint32_t kSfSlotCol0 = 2 * BN, kSfSlotCols = 4 * (4 + 6), kSfbOfs = 16;
 static_assert(kSfSlotCol0 + kSfSlots * kSfSlotCols <= 512, "tensor memory columns");
 constexpr long long kWaitCycles = 4000000000ll;  // about two seconds of SM clock per wait
 // barriers: stage_full[S] sf_ready[S] stage_free[S] acc_full[2] acc_empty[2]
@@ -250,19 +247,6 @@ __device__ __forceinline__ void tc_st4(uint32_t taddr, const uint4 &v) {
                  "r"(v.z), "r"(v.w)
                  : "memory");
 }
-__device__ __forceinline__ void tc_st8(uint32_t taddr, const uint4 &a, const uint4 &b) {
-    asm volatile("tcgen05.st.sync.aligned.32x32b.x8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"r"(taddr),
-                 "r"(a.x), "r"(a.y), "r"(a.z), "r"(a.w), "r"(b.x), "r"(b.y), "r"(b.z), "r"(b.w)
-                 : "memory");
-}
-__device__ __forceinline__ void tc_st16(uint32_t taddr, const uint4 &a, const uint4 &b, const uint4 &c, const uint4 &d) {
-    asm volatile(
-        "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, "
-        "%15, %16};" ::"r"(taddr),
-        "r"(a.x), "r"(a.y), "r"(a.z), "r"(a.w), "r"(b.x), "r"(b.y), "r"(b.z), "r"(b.w), "r"(c.x), "r"(c.y), "r"(c.z),
-        "r"(c.w), "r"(d.x), "r"(d.y), "r"(d.z), "r"(d.w)
-        : "memory");
-}
 __device__ __forceinline__ void tc_st2(uint32_t taddr, uint32_t a, uint32_t b) {
     asm volatile("tcgen05.st.sync.aligned.32x32b.x2.b32 [%0], {%1, %2};" ::"r"(taddr), "r"(a), "r"(b) : "memory");
 }
@@ -293,10 +277,9 @@ __device__ __forceinline__ uint64_t operand_desc(uint32_t smem_addr) {
     return static_cast<uint64_t>((smem_addr & 0x3FFFFu) >> 4) | (1ull << 16) | (64ull << 32) | (1ull << 46) |
            (2ull << 61);
 }
-// Instruction descriptor: E2M1 x E2M1, UE4M3 scales, both K-major, M = 256 (128 rows in each CTA of
-// the pair), N = BN, K = 64.
+// Instruction descriptor: E2M1 x E2M1, UE4M3 scales, both K-major, M = 256 (pair), N = BN, K = 64.
 constexpr uint32_t kIdesc = (1u << 7) | (1u << 10) | (static_cast<uint32_t>(BN >> 3) << 17) | (0u << 23) |
-                            (static_cast<uint32_t>(256 >> 4) << 24);
+                            (static_cast<uint32_t>(BM >> 4) << 24);
 
 __device__ __forceinline__ uint32_t sf_slot_col(uint32_t t) { return kSfSlotCol0 + t * kSfSlotCols; }
 
@@ -325,8 +308,8 @@ gemm_w4a4_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
     auto stage_full_bar = [&](int s) { return bars + 8u * s; };
     auto sf_ready_bar = [&](int s) { return bars + 8u * (kStages + s); };     // scale blocks landed (own CTA)
     auto stage_free_bar = [&](int s) { return bars + 8u * (2 * kStages + s); };  // the stage's MMAs have run
-    auto acc_full_bar = [&](int h) { return bars + 8u * (3 * kStages + h); };    // row half h of the tile is complete
-    auto acc_empty_bar = [&](int h) { return bars + 8u * (3 * kStages + 2 + h); };  // leader's copy only
+    auto acc_full_bar = [&](int b) { return bars + 8u * (3 * kStages + b); };
+    auto acc_empty_bar = [&](int b) { return bars + 8u * (3 * kStages + 2 + b); };  // leader's copy only
     uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars_ptr + 8 * kNumBars);
     volatile int *abort_flag = reinterpret_cast<volatile int *>(bars_ptr + 8 * kNumBars + 8);
 
@@ -340,9 +323,9 @@ gemm_w4a4_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
             mbar_init(sf_ready_bar(s), 1);
             mbar_init(stage_free_bar(s), 1);
         }
-        for (int h = 0; h < 2; ++h) {
-            mbar_init(acc_full_bar(h), 1);
-            mbar_init(acc_empty_bar(h), 8);  // 4 epilogue warps in each CTA
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(acc_full_bar(b), 1);
+            mbar_init(acc_empty_bar(b), 8);  // 4 epilogue warps in each CTA
         }
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -368,21 +351,18 @@ gemm_w4a4_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
 
     const int total_tiles = p.m_tiles * p.n_tiles;
 
-    // The producer and the MMA issuer run their loops with the whole warp (uniform control flow)
-    // and single out one lane with elect.sync only around the TMA / tcgen05 instructions.
     if (warp == 0) {
         // ------------------------------------------------------------ producer
         uint32_t it = 0;
         bool ok = true;
         for (int tile = pair; tile < total_tiles && ok; tile += num_pairs) {
             const int m_blk = tile % p.m_tiles, n_blk = tile / p.m_tiles;
-            const int m0 = m_blk * BM + static_cast<int>(rank) * BM_CTA;  // this CTA's 256 rows
+            const int m0 = m_blk * BM + static_cast<int>(rank) * BM_CTA;
             const int n0 = n_blk * BN;
-            const int ra0 = min(m0 >> 7, p.m_rowblocks - 1), ra1 = min((m0 >> 7) + 1, p.m_rowblocks - 1);
+            const int ra = min(m0 >> 7, p.m_rowblocks - 1);
             const int nb0 = n0 >> 7;
             const int rb0 = min(nb0, p.n_rowblocks - 1), rb1 = min(nb0 + 1, p.n_rowblocks - 1);
-            const uint8_t *sfa0_src = p.sfx + static_cast<int64_t>(ra0) * p.kb4 * kSfBlock;
-            const uint8_t *sfa1_src = p.sfx + static_cast<int64_t>(ra1) * p.kb4 * kSfBlock;
+            const uint8_t *sfa_src = p.sfx + static_cast<int64_t>(ra) * p.kb4 * kSfBlock;
             const uint8_t *sfb0_src = p.sfw + static_cast<int64_t>(rb0) * p.kb4 * kSfBlock;
             const uint8_t *sfb1_src = p.sfw + static_cast<int64_t>(rb1) * p.kb4 * kSfBlock;
             for (int kt = 0; kt < p.k_tiles; ++kt, ++it) {
@@ -397,13 +377,11 @@ gemm_w4a4_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
                 const int64_t kofs = static_cast<int64_t>(kt) * 4 * kSfBlock;
                 if (elect_one()) {
                     if (rank == 0) mbar_expect_tx(stage_full_bar(s), 2u * (kABytes + kBBytes));
-                    mbar_expect_tx(sf_ready_bar(s), 4u * sf_bytes);
-                    bulk_load(stage + kSfaOfs, sfa0_src + kofs, sf_bytes, sf_ready_bar(s));
-                    bulk_load(stage + kSfaOfs + kSfaBytes, sfa1_src + kofs, sf_bytes, sf_ready_bar(s));
-                    bulk_load(stage + kSfbOfsSmem, sfb0_src + kofs, sf_bytes, sf_ready_bar(s));
-                    bulk_load(stage + kSfbOfsSmem + kSfaBytes, sfb1_src + kofs, sf_bytes, sf_ready_bar(s));
+                    mbar_expect_tx(sf_ready_bar(s), 3u * sf_bytes);
+                    bulk_load(stage + kABytes + kBBytes, sfa_src + kofs, sf_bytes, sf_ready_bar(s));
+                    bulk_load(stage + kABytes + kBBytes + kSfaBytes, sfb0_src + kofs, sf_bytes, sf_ready_bar(s));
+                    bulk_load(stage + kABytes + kBBytes + 2 * kSfaBytes, sfb1_src + kofs, sf_bytes, sf_ready_bar(s));
                     tma_load_2d_pair(stage, &map_a, kt * (BK / 2), m0, full_leader);
-                    tma_load_2d_pair(stage + kAHalfBytes, &map_a, kt * (BK / 2), m0 + 128, full_leader);
                     tma_load_2d_pair(stage + kABytes, &map_b, kt * (BK / 2), n0 + static_cast<int>(rank) * BN_CTA,
                                      full_leader);
                 }
@@ -425,66 +403,42 @@ gemm_w4a4_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
             uint32_t s = 0, ph = 0, t = 0, tcount = 0;
             bool ok = true;
             for (int tile = pair; tile < total_tiles && ok; tile += num_pairs, ++tcount) {
-                const uint32_t accpar = (tcount & 1u) ^ 1u;  // the epilogue has drained the previous tile
+                const uint32_t b = tcount & 1u, accpar = (tcount >> 1) & 1u;
+                ok = mbar_wait_warp(acc_empty_bar(b), accpar ^ 1u, abort_flag, p.status);
+                if (!ok) break;
+                const uint32_t d_tmem = tmem_base + b * kAccStride;
+                uint32_t acc = 0;
                 for (int kt = 0; kt < p.k_tiles; ++kt) {
                     ok = mbar_wait_warp(stage_full_bar(s), ph, abort_flag, p.status);
                     if (!ok) break;
-                    if (kt == 0) {
-                        ok = mbar_wait_warp(acc_empty_bar(0), accpar, abort_flag, p.status);
-                        if (!ok) break;
-                    }
                     tc_fence_after();
                     const uint32_t stage = base + s * kStageBytes;
-                    const uint64_t da0 = operand_desc(stage), da1 = operand_desc(stage + kAHalfBytes);
-                    const uint64_t db = operand_desc(stage + kABytes);
-                    const uint32_t slot = tmem_base + sf_slot_col(t);
-                    const uint32_t sfb_t = slot + kSfbOfs;
-                    const uint32_t d0 = tmem_base, d1 = tmem_base + kAccStride;
+                    const uint64_t da = operand_desc(stage), db = operand_desc(stage + kABytes);
+                    const uint32_t sfa_t = tmem_base + sf_slot_col(t), sfb_t = sfa_t + kSfbOfs;
                     const int kb_valid = min(4, p.kb_total - kt * 4);
-                    const uint32_t acc = kt ? 1u : 0u;
-                    const bool last = kt + 1 == p.k_tiles;
-                    // first row half
                     if (elect_one()) {
                         if (kb_valid == 4) {
-                            tc_mma_pair(d0, da0, db, kIdesc, slot, sfb_t, acc);
-                            tc_mma_pair(d0, da0 + 2, db + 2, kIdesc, slot + 4, sfb_t + 6, 1u);
-                            tc_mma_pair(d0, da0 + 4, db + 4, kIdesc, slot + 8, sfb_t + 12, 1u);
-                            tc_mma_pair(d0, da0 + 6, db + 6, kIdesc, slot + 12, sfb_t + 18, 1u);
+                            tc_mma_pair(d_tmem, da, db, kIdesc, sfa_t, sfb_t, acc);
+                            tc_mma_pair(d_tmem, da + 2, db + 2, kIdesc, sfa_t + 4, sfb_t + 6, 1u);
+                            tc_mma_pair(d_tmem, da + 4, db + 4, kIdesc, sfa_t + 8, sfb_t + 12, 1u);
+                            tc_mma_pair(d_tmem, da + 6, db + 6, kIdesc, sfa_t + 12, sfb_t + 18, 1u);
                         } else {
                             for (int kk = 0; kk < kb_valid; ++kk)
-                                tc_mma_pair(d0, da0 + 2 * kk, db + 2 * kk, kIdesc, slot + 4 * kk, sfb_t + 6 * kk,
-                                            acc | static_cast<uint32_t>(kk));
-                        }
-                        if (last) tc_commit_pair(acc_full_bar(0));  // the leader's epilogue passes it on
-                    }
-                    __syncwarp();
-                    if (kt == 0) {
-                        ok = mbar_wait_warp(acc_empty_bar(1), accpar, abort_flag, p.status);
-                        if (!ok) break;
-                        tc_fence_after();
-                    }
-                    // second row half
-                    if (elect_one()) {
-                        if (kb_valid == 4) {
-                            tc_mma_pair(d1, da1, db, kIdesc, slot + 16, sfb_t, acc);
-                            tc_mma_pair(d1, da1 + 2, db + 2, kIdesc, slot + 20, sfb_t + 6, 1u);
-                            tc_mma_pair(d1, da1 + 4, db + 4, kIdesc, slot + 24, sfb_t + 12, 1u);
-                            tc_mma_pair(d1, da1 + 6, db + 6, kIdesc, slot + 28, sfb_t + 18, 1u);
-                        } else {
-                            for (int kk = 0; kk < kb_valid; ++kk)
-                                tc_mma_pair(d1, da1 + 2 * kk, db + 2 * kk, kIdesc, slot + 16 + 4 * kk, sfb_t + 6 * kk,
+                                tc_mma_pair(d_tmem, da + 2 * kk, db + 2 * kk, kIdesc, sfa_t + 4 * kk, sfb_t + 6 * kk,
                                             acc | static_cast<uint32_t>(kk));
                         }
                         // the stage (and its scale slot) is free in both CTAs once these MMAs have run
                         tc_commit_pair(stage_free_bar(s));
                         tc_commit_pair(stage_free_bar(s) + peer);
-                        if (last) tc_commit_pair(acc_full_bar(1));
                     }
                     __syncwarp();
+                    acc = 1u;
                     s = (s + 1 == kStages) ? 0u : s + 1;
                     ph ^= (s == 0) ? 1u : 0u;
                     t = (t + 1 == kSfSlots) ? 0u : t + 1;
                 }
+                if (ok && elect_one()) tc_commit_pair(acc_full_bar(b));  // the leader's epilogue passes it on
+                __syncwarp();
             }
         }
     } else if (warp >= 6) {
@@ -502,26 +456,25 @@ gemm_w4a4_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
                 if ((it & 1u) != set) continue;
                 const int s = it % kStages;
                 const uint32_t t = it % kSfSlots;
+                // the stage's scale blocks have landed, and the MMAs that read this slot three
+                // iterations ago have completed (their commit released that iteration's stage)
                 if (!mbar_wait(sf_ready_bar(s), (it / kStages) & 1u, abort_flag, p.status)) {
                     ok = false;
                     break;
                 }
                 const int kb_valid = min(4, p.kb_total - kt * 4);
-                const uint32_t sf_s = base + s * kStageBytes + kSfaOfs + lane * 16u;
+                const uint32_t sf_s = base + s * kStageBytes + kABytes + kBBytes + lane * 16u;
                 const uint32_t sf_t = tmem_base + lane_ofs + sf_slot_col(t);
                 // the shared-memory reads do not depend on the slot: start them before waiting for it
-                uint4 a0[4], a1[4], b0[4], b1[4];
+                uint4 a[4], b0[4], b1[4];
                 if (kb_valid == 4) {
 #pragma unroll
                     for (int kk = 0; kk < 4; ++kk) {
-                        a0[kk] = lds128(sf_s + kk * kSfBlock);
-                        a1[kk] = lds128(sf_s + kSfaBytes + kk * kSfBlock);
-                        b0[kk] = lds128(sf_s + 2 * kSfaBytes + kk * kSfBlock);
-                        b1[kk] = lds128(sf_s + 3 * kSfaBytes + kk * kSfBlock);
+                        a[kk] = lds128(sf_s + kk * kSfBlock);
+                        b0[kk] = lds128(sf_s + kSfaBytes + kk * kSfBlock);
+                        b1[kk] = lds128(sf_s + 2 * kSfaBytes + kk * kSfBlock);
                     }
                 }
-                // the MMAs that read this slot kSfSlots iterations ago have completed (their commit
-                // released that iteration's stage)
                 if (it >= kSfSlots && !mbar_wait(stage_free_bar((it - kSfSlots) % kStages),
                                                  ((it - kSfSlots) / kStages) & 1u, abort_flag, p.status)) {
                     ok = false;
@@ -529,32 +482,18 @@ gemm_w4a4_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
                 }
                 tc_fence_after();
                 if (kb_valid == 4) {
-                    tc_st16(sf_t, a0[0], a0[1], a0[2], a0[3]);
-                    tc_st16(sf_t + 16, a1[0], a1[1], a1[2], a1[3]);
-                    // 24 columns of B scales: six 32-row words per K block
-                    uint32_t w[24];
 #pragma unroll
                     for (int kk = 0; kk < 4; ++kk) {
-                        w[6 * kk + 0] = mid ? b0[kk].z : b0[kk].x;
-                        w[6 * kk + 1] = mid ? b0[kk].w : b0[kk].y;
-                        w[6 * kk + 2] = mid ? b1[kk].x : b0[kk].z;
-                        w[6 * kk + 3] = mid ? b1[kk].y : b0[kk].w;
-                        w[6 * kk + 4] = mid ? b1[kk].z : b1[kk].x;
-                        w[6 * kk + 5] = mid ? b1[kk].w : b1[kk].y;
+                        tc_st4(sf_t + 4 * kk, a[kk]);
+                        stage_b_scales(sf_t + kSfbOfs + 6 * kk, b0[kk], b1[kk], mid);
                     }
-                    tc_st16(sf_t + kSfbOfs, make_uint4(w[0], w[1], w[2], w[3]), make_uint4(w[4], w[5], w[6], w[7]),
-                            make_uint4(w[8], w[9], w[10], w[11]), make_uint4(w[12], w[13], w[14], w[15]));
-                    tc_st8(sf_t + kSfbOfs + 16, make_uint4(w[16], w[17], w[18], w[19]),
-                           make_uint4(w[20], w[21], w[22], w[23]));
                 } else {
                     for (int kk = 0; kk < kb_valid; ++kk) {
-                        const uint4 x0 = lds128(sf_s + kk * kSfBlock);
-                        const uint4 x1 = lds128(sf_s + kSfaBytes + kk * kSfBlock);
-                        const uint4 y0 = lds128(sf_s + 2 * kSfaBytes + kk * kSfBlock);
-                        const uint4 y1 = lds128(sf_s + 3 * kSfaBytes + kk * kSfBlock);
-                        tc_st4(sf_t + 4 * kk, x0);
-                        tc_st4(sf_t + 16 + 4 * kk, x1);
-                        stage_b_scales(sf_t + kSfbOfs + 6 * kk, y0, y1, mid);
+                        const uint4 a = lds128(sf_s + kk * kSfBlock);
+                        const uint4 b0 = lds128(sf_s + kSfaBytes + kk * kSfBlock);
+                        const uint4 b1 = lds128(sf_s + 2 * kSfaBytes + kk * kSfBlock);
+                        tc_st4(sf_t + 4 * kk, a);
+                        stage_b_scales(sf_t + kSfbOfs + 6 * kk, b0, b1, mid);
                     }
                 }
                 tc_wait_st();
@@ -567,54 +506,49 @@ gemm_w4a4_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
         // ------------------------------------------------------------ epilogue
         const int q = warp & 3;  // tensor-memory lane quadrant this warp may read
         const float alpha = __fmul_rn(__ldg(p.ts_x), __ldg(p.ts_w));
-        const uint32_t buf = epi + static_cast<uint32_t>(q) * kEpiBox;
+        const uint32_t my_epi = epi + static_cast<uint32_t>(q) * (2 * kEpiBox);
         const uint32_t row_ofs = static_cast<uint32_t>(lane) * 128u, sw = static_cast<uint32_t>(lane & 7);
-        uint32_t tcount = 0;
-        bool ok = true;
-        for (int tile = pair; tile < total_tiles && ok; tile += num_pairs, ++tcount) {
+        uint32_t tcount = 0, boxes = 0;
+        for (int tile = pair; tile < total_tiles; tile += num_pairs, ++tcount) {
             const int m_blk = tile % p.m_tiles, n_blk = tile / p.m_tiles;
-            const int n0 = n_blk * BN;
-            for (int h = 0; h < 2; ++h) {
-                const int m0 = m_blk * BM + static_cast<int>(rank) * BM_CTA + h * 128 + q * 32;
-                const bool got = mbar_wait(acc_full_bar(h), tcount & 1u, abort_flag, p.status);
-                if (!__all_sync(0xFFFFFFFFu, got)) {
-                    ok = false;
-                    break;
-                }
-                if (rank == 0 && q == 0 && lane == 0) mbar_arrive_remote(acc_full_bar(h), 1);
-                tc_fence_after();
-                const uint32_t acc = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + h * kAccStride;
+            const int m0 = m_blk * BM + static_cast<int>(rank) * BM_CTA + q * 32, n0 = n_blk * BN;
+            const uint32_t b = tcount & 1u, accpar = (tcount >> 1) & 1u;
+            const bool got = mbar_wait(acc_full_bar(b), accpar, abort_flag, p.status);
+            if (!__all_sync(0xFFFFFFFFu, got)) break;
+            if (rank == 0 && q == 0 && lane == 0) mbar_arrive_remote(acc_full_bar(b), 1);
+            tc_fence_after();
+            const uint32_t acc = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + b * kAccStride;
 #pragma unroll 1
-                for (int c = 0; c < BN / 64; ++c) {
-                    uint32_t v[32], w[32];
-                    tc_ld32(acc + c * 64, v);
-                    tc_ld32(acc + c * 64 + 32, w);
-                    tc_wait_ld();
-                    if (c == BN / 64 - 1) {
-                        // this row half has been read: hand it back to the MMA issuer
-                        tc_fence_before();
-                        __syncwarp();
-                        if (lane == 0) mbar_arrive_leader(acc_empty_bar(h), rank);
-                    }
-                    // the TMA store that read the staging box before must have finished reading it
-                    if (lane == 0) bulk_wait_read<0>();
+            for (int c = 0; c < BN / 64; ++c, ++boxes) {
+                uint32_t v[32], w[32];
+                tc_ld32(acc + c * 64, v);
+                tc_ld32(acc + c * 64 + 32, w);
+                tc_wait_ld();
+                if (c == BN / 64 - 1) {
+                    // the whole accumulator has been read: hand it back to the MMA issuer
+                    tc_fence_before();
                     __syncwarp();
+                    if (lane == 0) mbar_arrive_leader(acc_empty_bar(b), rank);
+                }
+                const uint32_t buf = my_epi + (boxes & 1u) * kEpiBox;
+                // the TMA store that read this box two boxes ago must have finished reading it
+                if (lane == 0) bulk_wait_read<1>();
+                __syncwarp();
 #pragma unroll
-                    for (int i = 0; i < 4; ++i)
-                        sts128(buf + row_ofs + ((static_cast<uint32_t>(i) ^ sw) << 4),
-                               pack_bf16(v[8 * i], v[8 * i + 1], alpha), pack_bf16(v[8 * i + 2], v[8 * i + 3], alpha),
-                               pack_bf16(v[8 * i + 4], v[8 * i + 5], alpha), pack_bf16(v[8 * i + 6], v[8 * i + 7], alpha));
+                for (int i = 0; i < 4; ++i)
+                    sts128(buf + row_ofs + ((static_cast<uint32_t>(i) ^ sw) << 4), pack_bf16(v[8 * i], v[8 * i + 1], alpha),
+                           pack_bf16(v[8 * i + 2], v[8 * i + 3], alpha), pack_bf16(v[8 * i + 4], v[8 * i + 5], alpha),
+                           pack_bf16(v[8 * i + 6], v[8 * i + 7], alpha));
 #pragma unroll
-                    for (int i = 0; i < 4; ++i)
-                        sts128(buf + row_ofs + ((static_cast<uint32_t>(i + 4) ^ sw) << 4),
-                               pack_bf16(w[8 * i], w[8 * i + 1], alpha), pack_bf16(w[8 * i + 2], w[8 * i + 3], alpha),
-                               pack_bf16(w[8 * i + 4], w[8 * i + 5], alpha), pack_bf16(w[8 * i + 6], w[8 * i + 7], alpha));
-                    fence_async_smem();
-                    __syncwarp();
-                    if (lane == 0) {
-                        if (m0 < p.M && n0 + c * 64 < p.N) tma_store_2d(&map_y, n0 + c * 64, m0, buf);
-                        bulk_commit();
-                    }
+                for (int i = 0; i < 4; ++i)
+                    sts128(buf + row_ofs + ((static_cast<uint32_t>(i + 4) ^ sw) << 4),
+                           pack_bf16(w[8 * i], w[8 * i + 1], alpha), pack_bf16(w[8 * i + 2], w[8 * i + 3], alpha),
+                           pack_bf16(w[8 * i + 4], w[8 * i + 5], alpha), pack_bf16(w[8 * i + 6], w[8 * i + 7], alpha));
+                fence_async_smem();
+                __syncwarp();
+                if (lane == 0) {
+                    if (m0 < p.M && n0 + c * 64 < p.N) tma_store_2d(&map_y, n0 + c * 64, m0, buf);
+                    bulk_commit();
                 }
             }
         }
@@ -734,7 +668,7 @@ pq_status gemm_launch(const uint8_t *xq, const uint8_t *sfx, const float *ts_x, 
     cudaStream_t st = static_cast<cudaStream_t>(stream);
 
     CUtensorMap map_a, map_b, map_y;
-    if (!make_map(&map_a, xq, M, K / 2, K / 2, 128, 1) || !make_map(&map_b, wq, N, K / 2, K / 2, BN_CTA, 1) ||
+    if (!make_map(&map_a, xq, M, K / 2, K / 2, BM_CTA, 1) || !make_map(&map_b, wq, N, K / 2, K / 2, BN_CTA, 1) ||
         !make_map(&map_y, Y, M, N * 2, ldy * 2, 32, 2))
         return PQ_ERR_CUDA;
 
