@@ -27,7 +27,8 @@
 #include <stdlib.h>
 #include <string.h>
 
-#define PQO_CHUNK 16 /* rows per fp32 partial before it is folded into the fp64 total */
+#define PQO_CHUNK 16 /* rows per fp32 partial */
+#define PQO_SLAB 128 /* rows per fp64 slab sum: 8 chunks, added in order starting from zero */
 
 /* ------------------------------------------------------------------ scalar formats */
 
@@ -177,24 +178,31 @@ static int format_ok(int kind, int bits, int group, int64_t K) {
 /* ------------------------------------------------------------------ column statistics */
 
 /* Per channel i: sumsq[i] += sum_t x[t,i]^2 and amax[i] = max(amax[i], |x[t,i]|)  (second
- * moment of Assumption 3.1 before the division by the row count).  Rows are cut into chunks of
- * PQO_CHUNK; inside a chunk the squares are added in fp32 in row order, chunk partials are
- * folded into the fp64 total in ascending order. */
+ * moment of Assumption 3.1 before the division by the row count).  Rows are cut into slabs of
+ * PQO_SLAB and slabs into chunks of PQO_CHUNK; inside a chunk the squares are added in fp32 in
+ * row order, a slab's chunk partials are added in fp64 in ascending order starting from zero, and
+ * the slab sums are added to the fp64 total in ascending order. */
 int pqo_calib_stats(const uint16_t *T, int64_t rows, int64_t K, int64_t ld, double *sumsq,
                     float *amax) {
     if (!T || !sumsq || !amax || rows <= 0 || K <= 0 || ld < K) return 1;
-    for (int64_t r0 = 0; r0 < rows; r0 += PQO_CHUNK) {
-        int64_t r1 = (r0 + PQO_CHUNK < rows) ? r0 + PQO_CHUNK : rows;
+    for (int64_t s0 = 0; s0 < rows; s0 += PQO_SLAB) {
+        int64_t s1 = (s0 + PQO_SLAB < rows) ? s0 + PQO_SLAB : rows;
 #pragma omp parallel for schedule(static)
         for (int64_t i = 0; i < K; ++i) {
-            float p = 0.0f, a = amax[i];
-            for (int64_t t = r0; t < r1; ++t) {
-                float x = pqo_bf16_to_f32(T[t * ld + i]);
-                p = fmaf(x, x, p);
-                float ax = fabsf(x);
-                if (ax > a) a = ax;
+            double slab = 0.0;
+            float a = amax[i];
+            for (int64_t r0 = s0; r0 < s1; r0 += PQO_CHUNK) {
+                int64_t r1 = (r0 + PQO_CHUNK < s1) ? r0 + PQO_CHUNK : s1;
+                float p = 0.0f;
+                for (int64_t t = r0; t < r1; ++t) {
+                    float x = pqo_bf16_to_f32(T[t * ld + i]);
+                    p = fmaf(x, x, p);
+                    float ax = fabsf(x);
+                    if (ax > a) a = ax;
+                }
+                slab += (double)p;
             }
-            sumsq[i] += (double)p;
+            sumsq[i] += slab;
             amax[i] = a;
         }
     }
@@ -247,7 +255,8 @@ int pqo_select_perm(const double *sumsq_a, int64_t rows_a, const double *sumsq_w
 /* Eq. 3 on one batch: for every candidate order p and group column k,
  *   err[p*Kg + k] += sum_t || e - e_hat ||^2  with  e_j = T[t, perm_p(k*g + j)].
  * kind 0 = NVFP4 (bits ignored, ts used), kind 1 = INT (bits, ts ignored).
- * perms == NULL means one candidate, the identity.  Row chunking as in pqo_calib_stats. */
+ * perms == NULL means one candidate, the identity.  Rows in slabs and chunks as in
+ * pqo_calib_stats. */
 int pqo_group_error(const uint16_t *T, int64_t rows, int64_t K, int64_t ld, int kind, int bits,
                     int group, float ts, const int32_t *perms, int P, double *err) {
     if (!T || !err || rows <= 0 || K <= 0 || ld < K || P < 1) return 1;
@@ -261,9 +270,10 @@ int pqo_group_error(const uint16_t *T, int64_t rows, int64_t K, int64_t ld, int 
             const int32_t *perm = perms ? perms + (int64_t)p * K : NULL;
             float x[512], q[512];
             uint8_t code[512];
-            double total = err[(int64_t)p * Kg + k];
+            double total = err[(int64_t)p * Kg + k], slab = 0.0;
             for (int64_t r0 = 0; r0 < rows; r0 += PQO_CHUNK) {
-                int64_t r1 = (r0 + PQO_CHUNK < rows) ? r0 + PQO_CHUNK : rows;
+                int64_t r1 = (r0 + PQO_CHUNK < rows) ? r0 + PQO_CHUNK : rows; /* PQO_SLAB % PQO_CHUNK == 0 */
+                if (r0 % PQO_SLAB == 0) slab = 0.0;
                 float part = 0.0f;
                 for (int64_t t = r0; t < r1; ++t) {
                     for (int j = 0; j < g; ++j) {
@@ -280,7 +290,8 @@ int pqo_group_error(const uint16_t *T, int64_t rows, int64_t K, int64_t ld, int 
                     }
                     part = part + group_sse(x, q, d, g);
                 }
-                total += (double)part;
+                slab += (double)part;
+                if (r1 % PQO_SLAB == 0 || r1 == rows) total += slab;
             }
             err[(int64_t)p * Kg + k] = total;
         }
@@ -447,3 +458,4 @@ int pqo_gemm_bf16_ref(const uint16_t *X, const uint16_t *Wt, int64_t M, int64_t 
 }
 
 int pqo_chunk_rows(void) { return PQO_CHUNK; }
+int pqo_slab_rows(void) { return PQO_SLAB; }

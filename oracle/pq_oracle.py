@@ -56,6 +56,7 @@ def _declare(L):
     L.pqo_gemm_ref_sampled.argtypes = [_P, _P, C.c_float, _P, _P, C.c_float, _i64, _P, _P, _i64, _P]
     L.pqo_gemm_bf16_ref.argtypes = [_P, _P, _i64, _i64, _i64, _P, _P]
     L.pqo_chunk_rows.restype = C.c_int
+    L.pqo_slab_rows.restype = C.c_int
 
 
 def _ptr(a):
@@ -253,3 +254,7 @@ def gemm_bf16_ref(X, Wt, perm=None):
 
 def chunk_rows():
     return int(lib().pqo_chunk_rows())
+
+
+def slab_rows():
+    return int(lib().pqo_slab_rows())

@@ -34,20 +34,53 @@ def test_stats_against_float64_sum_and_accumulation():
     assert np.array_equal(A, np.abs(both).max(axis=0).astype(np.float32))
 
 
+def _fold(xf, rows, chunk=16, slab=128, flat=False):
+    """Column sums of squares of float32 xf in the stated order, written out with numpy scalars."""
+    want = np.zeros(xf.shape[1])
+    for s0 in range(0, rows, slab):
+        acc = np.zeros(xf.shape[1])
+        for r0 in range(s0, min(s0 + slab, rows), chunk):
+            p = np.zeros(xf.shape[1], dtype=np.float32)
+            for t in range(r0, min(r0 + chunk, s0 + slab, rows)):
+                p = (p.astype(np.float64) + xf[t].astype(np.float64) ** 2).astype(np.float32)  # = fmaf
+            if flat:
+                want += p.astype(np.float64)
+            else:
+                acc += p.astype(np.float64)
+        if not flat:
+            want += acc
+    return want
+
+
 def test_stats_chunk_order_is_the_stated_one():
-    """Rows in chunks of 16: fp32 fused accumulate inside a chunk, fp64 across chunks."""
-    assert O.chunk_rows() == 16
+    """Rows in chunks of 16 (fp32 fused accumulate), chunks in slabs of 128 rows (fp64 from zero),
+    slab sums added to the fp64 total in order."""
+    assert O.chunk_rows() == 16 and O.slab_rows() == 128
     x = inputs.bits(inputs.activations(inputs.CONFIGS["tiny"], 1, 0, rows=150))[:, :16]
     x = np.ascontiguousarray(x)
+    S, _ = O.calib_stats(x)
+    assert np.array_equal(S, _fold(O.bf16_to_f32(x), 150))
+
+
+def test_stats_slab_sums_start_from_zero():
+    """A column whose first slab is huge and whose later rows are tiny: adding the later chunk
+    partials one by one to the running total rounds differently from adding their slab sum."""
+    rng = np.random.default_rng(5)
+    xf = np.zeros((400, 16), dtype=np.float32)
+    xf[:128] = 2.0 ** 14 * (1 + rng.random((128, 16)))
+    xf[128:] = 2.0 ** -9 * (1 + rng.random((272, 16)))
+    x = np.ascontiguousarray((xf.view(np.uint32) >> 16).astype(np.uint16))     # exact bf16 truncation
     xf = O.bf16_to_f32(x)
-    want = np.zeros(16)
-    for r0 in range(0, 150, 16):
-        p = np.zeros(16, dtype=np.float32)
-        for t in range(r0, min(r0 + 16, 150)):
-            p = (p.astype(np.float64) + xf[t].astype(np.float64) ** 2).astype(np.float32)  # = fmaf
-        want += p.astype(np.float64)
+    want, flat = _fold(xf, 400), _fold(xf, 400, flat=True)
+    assert np.any(want != flat)                  # the case separates the two orders
     S, _ = O.calib_stats(x)
     assert np.array_equal(S, want)
+    # starting from an earlier total, slab sums are added to it one by one
+    S2, _ = O.calib_stats(x, S.copy(), np.zeros(16, dtype=np.float32))
+    again = want.copy()
+    for s0 in range(0, 400, 128):
+        again += _fold(xf[s0:s0 + 128], min(128, 400 - s0))
+    assert np.array_equal(S2, again)
 
 
 # ---------------------------------------------------------------- sorting

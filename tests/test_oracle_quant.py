@@ -156,6 +156,28 @@ def test_nvfp4_group_error_matches_dequant_difference():
     assert np.all(err >= 0)
 
 
+def test_group_error_row_order_is_chunks_then_slabs():
+    """One call on 300 rows = slab sums (128 rows, fp64 from zero, over 16-row chunk partials)
+    added in order; a one-chunk call returns that chunk's fp32 partial exactly."""
+    rng = np.random.default_rng(11)
+    xf = (rng.standard_normal((300, 64)) * np.where(np.arange(300)[:, None] < 128, 3e4, 1e-3)).astype(np.float32)
+    x = np.ascontiguousarray((xf.view(np.uint32) >> 16).astype(np.uint16))
+    for fmt in ((1, 4, 32, 1.0), (0, 4, 16, 2.0)):
+        whole = O.group_error(x, *fmt)
+        total = np.zeros_like(whole)
+        flat = np.zeros_like(whole)
+        for s0 in range(0, 300, 128):
+            slab = np.zeros_like(whole)
+            for r0 in range(s0, min(s0 + 128, 300), 16):
+                part = O.group_error(np.ascontiguousarray(x[r0:min(r0 + 16, s0 + 128, 300)]), *fmt)
+                assert np.array_equal(part, part.astype(np.float32).astype(np.float64))
+                slab += part
+                flat += part
+            total += slab
+        assert np.array_equal(whole, total)
+        assert fmt[0] == 0 or np.any(flat != total)      # the integer case separates the two orders
+
+
 def test_group_error_accumulates_across_calls():
     x1, x2 = _random_tensor(64, 64, 30), _random_tensor(40, 64, 31)
     e = O.group_error(x1, 1, 3, 32)
