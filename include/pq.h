@@ -76,9 +76,12 @@ enum {
     PQ_OP_GEMM = 5
 };
 
-/* Rows per fp32 partial sum in pq_calib_stats and pq_group_error (part of the arithmetic
- * definition: results depend on it). */
+/* Row blocking of the sums in pq_calib_stats and pq_group_error (part of the arithmetic
+ * definition: results depend on it).  A chunk of PQ_CHUNK_ROWS rows is summed in fp32 in row
+ * order; the chunk partials of a slab of PQ_SLAB_ROWS rows are added in fp64 in ascending order
+ * starting from zero; slab sums are added to the fp64 total in ascending order. */
 #define PQ_CHUNK_ROWS 16
+#define PQ_SLAB_ROWS 128
 
 const char *pq_status_string(pq_status s);
 
@@ -96,9 +99,9 @@ size_t pq_sf_bytes(int64_t rows, int64_t K, int sf_layout);
 /* Channel statistics (second moment of Assumption 3.1 / Sec. 3.3 before the division by the
  * row count, and the absmax used for the tensor scale).  For every channel i:
  *     sumsq[i] += sum_t T[t,i]^2        amax[i] = max(amax[i], |T[t,i]|)
- * Rows are cut into chunks of PQ_CHUNK_ROWS; squares are accumulated in fp32 (fused
- * multiply-add, row order) inside a chunk, chunk partials are added to the fp64 total in
- * ascending order.  Call once per calibration batch (and once on Wt for the weight side);
+ * Squares are accumulated in fp32 (fused multiply-add, row order) inside a chunk of
+ * PQ_CHUNK_ROWS rows; chunks, slabs and the total combine in fp64 as stated at PQ_SLAB_ROWS.
+ * Call once per calibration batch (and once on Wt for the weight side);
  * the caller zeroes sumsq / amax before the first batch.
  *   T     : bf16 [rows, K], ld.  K % 8 == 0.
  *   sumsq : fp64 [K] in/out.  amax : fp32 [K] in/out.
@@ -114,13 +117,13 @@ pq_status pq_calib_stats(const void *T, int64_t rows, int64_t K, int64_t ld, dou
  * allocator, or on a path that must never hit the allocator's implicit device synchronisation.
  * They cannot produce the workspace pq_calib_stats asks for.  This entry point computes exactly
  * what pq_calib_stats computes (same kernels, same arithmetic, same results bit for bit) but
- * keeps the per-chunk partial sums in a fixed array that is part of the library image:
+ * keeps the per-slab partial sums in a fixed array that is part of the library image:
  * pq_calib_stats_static_max_bytes() bytes (8 MiB) on every GPU that loads the library, for the
  * life of the process.  It calls no cudaMalloc / cudaFree and no allocating library routine.
  *
  *   - Limit: pq_workspace_bytes(PQ_OP_CALIB_STATS, rows, K, 0, 0) must not exceed
  *     pq_calib_stats_static_max_bytes(); larger problems return PQ_ERR_WORKSPACE before anything
- *     is launched (8 MiB covers e.g. 4608 x 3072 or 1536 x 9216; split bigger batches by rows,
+ *     is launched (8 MiB covers e.g. 4608 x 12288 or 18432 x 3072; split bigger batches by rows,
  *     the totals accumulate across calls anyway).
  *   - The first call on a device looks up the array's device address (once per device, with that
  *     device current) and remembers it; make that first call outside any stream capture.
@@ -153,7 +156,7 @@ pq_status pq_select_perm(const double *sumsq_a, int64_t rows_a, const double *su
  * where ehat is the per-group quantize-dequantize of e in format `fmt` (NVFP4 with tensor scale
  * *ts, or Eq. 1-2 integers).  perms == NULL means P == 1 and the original order.  fp32
  * arithmetic: residual by one fused multiply-add, squares summed in runs of 8 channels, runs
- * combined pairwise; rows chunked as in pq_calib_stats; fp64 across chunks and calls.
+ * combined pairwise; rows in chunks and slabs as in pq_calib_stats; fp64 across slabs and calls.
  *   T : bf16 [rows, K], ld.  K % group == 0, K <= 16384, 1 <= P <= 8.
  *   ts: device fp32 scalar (NVFP4 only, else may be NULL).
  *   err : fp64 [P, K/g] in/out (caller zeroes before the first batch).

@@ -23,8 +23,9 @@ extern "C" size_t pq_workspace_bytes(int op, int64_t rows, int64_t K, int64_t N,
     (void)N;
     if (K <= 0) return 0;
     const int64_t chunks = rows > 0 ? pq_ceil_div(rows, PQ_CHUNK_ROWS) : 0;
+    const int64_t slabs = rows > 0 ? pq_ceil_div(rows, PQ_SLAB_ROWS) : 0;
     switch (op) {
-        case PQ_OP_CALIB_STATS: return round256(2 * static_cast<size_t>(chunks) * K * sizeof(float));
+        case PQ_OP_CALIB_STATS: return round256(static_cast<size_t>(slabs) * K * (sizeof(double) + sizeof(float)));
         case PQ_OP_SELECT_PERM: return round256(static_cast<size_t>(P > 0 ? P : 1) * K * sizeof(uint64_t));
         case PQ_OP_GROUP_ERROR:
             return round256(static_cast<size_t>(chunks) * (P > 0 ? P : 1) * (K / 16 + 1) * sizeof(float));

@@ -160,54 +160,142 @@ __device__ __forceinline__ float run_sse(const float (&x)[8], const float (&q)[8
     return acc;
 }
 
+// ---- error path on magnitudes.  (x - q d)^2 does not depend on the common sign of x and q, so the
+// error kernels quantize |x| and skip the sign handling; every operation below is sign-symmetric
+// (round to nearest even), hence the squares equal those of the signed computation bit for bit.
+
+// |x| * r rounded to E2M1, returned as the fp32 values of the codes.  The decode is a byte-table
+// lookup: for code c (0..7) the bf16 pattern of its value {0, .5, 1, 1.5, 2, 3, 4, 6} is
+// {0x0000, 0x3F00, 0x3F80, 0x3FC0, 0x4000, 0x4040, 0x4080, 0x40C0}; prmt picks the high and low
+// bytes with the four codes of a 16-bit half as selectors, a second prmt interleaves them into
+// bf16 pairs, and a bf16 widens to fp32 by a shift.
+__device__ __forceinline__ void nvfp4_levels_abs(const float (&x)[8], float r, float (&q)[8]) {
+    float y[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) y[i] = __fmul_rn(fabsf(x[i]), r);
+    const uint32_t codes = f32x8_to_e2m1(y);
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+        const uint32_t sel = h ? codes >> 16 : codes & 0xFFFFu;
+        const uint32_t hi = __byte_perm(0x3F3F3F00u, 0x40404040u, sel);
+        const uint32_t lo = __byte_perm(0xC0800000u, 0xC0804000u, sel);
+        const uint32_t p01 = __byte_perm(lo, hi, 0x5140u), p23 = __byte_perm(lo, hi, 0x7362u);
+        q[4 * h + 0] = __uint_as_float(p01 << 16);
+        q[4 * h + 1] = __uint_as_float(p01 & 0xFFFF0000u);
+        q[4 * h + 2] = __uint_as_float(p23 << 16);
+        q[4 * h + 3] = __uint_as_float(p23 & 0xFFFF0000u);
+    }
+}
+
+// min(rint(|x| * r), Q).  For |y| < 2^22 adding and subtracting 1.5 * 2^23 rounds to the nearest
+// integer, ties to even, exactly like rint; beyond that (and for inf) the result is at least Q and
+// the clamp takes over; NaN (0 * inf) goes to -Q in the signed definition (fmaxf drops the NaN),
+// i.e. to magnitude Q, which fminf(NaN, Q) gives here as well.
+__device__ __forceinline__ void int_levels_abs(const float (&x)[8], float r, float Qf, float (&z)[8]) {
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        const float y = __fmul_rn(fabsf(x[i]), r);
+        const float q = __fadd_rn(__fadd_rn(y, 12582912.0f), -12582912.0f);
+        z[i] = fminf(q, Qf);
+    }
+}
+
+// Sum of squared residuals of eight magnitudes: delta = fma(-q, d, |x|); acc = fma(delta, delta, acc).
+__device__ __forceinline__ float run_sse_abs(const float (&x)[8], const float (&q)[8], float d) {
+    float acc = 0.0f;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        const float delta = __fmaf_rn(-q[i], d, fabsf(x[i]));
+        acc = __fmaf_rn(delta, delta, acc);
+    }
+    return acc;
+}
+
 // Byte offset of scale (row, col) in the tensor-core layout; kb4 = number of 4-column blocks.
 __device__ __host__ __forceinline__ int64_t sf_tc_offset(int64_t row, int64_t col, int64_t kb4) {
     return ((row >> 7) * kb4 + (col >> 2)) * 512 + (row & 31) * 16 + ((row >> 5) & 3) * 4 + (col & 3);
 }
 
-// total[i] += sum over chunks (ascending) of (double) part[chunk * n + i], and, WITH_MAX,
-// vmax[i] = max(vmax[i], part_max[chunk * n + i]).  The fp64 additions are sequential per output
-// (the order is part of the arithmetic definition) but the loads are not: a block owns 32
-// consecutive outputs, all its threads stage 128 chunks of partials in shared memory with
-// coalesced loads, then one warp adds them in order.
-constexpr int kFoldThreads = 256, kFoldChunks = 128;
+// Programmatic dependent launch: a kernel that calls dependents_may_launch() lets the next
+// kernel of the stream (launched with launch_dependent) start its blocks early; that kernel calls
+// wait_for_prior_grid() before it touches anything the earlier kernel wrote.  Both are no-ops in
+// a plain launch.
+__device__ __forceinline__ void dependents_may_launch() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void wait_for_prior_grid() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 
-template <bool WITH_MAX>
+template <typename... KArgs, typename... Args>
+cudaError_t launch_dependent(void (*kern)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid, cfg.blockDim = block, cfg.dynamicSmemBytes = smem, cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr, cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kern, static_cast<KArgs>(args)...);
+}
+
+// Ordered fold of row-block partials into the fp64 totals (the order is part of the arithmetic
+// definition).  part[c * n + i] is the partial of row block c for output i, c ascending in rows.
+//   PER_SLAB == 1: the partials are fp64 slab sums:  total[i] += part[c][i], c ascending.
+//   PER_SLAB == 8: the partials are fp32 chunk sums: every run of 8 consecutive chunks (one slab)
+//                  is added in fp64 from zero, then the slab sum is added to total[i].
+// WITH_MAX also folds vmax[i] = max(vmax[i], part_max[c][i]).
+// The additions are sequential per output but the loads are not: a block owns 16 consecutive
+// outputs, all its threads stage a batch of 128 partials per output in shared memory with
+// coalesced loads, then 16 lanes add them in order.
+constexpr int kFoldThreads = 256, kFoldOutputs = 16, kFoldBatch = 128;
+
+template <typename PT, int PER_SLAB, bool WITH_MAX>
 __global__ void __launch_bounds__(kFoldThreads)
-fold_partials(const float *__restrict__ part, const float *__restrict__ part_max, int64_t chunks, int64_t n,
+fold_partials(const PT *__restrict__ part, const float *__restrict__ part_max, int64_t count, int64_t n,
               double *__restrict__ total, float *__restrict__ vmax) {
-    __shared__ float tile[kFoldChunks * 32];
-    __shared__ float tile_max[WITH_MAX ? kFoldChunks * 32 : 1];
-    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
-    const int64_t i = static_cast<int64_t>(blockIdx.x) * 32 + lane;
-    const bool live = i < n;
-    double s = 0.0;
+    static_assert(kFoldBatch % PER_SLAB == 0, "a batch holds whole slabs");
+    __shared__ PT tile[kFoldBatch * kFoldOutputs];
+    __shared__ float tile_max[WITH_MAX ? kFoldBatch * kFoldOutputs : 1];
+    const int o = threadIdx.x % kFoldOutputs, g = threadIdx.x / kFoldOutputs;  // output, row of the batch
+    constexpr int kRowsPerPass = kFoldThreads / kFoldOutputs;
+    const int64_t i = static_cast<int64_t>(blockIdx.x) * kFoldOutputs + o;
+    const bool live = i < n, adder = threadIdx.x < kFoldOutputs;
+    double s = 0.0, slab = 0.0;
     float a = 0.0f;
-    if (w == 0 && live) {
+    if (adder && live) {
         s = total[i];
         if (WITH_MAX) a = vmax[i];
     }
-    for (int64_t c0 = 0; c0 < chunks; c0 += kFoldChunks) {
-        const int nc = static_cast<int>(min(static_cast<int64_t>(kFoldChunks), chunks - c0));
+    wait_for_prior_grid();
+    for (int64_t c0 = 0; c0 < count; c0 += kFoldBatch) {
+        const int nc = static_cast<int>(min(static_cast<int64_t>(kFoldBatch), count - c0));
         __syncthreads();
-        for (int c = w; c < nc; c += kFoldThreads / 32) {
-            tile[c * 32 + lane] = live ? __ldcs(part + (c0 + c) * n + i) : 0.0f;
-            if (WITH_MAX) tile_max[c * 32 + lane] = live ? __ldcs(part_max + (c0 + c) * n + i) : 0.0f;
+#pragma unroll
+        for (int c = g; c < kFoldBatch; c += kRowsPerPass) {
+            if (c < nc) {
+                tile[c * kFoldOutputs + o] = live ? __ldcs(part + (c0 + c) * n + i) : PT(0);
+                if (WITH_MAX) tile_max[c * kFoldOutputs + o] = live ? __ldcs(part_max + (c0 + c) * n + i) : 0.0f;
+            }
         }
         __syncthreads();
-        if (w == 0) {
+        if (adder) {
 #pragma unroll 8
             for (int c = 0; c < nc; ++c) {
-                s = __dadd_rn(s, static_cast<double>(tile[c * 32 + lane]));
-                if (WITH_MAX) a = fmaxf(a, tile_max[c * 32 + lane]);
+                if (PER_SLAB == 1) {
+                    s = __dadd_rn(s, static_cast<double>(tile[c * kFoldOutputs + o]));
+                } else {
+                    slab = __dadd_rn(slab, static_cast<double>(tile[c * kFoldOutputs + o]));
+                    if ((c % PER_SLAB) == PER_SLAB - 1 || c0 + c == count - 1) {
+                        s = __dadd_rn(s, slab);
+                        slab = 0.0;
+                    }
+                }
+                if (WITH_MAX) a = fmaxf(a, tile_max[c * kFoldOutputs + o]);
             }
         }
     }
-    if (w == 0 && live) {
+    if (adder && live) {
         total[i] = s;
         if (WITH_MAX) vmax[i] = a;
     }
 }
+
 
 }  // namespace pq
 #endif  // __CUDACC__

@@ -1,14 +1,16 @@
 // Calibration quantization error per candidate order and group column (Eq. 3), the quantity
 // the candidate selection (Sec. 3.3) and the acceptance rule (Eq. 10) compare.
 //
-// Work decomposition mirrors the arithmetic definition: a TEAM of group/8 adjacent lanes owns
-// one (order, group column) pair for one 16-row chunk and walks the chunk's rows in order,
-// adding each row's group error to an fp32 partial.  Partials go to the workspace
-// [chunk][order][group column]; a second kernel folds them into the fp64 totals in ascending
-// chunk order.  No floating-point atomics.
+// The original-order kernel leaves fp64 slab sums [slab][group column] in the workspace, the
+// candidate kernel fp32 chunk partials [chunk][order][group column]; a second kernel, launched as a
+// programmatic dependent, adds them to the fp64 totals in ascending order (for chunk partials:
+// each slab's eight in fp64 from zero first).  No floating-point atomics.
 //
-//   original order (perms == NULL): rows are read straight from global memory with coalesced
-//     16-byte loads -- a pure streaming pass, bound by HBM bandwidth.
+//   original order (perms == NULL): a thread owns 16 adjacent channels (two 16-byte loads per
+//     row) of one chunk, i.e. a whole NVFP4 group or 1/2 .. 1/8 of an integer group; it loads
+//     eight rows at a time and walks them in order; a block covers the eight chunks of a slab.  The pass streams the tensor once from HBM;
+//     its cost per element is arithmetic (about ten instructions), so it sits between the HBM and
+//     the ALU roof.
 //   candidate orders: one block per (chunk, order); rows are staged in shared memory a few at a
 //     time (coalesced) and the lanes gather their eight channels from there, so the tensor is
 //     fetched from HBM once per chunk and served from L2 to the other orders' blocks.
@@ -18,6 +20,7 @@ namespace {
 
 constexpr int kErrThreads = 256;
 
+// Gather path: a TEAM of group/8 adjacent lanes owns a group, 8 channels per lane.
 template <int KIND, int TEAM>
 __device__ __forceinline__ float group_sse_lane(const float (&x)[8], float ts, float Qf) {
     const float amax = pq::team_max<TEAM>(pq::absmax8(x));
@@ -26,55 +29,91 @@ __device__ __forceinline__ float group_sse_lane(const float (&x)[8], float ts, f
         uint32_t sf8;
         float r;
         pq::nvfp4_scale(amax, ts, sf8, d, r);
-        pq::e2m1x8_to_f32(pq::nvfp4_codes(x, r), q);
+        pq::nvfp4_levels_abs(x, r, q);
     } else {
         float r;
         pq::int_scale(amax, Qf, d, r);
-        pq::int_levels(x, r, Qf, q);
+        pq::int_levels_abs(x, r, Qf, q);
     }
-    return pq::team_sum<TEAM>(pq::run_sse(x, q, d));
+    return pq::team_sum<TEAM>(pq::run_sse_abs(x, q, d));
 }
 
 // ---------------------------------------------------------------- original order
 constexpr int kDirectThreads = 128;
+constexpr int kDirectRows = 8;  // rows in flight per thread (2 x 16 bytes each)
 
-template <int KIND, int TEAM>
+// Error of one row's 16 channels held by this lane; TEAM16 = group / 16 adjacent lanes share a group.
+template <int KIND, int TEAM16>
+__device__ __forceinline__ float row_sse16(const uint4 &lo, const uint4 &hi, float ts, float Qf) {
+    float xa[8], xb[8];
+    pq::unpack8(lo, xa);
+    pq::unpack8(hi, xb);
+    const float amax = pq::team_max<TEAM16>(fmaxf(pq::absmax8(xa), pq::absmax8(xb)));
+    float qa[8], qb[8], d, r;
+    if (KIND == 0) {
+        uint32_t sf8;
+        pq::nvfp4_scale(amax, ts, sf8, d, r);
+        pq::nvfp4_levels_abs(xa, r, qa);
+        pq::nvfp4_levels_abs(xb, r, qb);
+    } else {
+        pq::int_scale(amax, Qf, d, r);
+        pq::int_levels_abs(xa, r, Qf, qa);
+        pq::int_levels_abs(xb, r, Qf, qb);
+    }
+    // runs of 8 channels, then the balanced adjacent-pair tree: its first level is this lane's two runs
+    return pq::team_sum<TEAM16>(__fadd_rn(pq::run_sse_abs(xa, qa, d), pq::run_sse_abs(xb, qb, d)));
+}
+
+constexpr int kSlabChunks = PQ_SLAB_ROWS / PQ_CHUNK_ROWS;  // 8
+constexpr int kDirectRuns = kDirectThreads / kSlabChunks;  // 16 runs of 16 channels per block
+static_assert(kDirectRuns == 16, "a warp holds two chunks of 16 runs");
+
+// One block = one 128-row slab x 256 channels: thread (c, j) owns chunk c of the slab and the
+// j-th 16-channel run, so a warp reads 2 x 512 contiguous bytes per row step.  The eight chunk
+// partials of a group meet in shared memory and one thread adds them in fp64 in chunk order;
+// the workspace receives fp64 slab sums [slab][K/g].
+template <int KIND, int TEAM16>
 __global__ void __launch_bounds__(kDirectThreads)
 group_error_direct(const uint16_t *__restrict__ T, int64_t rows, int64_t K, int64_t ld,
-                   const float *__restrict__ ts_ptr, float Qf, float *__restrict__ part /*[chunks, K/g]*/) {
-    const int64_t oct = static_cast<int64_t>(blockIdx.y) * kDirectThreads + threadIdx.x;
-    const bool live = oct * 8 < K;  // K % (8*TEAM) == 0, so a team is live or dead as a whole
-    const int64_t chunk = blockIdx.x;
-    const int64_t r0 = chunk * PQ_CHUNK_ROWS;
-    const int n = static_cast<int>(min(static_cast<int64_t>(PQ_CHUNK_ROWS), rows - r0));
+                   const float *__restrict__ ts_ptr, float Qf, double *__restrict__ slab_part /*[slabs, K/g]*/) {
+    __shared__ float part_s[kSlabChunks][kDirectRuns];
+    pq::dependents_may_launch();
+    const int runs = static_cast<int>(K >> 4);  // K % (16 * TEAM16) == 0
+    const int c = threadIdx.x / kDirectRuns, j = threadIdx.x % kDirectRuns;
+    const int run = blockIdx.y * kDirectRuns + j;
+    const int64_t slab = blockIdx.x;
+    const int64_t r0 = slab * PQ_SLAB_ROWS + c * PQ_CHUNK_ROWS;
+    // 16 % TEAM16 == 0 and runs % TEAM16 == 0: a team is live or dead as a whole, and the
+    // shuffles below stay inside its 16-lane half of the warp
+    const bool live = run < runs && r0 < rows;
+    const int n = live ? static_cast<int>(min(static_cast<int64_t>(PQ_CHUNK_ROWS), rows - r0)) : 0;
     const float ts = (KIND == 0) ? __ldg(ts_ptr) : 1.0f;
-    const uint16_t *p = T + r0 * ld + (live ? oct * 8 : 0);
-    const uint4 zero = make_uint4(0, 0, 0, 0);
+    const uint16_t *p = T + (live ? r0 * ld + static_cast<int64_t>(run) * 16 : 0);
     float acc = 0.0f;
-    if (n == PQ_CHUNK_ROWS) {
-        // all of the chunk's loads first, then the per-row errors (independent of one another),
-        // then the row-ordered sum
-        uint4 v[PQ_CHUNK_ROWS];
+#pragma unroll 1
+    for (int t0 = 0; t0 < PQ_CHUNK_ROWS; t0 += kDirectRows) {
+        uint4 lo[kDirectRows], hi[kDirectRows];
+        const uint4 zero = make_uint4(0, 0, 0, 0);
 #pragma unroll
-        for (int u = 0; u < PQ_CHUNK_ROWS; ++u)
-            v[u] = live ? __ldcs(reinterpret_cast<const uint4 *>(p + static_cast<int64_t>(u) * ld)) : zero;
-        float e[PQ_CHUNK_ROWS];
-#pragma unroll
-        for (int u = 0; u < PQ_CHUNK_ROWS; ++u) {
-            float x[8];
-            pq::unpack8(v[u], x);
-            e[u] = group_sse_lane<KIND, TEAM>(x, ts, Qf);
+        for (int u = 0; u < kDirectRows; ++u) {
+            const bool have = t0 + u < n;
+            const uint4 *src = reinterpret_cast<const uint4 *>(p + static_cast<int64_t>(t0 + u) * ld);
+            lo[u] = have ? __ldg(src) : zero;
+            hi[u] = have ? __ldg(src + 1) : zero;
         }
+        // rows past the end are all-zero groups: their error is +0.0 and adding it changes nothing
 #pragma unroll
-        for (int u = 0; u < PQ_CHUNK_ROWS; ++u) acc = __fadd_rn(acc, e[u]);
-    } else {
-        for (int t = 0; t < n; ++t) {
-            float x[8];
-            pq::unpack8(live ? __ldcs(reinterpret_cast<const uint4 *>(p + static_cast<int64_t>(t) * ld)) : zero, x);
-            acc = __fadd_rn(acc, group_sse_lane<KIND, TEAM>(x, ts, Qf));
-        }
+        for (int u = 0; u < kDirectRows; ++u) acc = __fadd_rn(acc, row_sse16<KIND, TEAM16>(lo[u], hi[u], ts, Qf));
     }
-    if (live && (oct % TEAM) == 0) part[chunk * (K / (8 * TEAM)) + oct / TEAM] = acc;
+    part_s[c][j] = acc;
+    __syncthreads();
+    // chunks past the last row hold +0.0, which leaves the slab sum unchanged
+    if (threadIdx.x < kDirectRuns && run < runs && (run % TEAM16) == 0) {
+        double sum = 0.0;
+#pragma unroll
+        for (int k = 0; k < kSlabChunks; ++k) sum = __dadd_rn(sum, static_cast<double>(part_s[k][j]));
+        slab_part[slab * (runs / TEAM16) + run / TEAM16] = sum;
+    }
 }
 
 // ---------------------------------------------------------------- candidate orders
@@ -86,6 +125,7 @@ group_error_gather(const uint16_t *__restrict__ T, int64_t rows, int64_t K, int6
                    const float *__restrict__ ts_ptr, float Qf, const int32_t *__restrict__ perms, int P,
                    int sub_rows, float *__restrict__ part /*[chunks, P, K/g]*/) {
     extern __shared__ __align__(16) uint16_t rows_s[];  // [sub_rows][K]
+    pq::dependents_may_launch();
     const int64_t chunk = blockIdx.x;
     const int p = blockIdx.y;
     const int32_t *perm = perms + static_cast<int64_t>(p) * K;
@@ -145,14 +185,25 @@ group_error_gather(const uint16_t *__restrict__ T, int64_t rows, int64_t K, int6
     }
 }
 
-template <int KIND, int TEAM>
+template <typename PT, int PER_SLAB>
+pq_status fold(const void *part, int64_t count, int64_t n, double *err, cudaStream_t st) {
+    PQ_CUDA_OK(pq::launch_dependent(pq::fold_partials<PT, PER_SLAB, false>,
+                                    dim3(static_cast<unsigned>(pq_ceil_div(n, pq::kFoldOutputs))), dim3(pq::kFoldThreads),
+                                    0, st, static_cast<const PT *>(part), static_cast<const float *>(nullptr), count, n,
+                                    err, static_cast<float *>(nullptr)));
+    return pq_launch_status();
+}
+
+template <int KIND, int TEAM>  // TEAM = group / 8
 pq_status launch(const uint16_t *T, int64_t rows, int64_t K, int64_t ld, const float *ts, float Qf,
-                 const int32_t *perms, int P, float *part, cudaStream_t st) {
-    const int64_t chunks = pq_ceil_div(rows, PQ_CHUNK_ROWS);
+                 const int32_t *perms, int P, void *ws, double *err, cudaStream_t st) {
+    const int64_t chunks = pq_ceil_div(rows, PQ_CHUNK_ROWS), slabs = pq_ceil_div(rows, PQ_SLAB_ROWS);
+    const int64_t Kg = K / (8 * TEAM);
     if (!perms) {
-        dim3 grid(static_cast<unsigned>(chunks), static_cast<unsigned>(pq_ceil_div(K / 8, kDirectThreads)));
-        group_error_direct<KIND, TEAM><<<grid, kDirectThreads, 0, st>>>(T, rows, K, ld, ts, Qf, part);
-        return pq_launch_status();
+        dim3 grid(static_cast<unsigned>(slabs), static_cast<unsigned>(pq_ceil_div(K / 16, kDirectRuns)));
+        group_error_direct<KIND, TEAM / 2><<<grid, kDirectThreads, 0, st>>>(T, rows, K, ld, ts, Qf, static_cast<double *>(ws));
+        if (pq_launch_status() != PQ_OK) return PQ_ERR_CUDA;
+        return fold<double, 1>(ws, slabs, Kg, err, st);
     }
     int sub_rows = static_cast<int>((96 * 1024) / (K * 2));
     if (sub_rows > 16) sub_rows = 16;
@@ -162,8 +213,10 @@ pq_status launch(const uint16_t *T, int64_t rows, int64_t K, int64_t ld, const f
         PQ_CUDA_OK(cudaFuncSetAttribute(group_error_gather<KIND, TEAM>,
                                         cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)));
     dim3 grid(static_cast<unsigned>(chunks), static_cast<unsigned>(P));
-    group_error_gather<KIND, TEAM><<<grid, kErrThreads, smem, st>>>(T, rows, K, ld, ts, Qf, perms, P, sub_rows, part);
-    return pq_launch_status();
+    group_error_gather<KIND, TEAM><<<grid, kErrThreads, smem, st>>>(T, rows, K, ld, ts, Qf, perms, P, sub_rows,
+                                                                 static_cast<float *>(ws));
+    if (pq_launch_status() != PQ_OK) return PQ_ERR_CUDA;
+    return fold<float, kSlabChunks>(ws, chunks, static_cast<int64_t>(P) * Kg, err, st);
 }
 
 }  // namespace
@@ -190,22 +243,12 @@ extern "C" pq_status pq_group_error(const void *T, int64_t rows, int64_t K, int6
 
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const uint16_t *t = static_cast<const uint16_t *>(T);
-    float *part = static_cast<float *>(ws);
     const float Qf = fmt.kind == 1 ? static_cast<float>((1 << (fmt.bits - 1)) - 1) : 0.0f;
-    pq_status rc;
-    if (fmt.kind == 0) {
-        rc = launch<0, 2>(t, rows, K, ld, ts, Qf, perms, P, part, st);
-    } else {
-        switch (group) {
-            case 16: rc = launch<1, 2>(t, rows, K, ld, ts, Qf, perms, P, part, st); break;
-            case 32: rc = launch<1, 4>(t, rows, K, ld, ts, Qf, perms, P, part, st); break;
-            case 64: rc = launch<1, 8>(t, rows, K, ld, ts, Qf, perms, P, part, st); break;
-            default: rc = launch<1, 16>(t, rows, K, ld, ts, Qf, perms, P, part, st); break;
-        }
+    if (fmt.kind == 0) return launch<0, 2>(t, rows, K, ld, ts, Qf, perms, P, ws, err, st);
+    switch (group) {
+        case 16: return launch<1, 2>(t, rows, K, ld, ts, Qf, perms, P, ws, err, st);
+        case 32: return launch<1, 4>(t, rows, K, ld, ts, Qf, perms, P, ws, err, st);
+        case 64: return launch<1, 8>(t, rows, K, ld, ts, Qf, perms, P, ws, err, st);
+        default: return launch<1, 16>(t, rows, K, ld, ts, Qf, perms, P, ws, err, st);
     }
-    if (rc != PQ_OK) return rc;
-    const int64_t n = static_cast<int64_t>(P) * (K / group);
-    pq::fold_partials<false><<<static_cast<unsigned>(pq_ceil_div(n, 32)), pq::kFoldThreads, 0, st>>>(part, nullptr, chunks, n,
-                                                                                                     err, nullptr);
-    return pq_launch_status();
 }

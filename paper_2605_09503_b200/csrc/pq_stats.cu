@@ -1,18 +1,23 @@
 // Channel statistics of the calibration pass (second moments of Assumption 3.1 / Sec. 3.3 and
 // the absmax behind the tensor scale), plus the small reductions derived from them.
 //
-// pq_calib_stats is a streaming read of the tensor (2 bytes per element): every thread owns 8
-// adjacent channels (one 16-byte load per row) of one 16-row chunk, issues the chunk's loads at
-// once and adds the squares in row order, so the fp32 partial of a (chunk, channel) pair is
-// produced by one thread in row order.  Partials go to the workspace; a second small kernel folds
-// them (and the per-chunk absmax) into the totals in ascending chunk order.  No atomics anywhere.
+// pq_calib_stats is a streaming read of the tensor (2 bytes per element).  A block of 8 warps owns
+// one 128-row slab x 256 channels: warp w takes the slab's w-th 16-row chunk, each lane 8 adjacent
+// channels (one 16-byte load per row, the chunk's 16 loads in flight together) and adds the squares
+// in row order in fp32.  The eight chunk partials of a channel meet in shared memory, where one
+// thread per channel adds them in fp64 in chunk order; the slab sums (and slab absmax) go to the
+// workspace, 12 bytes per channel per 128 rows.  A second small kernel, launched as a programmatic
+// dependent, adds the slab sums to the totals in slab order.  No atomics anywhere.
 #include <mutex>
 
 #include "pq_common.cuh"
 
 namespace {
 
-constexpr int kStatsThreads = 128;  // 128 threads x 8 channels = 1024 channels per block
+constexpr int kStatsThreads = 256;                                // 8 warps = the 8 chunks of a slab
+constexpr int kStatsCols = 256;                                   // 32 lanes x 8 channels
+constexpr int kSlabChunks = PQ_SLAB_ROWS / PQ_CHUNK_ROWS;
+static_assert(kSlabChunks * 32 == kStatsThreads, "one warp per chunk of the slab");
 
 __device__ __forceinline__ void stats_row(const uint4 &v, float (&s)[8], float (&a)[8]) {
     float x[8];
@@ -25,34 +30,55 @@ __device__ __forceinline__ void stats_row(const uint4 &v, float (&s)[8], float (
 }
 
 __global__ void __launch_bounds__(kStatsThreads)
-calib_stats_partial(const uint16_t *__restrict__ T, int64_t rows, int64_t K, int64_t ld,
-                    float *__restrict__ part /*[chunks, K]*/, float *__restrict__ part_max /*[chunks, K]*/) {
-    const int64_t col = (static_cast<int64_t>(blockIdx.y) * kStatsThreads + threadIdx.x) * 8;
-    if (col >= K) return;
-    const int64_t chunk = blockIdx.x;
-    const int64_t r0 = chunk * PQ_CHUNK_ROWS;
-    const int n = static_cast<int>(min(static_cast<int64_t>(PQ_CHUNK_ROWS), rows - r0));
-    const uint16_t *p = T + r0 * ld + col;
+calib_stats_slab(const uint16_t *__restrict__ T, int64_t rows, int64_t K, int64_t ld,
+                 double *__restrict__ slab_sum /*[slabs, K]*/, float *__restrict__ slab_max /*[slabs, K]*/) {
+    __shared__ __align__(16) float sum_s[kSlabChunks][kStatsCols];
+    __shared__ __align__(16) float max_s[kSlabChunks][kStatsCols];
+    pq::dependents_may_launch();
+    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+    const int64_t col0 = static_cast<int64_t>(blockIdx.y) * kStatsCols;
+    const int64_t col = col0 + lane * 8;
+    const int64_t slab = blockIdx.x;
+    const int64_t r0 = slab * PQ_SLAB_ROWS + w * PQ_CHUNK_ROWS;
+    const int64_t left = rows - r0;
+    const int n = left >= PQ_CHUNK_ROWS ? PQ_CHUNK_ROWS : (left > 0 ? static_cast<int>(left) : 0);
 
     float s[8], a[8];
 #pragma unroll
     for (int i = 0; i < 8; ++i) s[i] = 0.0f, a[i] = 0.0f;
-
-    if (n == PQ_CHUNK_ROWS) {
-        uint4 v[PQ_CHUNK_ROWS];
+    if (col < K) {
+        const uint16_t *p = T + r0 * ld + col;
+        if (n == PQ_CHUNK_ROWS) {
+            uint4 v[PQ_CHUNK_ROWS];
 #pragma unroll
-        for (int u = 0; u < PQ_CHUNK_ROWS; ++u) v[u] = __ldcs(reinterpret_cast<const uint4 *>(p + static_cast<int64_t>(u) * ld));
+            for (int u = 0; u < PQ_CHUNK_ROWS; ++u) v[u] = __ldcs(reinterpret_cast<const uint4 *>(p + static_cast<int64_t>(u) * ld));
 #pragma unroll
-        for (int u = 0; u < PQ_CHUNK_ROWS; ++u) stats_row(v[u], s, a);
-    } else {
-        for (int t = 0; t < n; ++t) stats_row(__ldcs(reinterpret_cast<const uint4 *>(p + static_cast<int64_t>(t) * ld)), s, a);
+            for (int u = 0; u < PQ_CHUNK_ROWS; ++u) stats_row(v[u], s, a);
+        } else {
+            for (int t = 0; t < n; ++t) stats_row(__ldcs(reinterpret_cast<const uint4 *>(p + static_cast<int64_t>(t) * ld)), s, a);
+        }
     }
-    float4 *dst = reinterpret_cast<float4 *>(part + chunk * K + col);
-    dst[0] = make_float4(s[0], s[1], s[2], s[3]);
-    dst[1] = make_float4(s[4], s[5], s[6], s[7]);
-    float4 *dmax = reinterpret_cast<float4 *>(part_max + chunk * K + col);
-    dmax[0] = make_float4(a[0], a[1], a[2], a[3]);
-    dmax[1] = make_float4(a[4], a[5], a[6], a[7]);
+    float4 *ds = reinterpret_cast<float4 *>(&sum_s[w][lane * 8]);
+    ds[0] = make_float4(s[0], s[1], s[2], s[3]);
+    ds[1] = make_float4(s[4], s[5], s[6], s[7]);
+    float4 *dm = reinterpret_cast<float4 *>(&max_s[w][lane * 8]);
+    dm[0] = make_float4(a[0], a[1], a[2], a[3]);
+    dm[1] = make_float4(a[4], a[5], a[6], a[7]);
+    __syncthreads();
+    // one thread per channel: the slab's chunk partials in chunk order, from zero (a chunk past
+    // the last row contributes +0.0, which leaves the sum unchanged)
+    const int c = threadIdx.x;
+    if (col0 + c < K) {
+        double acc = 0.0;
+        float m = 0.0f;
+#pragma unroll
+        for (int k = 0; k < kSlabChunks; ++k) {
+            acc = __dadd_rn(acc, static_cast<double>(sum_s[k][c]));
+            m = fmaxf(m, max_s[k][c]);
+        }
+        slab_sum[slab * K + col0 + c] = acc;
+        slab_max[slab * K + col0 + c] = m;
+    }
 }
 
 __global__ void tensor_scale_kernel(const float *__restrict__ amax, int64_t K, float *ts) {
@@ -88,14 +114,16 @@ extern "C" pq_status pq_calib_stats(const void *T, int64_t rows, int64_t K, int6
     const size_t need = pq_workspace_bytes(PQ_OP_CALIB_STATS, rows, K, 0, 0);
     PQ_REQUIRE(ws && ws_bytes >= need, PQ_ERR_WORKSPACE);
     PQ_REQUIRE(pq_aligned256(ws), PQ_ERR_ALIGN);
-    const int64_t chunks = pq_ceil_div(rows, PQ_CHUNK_ROWS);
-    PQ_REQUIRE(chunks < (1ll << 31) && K <= 65535ll * kStatsThreads * 8, PQ_ERR_SHAPE);
+    const int64_t slabs = pq_ceil_div(rows, PQ_SLAB_ROWS);
+    PQ_REQUIRE(slabs < (1ll << 31) && K <= 65535ll * kStatsCols, PQ_ERR_SHAPE);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    dim3 grid(static_cast<unsigned>(chunks), static_cast<unsigned>(pq_ceil_div(K, kStatsThreads * 8)));
-    float *part = static_cast<float *>(ws), *part_max = part + chunks * K;
-    calib_stats_partial<<<grid, kStatsThreads, 0, st>>>(static_cast<const uint16_t *>(T), rows, K, ld, part, part_max);
-    pq::fold_partials<true><<<static_cast<unsigned>(pq_ceil_div(K, 32)), pq::kFoldThreads, 0, st>>>(part, part_max, chunks,
-                                                                                                    K, sumsq, amax);
+    dim3 grid(static_cast<unsigned>(slabs), static_cast<unsigned>(pq_ceil_div(K, kStatsCols)));
+    double *slab_sum = static_cast<double *>(ws);
+    float *slab_max = reinterpret_cast<float *>(slab_sum + slabs * K);
+    calib_stats_slab<<<grid, kStatsThreads, 0, st>>>(static_cast<const uint16_t *>(T), rows, K, ld, slab_sum, slab_max);
+    PQ_CUDA_OK(pq::launch_dependent(pq::fold_partials<double, 1, true>, dim3(static_cast<unsigned>(pq_ceil_div(K, pq::kFoldOutputs))),
+                                    dim3(pq::kFoldThreads), 0, st, static_cast<const double *>(slab_sum),
+                                    static_cast<const float *>(slab_max), slabs, K, sumsq, amax));
     return pq_launch_status();
 }
 

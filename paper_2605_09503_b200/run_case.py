@@ -31,6 +31,8 @@ def main():
     ap.add_argument("--iters", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--rot", type=int, default=4)
+    ap.add_argument("--graph", action="store_true",
+                    help="capture the timed launches in one CUDA graph (takes the host's launch rate out of the number)")
     args = ap.parse_args()
     dev = "cuda"
     M, N, K, R = args.M, args.N, args.K, args.rot
@@ -112,13 +114,24 @@ def main():
         fn(i)
     torch.cuda.synchronize()
     a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    a.record()
-    for i in range(args.iters):
-        fn(i)
-    b.record()
+    if args.graph:
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph):
+            for i in range(args.iters):
+                fn(i)
+        graph.replay()
+        torch.cuda.synchronize()
+        a.record()
+        graph.replay()
+        b.record()
+    else:
+        a.record()
+        for i in range(args.iters):
+            fn(i)
+        b.record()
     torch.cuda.synchronize()
     ms = a.elapsed_time(b) / args.iters
-    line = {"case": args.case, "M": M, "N": N, "K": K, "ms": ms}
+    line = {"case": args.case, "M": M, "N": N, "K": K, "ms": ms, "graph": args.graph}
     if work:
         line["TFLOP/s"] = work / ms / 1e9
     if bytes_moved:

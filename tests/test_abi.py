@@ -45,7 +45,7 @@ def test_status_strings_and_sizes(L):
     assert binding.sf_bytes(256, 512, binding.PQ_SF_LINEAR) == 256 * 32
     assert binding.sf_bytes(130, 512, binding.PQ_SF_TCGEN05) == 2 * 8 * 512
     assert binding.sf_bytes(130, 500, binding.PQ_SF_LINEAR) == 0
-    assert binding.workspace_bytes(binding.OP_CALIB_STATS, 4608, 3072) == 2 * 288 * 3072 * 4
+    assert binding.workspace_bytes(binding.OP_CALIB_STATS, 4608, 3072) == 36 * 3072 * (8 + 4)
     assert binding.workspace_bytes(binding.OP_GROUP_ERROR, 130, 512, 0, 7) >= 3 * 7 * 32 * 4
     assert binding.workspace_bytes(binding.OP_GEMM, 128, 64, 128) >= 4
     assert binding.workspace_bytes(99, 1, 1) == 0

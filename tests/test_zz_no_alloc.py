@@ -25,7 +25,7 @@ def test_rejects_problems_larger_than_the_static_array():
     limit = int(L.pq_calib_stats_static_max_bytes())
     assert limit == 8 << 20
     p = C.c_void_p(0x1000)
-    rows, K = 8192, 8192
+    rows, K = 32768, 8192
     assert B.workspace_bytes(B.OP_CALIB_STATS, rows, K) > limit
     assert L.pq_calib_stats_static(p, rows, K, K, p, p, None) == 5          # PQ_ERR_WORKSPACE
     assert L.pq_calib_stats_static(p, 0, K, K, p, p, None) == 2             # PQ_ERR_SHAPE
