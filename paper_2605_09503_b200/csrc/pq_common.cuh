@@ -241,21 +241,32 @@ cudaError_t launch_dependent(void (*kern)(KArgs...), dim3 grid, dim3 block, size
 //                  is added in fp64 from zero, then the slab sum is added to total[i].
 // WITH_MAX also folds vmax[i] = max(vmax[i], part_max[c][i]).
 // The additions are sequential per output but the loads are not: a block owns 16 consecutive
-// outputs, all its threads stage a batch of 128 partials per output in shared memory with
-// coalesced loads, then 16 lanes add them in order.
-constexpr int kFoldThreads = 256, kFoldOutputs = 16, kFoldBatch = 128;
+// outputs; batches of 64 partials per output are staged in shared memory with coalesced loads by
+// warps 1-7 while 16 lanes of warp 0 add the previous batch in order (two buffers).
+constexpr int kFoldThreads = 256, kFoldOutputs = 16, kFoldBatch = 64;
+
+template <typename PT, bool WITH_MAX>
+__device__ __forceinline__ void fold_stage(const PT *__restrict__ part, const float *__restrict__ part_max, int64_t c0,
+                                           int nc, int64_t n, int64_t i, bool live, int first, int step, PT *tile,
+                                           float *tile_max) {
+    const int o = threadIdx.x % kFoldOutputs;
+    for (int c = first; c < nc; c += step) {
+        tile[c * kFoldOutputs + o] = live ? __ldcs(part + (c0 + c) * n + i) : PT(0);
+        if (WITH_MAX) tile_max[c * kFoldOutputs + o] = live ? __ldcs(part_max + (c0 + c) * n + i) : 0.0f;
+    }
+}
 
 template <typename PT, int PER_SLAB, bool WITH_MAX>
 __global__ void __launch_bounds__(kFoldThreads)
 fold_partials(const PT *__restrict__ part, const float *__restrict__ part_max, int64_t count, int64_t n,
               double *__restrict__ total, float *__restrict__ vmax) {
     static_assert(kFoldBatch % PER_SLAB == 0, "a batch holds whole slabs");
-    __shared__ PT tile[kFoldBatch * kFoldOutputs];
-    __shared__ float tile_max[WITH_MAX ? kFoldBatch * kFoldOutputs : 1];
-    const int o = threadIdx.x % kFoldOutputs, g = threadIdx.x / kFoldOutputs;  // output, row of the batch
-    constexpr int kRowsPerPass = kFoldThreads / kFoldOutputs;
+    __shared__ PT tile[2][kFoldBatch * kFoldOutputs];
+    __shared__ float tile_max[2][WITH_MAX ? kFoldBatch * kFoldOutputs : 1];
+    constexpr int kRows = kFoldThreads / kFoldOutputs;  // batch rows covered by one pass of all threads
+    const int o = threadIdx.x % kFoldOutputs, g = threadIdx.x / kFoldOutputs;
     const int64_t i = static_cast<int64_t>(blockIdx.x) * kFoldOutputs + o;
-    const bool live = i < n, adder = threadIdx.x < kFoldOutputs;
+    const bool live = i < n, adder = threadIdx.x < kFoldOutputs, loader = threadIdx.x >= 32;
     double s = 0.0, slab = 0.0;
     float a = 0.0f;
     if (adder && live) {
@@ -263,39 +274,42 @@ fold_partials(const PT *__restrict__ part, const float *__restrict__ part_max, i
         if (WITH_MAX) a = vmax[i];
     }
     wait_for_prior_grid();
-    for (int64_t c0 = 0; c0 < count; c0 += kFoldBatch) {
+    const int64_t batches = (count + kFoldBatch - 1) / kFoldBatch;
+    fold_stage<PT, WITH_MAX>(part, part_max, 0, static_cast<int>(min(static_cast<int64_t>(kFoldBatch), count)), n, i, live,
+                             g, kRows, tile[0], tile_max[0]);
+    __syncthreads();
+    for (int64_t b = 0; b < batches; ++b) {
+        const int64_t c0 = b * kFoldBatch;
         const int nc = static_cast<int>(min(static_cast<int64_t>(kFoldBatch), count - c0));
-        __syncthreads();
-#pragma unroll
-        for (int c = g; c < kFoldBatch; c += kRowsPerPass) {
-            if (c < nc) {
-                tile[c * kFoldOutputs + o] = live ? __ldcs(part + (c0 + c) * n + i) : PT(0);
-                if (WITH_MAX) tile_max[c * kFoldOutputs + o] = live ? __ldcs(part_max + (c0 + c) * n + i) : 0.0f;
-            }
-        }
-        __syncthreads();
+        if (loader && b + 1 < batches)
+            fold_stage<PT, WITH_MAX>(part, part_max, c0 + kFoldBatch,
+                                     static_cast<int>(min(static_cast<int64_t>(kFoldBatch), count - c0 - kFoldBatch)), n, i,
+                                     live, g - 32 / kFoldOutputs, kRows - 32 / kFoldOutputs, tile[(b + 1) & 1],
+                                     tile_max[(b + 1) & 1]);
         if (adder) {
+            const PT *t = tile[b & 1];
+            const float *tm = tile_max[b & 1];
 #pragma unroll 8
             for (int c = 0; c < nc; ++c) {
                 if (PER_SLAB == 1) {
-                    s = __dadd_rn(s, static_cast<double>(tile[c * kFoldOutputs + o]));
+                    s = __dadd_rn(s, static_cast<double>(t[c * kFoldOutputs + o]));
                 } else {
-                    slab = __dadd_rn(slab, static_cast<double>(tile[c * kFoldOutputs + o]));
+                    slab = __dadd_rn(slab, static_cast<double>(t[c * kFoldOutputs + o]));
                     if ((c % PER_SLAB) == PER_SLAB - 1 || c0 + c == count - 1) {
                         s = __dadd_rn(s, slab);
                         slab = 0.0;
                     }
                 }
-                if (WITH_MAX) a = fmaxf(a, tile_max[c * kFoldOutputs + o]);
+                if (WITH_MAX) a = fmaxf(a, tm[c * kFoldOutputs + o]);
             }
         }
+        __syncthreads();
     }
     if (adder && live) {
         total[i] = s;
         if (WITH_MAX) vmax[i] = a;
     }
 }
-
 
 }  // namespace pq
 #endif  // __CUDACC__
