@@ -225,6 +225,26 @@ pq_status pq_linear_w4a4(const void *X, int64_t M, int64_t K, int64_t ld, const 
                          const float *ts_w, int64_t N, void *Y, int64_t ldy, void *ws,
                          size_t ws_bytes, void *stream);
 
+/* The runtime path of Eq. 8 for n independent batches through one layer (image batches, micro-
+ * batches): batch i is quantized into intermediates set i % n_sets and multiplied into Y[i].  The
+ * quantizer of a batch runs on one internal stream, the GEMMs on another, ordered by events, so the
+ * quantization of the following batches overlaps the GEMM of the current one (the quantizer's
+ * small thread blocks fit beside the GEMM's one CTA per SM), and every second GEMM is launched as a
+ * programmatic dependent of the one before it.  Results are those of n calls of pq_linear_w4a4.
+ *   X, Y   : HOST arrays of n device pointers (bf16 [M, K] ld, bf16 [M, N] ldy); read during the call.
+ *   xq, sfx: HOST arrays of n_sets device pointers, 2 <= n_sets <= 8, each as in pq_linear_w4a4;
+ *            with more sets the quantizer may run further ahead.
+ *   ws     : as for pq_gemm_w4a4 (shared by all batches).
+ * Ordering: all work is ordered after what `stream` already holds and before what is enqueued in
+ * `stream` afterwards; the call may be captured in a CUDA graph.  The first call on a device creates
+ * two streams and a few events (host objects, no device memory) that live until the process exits;
+ * calls on the same device from several host threads must be serialised by the caller. */
+pq_status pq_linear_w4a4_batched(int n, const void *const *X, int64_t M, int64_t K, int64_t ld,
+                                 const float *ts_x, uint8_t *const *xq, uint8_t *const *sfx,
+                                 int n_sets, const uint8_t *wq, const uint8_t *sfw,
+                                 const float *ts_w, int64_t N, void *const *Y, int64_t ldy, void *ws,
+                                 size_t ws_bytes, void *stream);
+
 /* The same runtime path for a caller whose tensors live in HOST memory (the end-to-end
  * measurement): copies X_host -> X_dev on `stream`, runs pq_linear_w4a4, copies Y_dev -> Y_host,
  * all asynchronously on `stream` (the caller synchronises the stream before reading Y_host).

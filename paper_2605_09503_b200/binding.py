@@ -51,6 +51,8 @@ _SIGNATURES = {
     "pq_gemm_w4a4": (_int, [_vp, _vp, _vp, _vp, _vp, _vp, _i64, _i64, _i64, _vp, _i64, _vp, _sz, _vp]),
     "pq_linear_w4a4": (_int, [_vp, _i64, _i64, _i64, _vp, _vp, _vp, _vp, _vp, _vp, _i64, _vp, _i64,
                               _vp, _sz, _vp]),
+    "pq_linear_w4a4_batched": (_int, [_int, _vp, _i64, _i64, _i64, _vp, _vp, _vp, _int, _vp, _vp, _vp, _i64, _vp, _i64,
+                                      _vp, _sz, _vp]),
     "pq_linear_w4a4_host": (_int, [_vp, _i64, _i64, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _i64, _vp, _vp,
                                    _vp, _sz, _vp]),
     "pq_fakequant_int": (_int, [_vp, _i64, _i64, _i64, pq_format, _vp, _vp, _i64, _vp]),
@@ -212,6 +214,23 @@ def pq_linear_w4a4(X, ts_x, xq, sfx, wq, sfw, ts_w, Y, ws):
     w, wb = _ws(ws)
     _check("pq_linear_w4a4", lib().pq_linear_w4a4(_p(X), M, K, X.stride(0), _p(ts_x), _p(xq), _p(sfx), _p(wq),
                                                   _p(sfw), _p(ts_w), N, _p(Y), Y.stride(0), w, wb, _stream()))
+
+
+def pq_linear_w4a4_batched(Xs, ts_x, xqs, sfxs, wq, sfw, ts_w, Ys, ws):
+    """n batches through one layer; Xs / Ys lists of n tensors, xqs / sfxs lists of n_sets intermediates."""
+    n, n_sets = len(Xs), len(xqs)
+    assert len(Ys) == n and len(sfxs) == n_sets
+    M, K = Xs[0].shape
+    N = wq.shape[0]
+    for x, y in zip(Xs, Ys):
+        _bf16(x)
+        assert x.shape == (M, K) and x.stride(0) == Xs[0].stride(0)
+        assert y.dtype == torch.bfloat16 and y.shape == (M, N) and y.stride(1) == 1 and y.stride(0) == Ys[0].stride(0)
+    arr = lambda ts: (C.c_void_p * len(ts))(*[t.data_ptr() for t in ts])
+    w, wb = _ws(ws)
+    _check("pq_linear_w4a4_batched", lib().pq_linear_w4a4_batched(
+        n, arr(Xs), M, K, Xs[0].stride(0), _p(ts_x), arr(xqs), arr(sfxs), n_sets, _p(wq), _p(sfw), _p(ts_w), N,
+        arr(Ys), Ys[0].stride(0), w, wb, _stream()))
 
 
 def pq_linear_w4a4_host(X_host, ts_x, X_dev, xq, sfx, wq, sfw, ts_w, Y_dev, Y_host, ws):

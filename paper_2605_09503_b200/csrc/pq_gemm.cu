@@ -49,6 +49,8 @@
 // and falls through to the common teardown (cluster barrier, tensor-memory release).
 #include <cuda.h>
 
+#include <mutex>
+
 #include "pq_common.cuh"
 
 namespace {
@@ -293,7 +295,11 @@ __device__ __forceinline__ uint32_t pack_bf16(uint32_t lo_bits, uint32_t hi_bits
 }
 
 // ---------------------------------------------------------------- kernel
-__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
+// Register budget: with 112 registers per thread the four warps an SM sub-partition gets from
+// this CTA leave it 2048 registers, room for two warps of a 32-register kernel, so a 256-thread
+// block of the activation quantizer can run on the SM beside the GEMM (batched linear path).
+constexpr int kMaxRegs = 112;
+__global__ void __cluster_dims__(2, 1, 1) __maxnreg__(kMaxRegs)
 gemm_w4a4_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                  const __grid_constant__ CUtensorMap map_y, const GemmParams p) {
     extern __shared__ uint8_t smem_raw[];
@@ -348,6 +354,9 @@ gemm_w4a4_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
     // while that kernel was finishing; its output (and any earlier work in the stream) is complete
     // and visible from here on.  A no-op for an ordinary launch.
     asm volatile("griddepcontrol.wait;" ::: "memory");
+    // ... and a kernel launched as this one's programmatic dependent may start its own set-up as
+    // soon as this kernel's CTAs leave their SMs.
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
     const int total_tiles = p.m_tiles * p.n_tiles;
 
@@ -656,7 +665,7 @@ int resident_pairs() {
 namespace {
 pq_status gemm_launch(const uint8_t *xq, const uint8_t *sfx, const float *ts_x, const uint8_t *wq, const uint8_t *sfw,
                       const float *ts_w, int64_t M, int64_t N, int64_t K, void *Y, int64_t ldy, void *ws,
-                      size_t ws_bytes, void *stream, bool after_quantizer) {
+                      size_t ws_bytes, void *stream, bool programmatic) {
     PQ_REQUIRE(xq && sfx && ts_x && wq && sfw && ts_w && Y, PQ_ERR_NULL);
     PQ_REQUIRE(M > 0 && N > 0 && K >= 64 && K % 64 == 0 && N % 8 == 0 && ldy >= N, PQ_ERR_SHAPE);
     PQ_REQUIRE(M < (1ll << 31) - 256 && N < (1ll << 31) - 256 && K < (1ll << 31), PQ_ERR_SHAPE);
@@ -706,7 +715,7 @@ pq_status gemm_launch(const uint8_t *xq, const uint8_t *sfx, const float *ts_x, 
     attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr.val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = &attr;
-    cfg.numAttrs = after_quantizer ? 1 : 0;
+    cfg.numAttrs = programmatic ? 1 : 0;
     PQ_CUDA_OK(cudaLaunchKernelEx(&cfg, gemm_w4a4_kernel, map_a, map_b, map_y, p));
     return PQ_OK;
 }
@@ -738,6 +747,89 @@ extern "C" pq_status pq_linear_w4a4_host(const void *X_host, int64_t M, int64_t 
     if (rc != PQ_OK) return rc;
     PQ_CUDA_OK(cudaMemcpyAsync(Y_host, Y_dev, static_cast<size_t>(M) * N * 2, cudaMemcpyDeviceToHost, st));
     return PQ_OK;
+}
+
+// ---------------------------------------------------------------- batches through one layer
+namespace {
+constexpr int kMaxSets = 8, kMaxPipeDevices = 64;
+
+// Two internal streams and the events that order them, created once per device (host objects,
+// no device memory).
+struct Pipe {
+    cudaStream_t q = nullptr, g = nullptr;
+    cudaEvent_t fork = nullptr, join_q = nullptr, join_g = nullptr;
+    cudaEvent_t q_done[kMaxSets] = {}, g_done[kMaxSets] = {};
+    bool ready = false;
+};
+
+Pipe *pipe_for_current_device() {
+    static std::mutex lock;
+    static Pipe pipes[kMaxPipeDevices];
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxPipeDevices) return nullptr;
+    std::lock_guard<std::mutex> guard(lock);
+    Pipe &p = pipes[dev];
+    if (!p.ready) {
+        bool ok = cudaStreamCreateWithFlags(&p.q, cudaStreamNonBlocking) == cudaSuccess &&
+                  cudaStreamCreateWithFlags(&p.g, cudaStreamNonBlocking) == cudaSuccess;
+        auto make = [&](cudaEvent_t *e) { ok = ok && cudaEventCreateWithFlags(e, cudaEventDisableTiming) == cudaSuccess; };
+        make(&p.fork), make(&p.join_q), make(&p.join_g);
+        for (int i = 0; i < kMaxSets; ++i) make(&p.q_done[i]), make(&p.g_done[i]);
+        if (!ok) {
+            (void)cudaGetLastError();
+            return nullptr;
+        }
+        p.ready = true;
+    }
+    return &p;
+}
+}  // namespace
+
+extern "C" pq_status pq_linear_w4a4_batched(int n, const void *const *X, int64_t M, int64_t K, int64_t ld,
+                                            const float *ts_x, uint8_t *const *xq, uint8_t *const *sfx, int n_sets,
+                                            const uint8_t *wq, const uint8_t *sfw, const float *ts_w, int64_t N,
+                                            void *const *Y, int64_t ldy, void *ws, size_t ws_bytes, void *stream) {
+    PQ_REQUIRE(X && xq && sfx && Y, PQ_ERR_NULL);
+    PQ_REQUIRE(n >= 1 && n_sets >= 2 && n_sets <= kMaxSets, PQ_ERR_SHAPE);
+    for (int i = 0; i < n; ++i) PQ_REQUIRE(X[i] && Y[i], PQ_ERR_NULL);
+    for (int s = 0; s < n_sets; ++s) PQ_REQUIRE(xq[s] && sfx[s], PQ_ERR_NULL);
+    Pipe *pipe = pipe_for_current_device();
+    if (!pipe) return PQ_ERR_CUDA;
+    cudaStream_t user = static_cast<cudaStream_t>(stream);
+    // fork: both internal streams start after everything already in the caller's stream
+    PQ_CUDA_OK(cudaEventRecord(pipe->fork, user));
+    PQ_CUDA_OK(cudaStreamWaitEvent(pipe->q, pipe->fork, 0));
+    PQ_CUDA_OK(cudaStreamWaitEvent(pipe->g, pipe->fork, 0));
+    pq_status rc = PQ_OK;
+    // The GEMMs go out in pairs: both quantizer events are awaited in front of the pair, so the
+    // second GEMM directly follows the first in its stream and may be its programmatic dependent
+    // (its set-up overlaps the first one's last tiles).
+    for (int i0 = 0; i0 < n && rc == PQ_OK; i0 += 2) {
+        const int i1 = (i0 + 2 < n) ? i0 + 2 : n;
+        for (int i = i0; i < i1 && rc == PQ_OK; ++i) {
+            const int s = i % n_sets;
+            // the GEMM that last read this set of intermediates has to be done with it
+            if (i >= n_sets && cudaStreamWaitEvent(pipe->q, pipe->g_done[s], 0) != cudaSuccess) rc = PQ_ERR_CUDA;
+            if (rc == PQ_OK) rc = pq_quant_act_nvfp4(X[i], M, K, ld, ts_x, xq[s], sfx[s], PQ_SF_TCGEN05, pipe->q);
+            if (rc == PQ_OK && cudaEventRecord(pipe->q_done[s], pipe->q) != cudaSuccess) rc = PQ_ERR_CUDA;
+            if (rc == PQ_OK && cudaStreamWaitEvent(pipe->g, pipe->q_done[s], 0) != cudaSuccess) rc = PQ_ERR_CUDA;
+        }
+        for (int i = i0; i < i1 && rc == PQ_OK; ++i) {
+            const int s = i % n_sets;
+            rc = gemm_launch(xq[s], sfx[s], ts_x, wq, sfw, ts_w, M, N, K, Y[i], ldy, ws, ws_bytes, pipe->g, i > i0);
+            if (rc == PQ_OK && cudaEventRecord(pipe->g_done[s], pipe->g) != cudaSuccess) rc = PQ_ERR_CUDA;
+        }
+    }
+    // join (also after an error, so that a stream capture in progress stays well-formed)
+    bool joined = cudaEventRecord(pipe->join_q, pipe->q) == cudaSuccess &&
+                  cudaEventRecord(pipe->join_g, pipe->g) == cudaSuccess &&
+                  cudaStreamWaitEvent(user, pipe->join_q, 0) == cudaSuccess &&
+                  cudaStreamWaitEvent(user, pipe->join_g, 0) == cudaSuccess;
+    if (!joined) {
+        (void)cudaGetLastError();
+        return rc == PQ_OK ? PQ_ERR_CUDA : rc;
+    }
+    return rc;
 }
 
 extern "C" pq_status pq_device_status(const void *ws, void *stream) {

@@ -15,6 +15,10 @@
 namespace {
 
 constexpr int kQuantThreads = 256;
+#ifndef PQ_ACT_THREADS
+#define PQ_ACT_THREADS 256
+#endif
+constexpr int kActThreads = PQ_ACT_THREADS;  // activation quantizer
 
 // ---------------------------------------------------------------- activations (no gather)
 // One thread per 16-channel group: a 32-byte load (one 256-bit instruction when the tensor is
@@ -37,21 +41,25 @@ __device__ __forceinline__ void load_group(const uint16_t *p, uint4 &lo, uint4 &
 }
 
 template <int SF_LAYOUT, bool WIDE>
-__global__ void __launch_bounds__(kQuantThreads)
+__global__ void __launch_bounds__(kActThreads)
 quant_nvfp4_kernel(const uint16_t *__restrict__ X, int64_t rows, int64_t rows_pad, int64_t K,
                    int64_t ld, const float *__restrict__ ts_ptr, uint8_t *__restrict__ codes,
                    uint8_t *__restrict__ sf) {
     const uint32_t gpr = static_cast<uint32_t>(K >> 4);  // groups per row
-    const int64_t first = static_cast<int64_t>(blockIdx.x) * kQuantThreads;
+    const int64_t first = static_cast<int64_t>(blockIdx.x) * kActThreads;
     const int64_t row0 = first / gpr;
     const uint32_t g0 = static_cast<uint32_t>(first - row0 * gpr) + threadIdx.x;
     const uint32_t dr = g0 / gpr;
     const int64_t row = row0 + dr;
     const uint32_t g = g0 - dr * gpr;
     const bool in_range = row < rows_pad, live = row < rows;
-    // a kernel launched as a programmatic dependent of this one (the GEMM of pq_linear_w4a4) may
-    // begin its set-up now; it still waits for this grid to complete before reading the results
-    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    // This kernel is launched as a programmatic dependent of whatever precedes it in the stream:
+    // its blocks may become resident while that kernel's last blocks run, and wait here until it
+    // has completed and its writes are visible (ordinary stream order from here on).  In turn a
+    // programmatic dependent of this kernel (the GEMM of pq_linear_w4a4) may begin its set-up now;
+    // it waits for this grid to complete before reading the results.
+    pq::wait_for_prior_grid();
+    pq::dependents_may_launch();
     const float ts = __ldg(ts_ptr);
 
     uint4 lo = make_uint4(0, 0, 0, 0), hi = lo;
@@ -280,15 +288,25 @@ extern "C" pq_status pq_quant_act_nvfp4(const void *X, int64_t M, int64_t K, int
     // 256-bit loads need 32-byte aligned groups
     const bool wide = (reinterpret_cast<uintptr_t>(X) & 31u) == 0 && ld % 16 == 0;
     const int64_t rows_idx = sf_layout == PQ_SF_TCGEN05 ? pq_ceil_div(M, 128) * 128 : M;
-    const int64_t blocks = pq_ceil_div(rows_idx * (K / 16), kQuantThreads);
+    const int64_t blocks = pq_ceil_div(rows_idx * (K / 16), kActThreads);
     PQ_REQUIRE(blocks < (1ll << 31), PQ_ERR_SHAPE);
     const unsigned grid = static_cast<unsigned>(blocks);
+    // The quantizer's blocks should be able to run on an SM beside a GEMM CTA (the batched linear
+    // path overlaps the two kernels): ask for the GEMM's shared-memory carve-out, otherwise an SM
+    // has to drain before it can switch between the two configurations.
+    static bool carveout_set = false;
+    if (!carveout_set) {
+        cudaFuncSetAttribute(quant_nvfp4_kernel<PQ_SF_TCGEN05, true>, cudaFuncAttributePreferredSharedMemoryCarveout, 100);
+        cudaFuncSetAttribute(quant_nvfp4_kernel<PQ_SF_TCGEN05, false>, cudaFuncAttributePreferredSharedMemoryCarveout, 100);
+        (void)cudaGetLastError();
+        carveout_set = true;
+    }
     if (sf_layout == PQ_SF_TCGEN05) {
-        if (wide) quant_nvfp4_kernel<PQ_SF_TCGEN05, true><<<grid, kQuantThreads, 0, st>>>(x, M, rows_idx, K, ld, ts_x, codes, sf);
-        else quant_nvfp4_kernel<PQ_SF_TCGEN05, false><<<grid, kQuantThreads, 0, st>>>(x, M, rows_idx, K, ld, ts_x, codes, sf);
+        if (wide) PQ_CUDA_OK(pq::launch_dependent(quant_nvfp4_kernel<PQ_SF_TCGEN05, true>, dim3(grid), dim3(kActThreads), 0, st, x, M, rows_idx, K, ld, ts_x, codes, sf));
+        else PQ_CUDA_OK(pq::launch_dependent(quant_nvfp4_kernel<PQ_SF_TCGEN05, false>, dim3(grid), dim3(kActThreads), 0, st, x, M, rows_idx, K, ld, ts_x, codes, sf));
     } else {
-        if (wide) quant_nvfp4_kernel<PQ_SF_LINEAR, true><<<grid, kQuantThreads, 0, st>>>(x, M, rows_idx, K, ld, ts_x, codes, sf);
-        else quant_nvfp4_kernel<PQ_SF_LINEAR, false><<<grid, kQuantThreads, 0, st>>>(x, M, rows_idx, K, ld, ts_x, codes, sf);
+        if (wide) PQ_CUDA_OK(pq::launch_dependent(quant_nvfp4_kernel<PQ_SF_LINEAR, true>, dim3(grid), dim3(kActThreads), 0, st, x, M, rows_idx, K, ld, ts_x, codes, sf));
+        else PQ_CUDA_OK(pq::launch_dependent(quant_nvfp4_kernel<PQ_SF_LINEAR, false>, dim3(grid), dim3(kActThreads), 0, st, x, M, rows_idx, K, ld, ts_x, codes, sf));
     }
     return pq_launch_status();
 }

@@ -100,6 +100,7 @@ class QuantLinear:
         self.sfx = torch.empty(B.sf_bytes(M_max, self.K, B.PQ_SF_TCGEN05), dtype=torch.uint8, device=dev)
         self.ws = B.workspace(B.OP_GEMM, M_max, self.K, self.N)
         self.M_max = M_max
+        self._sets = []          # further (xq, sfx) pairs for forward_batches
 
     def __call__(self, X, Y=None):
         M = X.shape[0]
@@ -108,6 +109,18 @@ class QuantLinear:
             Y = torch.empty(M, self.N, dtype=torch.bfloat16, device=X.device)
         B.pq_linear_w4a4(X, self.ts_x, self.xq[:M], self.sfx, self.wq, self.sfw, self.ts_w, Y, self.ws)
         return Y
+
+    def forward_batches(self, Xs, Ys, n_sets=4):
+        """Independent batches through the layer, the quantizer of the next batches overlapped with
+        the GEMM of the current one (pq_linear_w4a4_batched).  Extra sets of intermediates are kept."""
+        M = Xs[0].shape[0]
+        assert M <= self.M_max
+        while len(self._sets) < n_sets:
+            self._sets.append((torch.empty_like(self.xq), torch.empty_like(self.sfx)))
+        xqs = [self.xq[:M]] + [a[:M] for a, _ in self._sets[:n_sets - 1]]
+        sfxs = [self.sfx] + [b for _, b in self._sets[:n_sets - 1]]
+        B.pq_linear_w4a4_batched(Xs, self.ts_x, xqs, sfxs, self.wq, self.sfw, self.ts_w, Ys, self.ws)
+        return Ys
 
     def check(self):
         """Synchronise and raise if a bounded device-side wait expired."""

@@ -14,7 +14,7 @@ import torch
 
 from . import binding as B
 
-CASES = ["gemm", "quant", "linear", "stats", "error", "error_perm", "fakequant", "fakequant_perm", "quant_weight",
+CASES = ["gemm", "quant", "linear", "batched", "stats", "error", "error_perm", "fakequant", "fakequant_perm", "quant_weight",
          "quant_weight_perm", "select_perm"]
 
 
@@ -52,7 +52,17 @@ def main():
     perms = torch.stack([torch.randperm(K, device=dev, generator=g) for _ in range(max(args.P, 1))]).to(torch.int32)
     work = bytes_moved = 0
 
-    if args.case in ("gemm", "linear"):
+    if args.case == "batched":
+        # one call = `rot` independent batches through the layer; time is reported per batch
+        X = [acts(M) for _ in range(R)]
+        xq = [torch.empty(M, K // 2, dtype=torch.uint8, device=dev) for _ in range(4)]
+        sfx = [torch.empty(B.sf_bytes(M, K, 1), dtype=torch.uint8, device=dev) for _ in range(4)]
+        wq, sfw = rbytes(N, K // 2), rbytes(B.sf_bytes(N, K, 1), hi=0x60)
+        Y = [torch.empty(M, N, dtype=torch.bfloat16, device=dev) for _ in range(R)]
+        ws = B.workspace(B.OP_GEMM, M, K, N)
+        work = 2.0 * M * N * K * R
+        fn = lambda i: B.pq_linear_w4a4_batched(X, ts, xq, sfx, wq, sfw, tsw, Y, ws)
+    elif args.case in ("gemm", "linear"):
         xq = [rbytes(M, K // 2) for _ in range(R)]
         sfx = [rbytes(B.sf_bytes(M, K, 1), hi=0x60) for _ in range(R)]
         wq = [rbytes(N, K // 2) for _ in range(R)]
@@ -132,6 +142,8 @@ def main():
     torch.cuda.synchronize()
     ms = a.elapsed_time(b) / args.iters
     line = {"case": args.case, "M": M, "N": N, "K": K, "ms": ms, "graph": args.graph}
+    if args.case == "batched":
+        line["ms_per_batch"] = ms / R
     if work:
         line["TFLOP/s"] = work / ms / 1e9
     if bytes_moved:
