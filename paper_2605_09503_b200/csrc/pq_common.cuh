@@ -241,32 +241,30 @@ cudaError_t launch_dependent(void (*kern)(KArgs...), dim3 grid, dim3 block, size
 //                  is added in fp64 from zero, then the slab sum is added to total[i].
 // WITH_MAX also folds vmax[i] = max(vmax[i], part_max[c][i]).
 // The additions are sequential per output but the loads are not: a block owns 16 consecutive
-// outputs; batches of 64 partials per output are staged in shared memory with coalesced loads by
-// warps 1-7 while 16 lanes of warp 0 add the previous batch in order (two buffers).
-constexpr int kFoldThreads = 256, kFoldOutputs = 16, kFoldBatch = 64;
+// outputs and stages up to kFoldRoundMax partials per output in (dynamic) shared memory with
+// coalesced loads, all in flight at once, then 16 threads add them in order.  Typical sizes take a
+// single round.
+constexpr int kFoldThreads = 256, kFoldOutputs = 16, kFoldRoundMax = 512;
 
 template <typename PT, bool WITH_MAX>
-__device__ __forceinline__ void fold_stage(const PT *__restrict__ part, const float *__restrict__ part_max, int64_t c0,
-                                           int nc, int64_t n, int64_t i, bool live, int first, int step, PT *tile,
-                                           float *tile_max) {
-    const int o = threadIdx.x % kFoldOutputs;
-    for (int c = first; c < nc; c += step) {
-        tile[c * kFoldOutputs + o] = live ? __ldcs(part + (c0 + c) * n + i) : PT(0);
-        if (WITH_MAX) tile_max[c * kFoldOutputs + o] = live ? __ldcs(part_max + (c0 + c) * n + i) : 0.0f;
-    }
+constexpr size_t fold_smem_bytes(int64_t count) {
+    return static_cast<size_t>(count < kFoldRoundMax ? count : kFoldRoundMax) * kFoldOutputs *
+           (sizeof(PT) + (WITH_MAX ? sizeof(float) : 0));
 }
 
 template <typename PT, int PER_SLAB, bool WITH_MAX>
 __global__ void __launch_bounds__(kFoldThreads)
 fold_partials(const PT *__restrict__ part, const float *__restrict__ part_max, int64_t count, int64_t n,
               double *__restrict__ total, float *__restrict__ vmax) {
-    static_assert(kFoldBatch % PER_SLAB == 0, "a batch holds whole slabs");
-    __shared__ PT tile[2][kFoldBatch * kFoldOutputs];
-    __shared__ float tile_max[2][WITH_MAX ? kFoldBatch * kFoldOutputs : 1];
-    constexpr int kRows = kFoldThreads / kFoldOutputs;  // batch rows covered by one pass of all threads
+    static_assert(kFoldRoundMax % PER_SLAB == 0, "a round holds whole slabs");
+    extern __shared__ __align__(16) unsigned char fold_smem[];
+    const int round_rows = static_cast<int>(min(static_cast<int64_t>(kFoldRoundMax), count));
+    PT *tile = reinterpret_cast<PT *>(fold_smem);
+    float *tile_max = reinterpret_cast<float *>(fold_smem + static_cast<size_t>(round_rows) * kFoldOutputs * sizeof(PT));
+    constexpr int kRows = kFoldThreads / kFoldOutputs;  // rows of the round covered by one pass of all threads
     const int o = threadIdx.x % kFoldOutputs, g = threadIdx.x / kFoldOutputs;
     const int64_t i = static_cast<int64_t>(blockIdx.x) * kFoldOutputs + o;
-    const bool live = i < n, adder = threadIdx.x < kFoldOutputs, loader = threadIdx.x >= 32;
+    const bool live = i < n, adder = threadIdx.x < kFoldOutputs;
     double s = 0.0, slab = 0.0;
     float a = 0.0f;
     if (adder && live) {
@@ -274,41 +272,49 @@ fold_partials(const PT *__restrict__ part, const float *__restrict__ part_max, i
         if (WITH_MAX) a = vmax[i];
     }
     wait_for_prior_grid();
-    const int64_t batches = (count + kFoldBatch - 1) / kFoldBatch;
-    fold_stage<PT, WITH_MAX>(part, part_max, 0, static_cast<int>(min(static_cast<int64_t>(kFoldBatch), count)), n, i, live,
-                             g, kRows, tile[0], tile_max[0]);
-    __syncthreads();
-    for (int64_t b = 0; b < batches; ++b) {
-        const int64_t c0 = b * kFoldBatch;
-        const int nc = static_cast<int>(min(static_cast<int64_t>(kFoldBatch), count - c0));
-        if (loader && b + 1 < batches)
-            fold_stage<PT, WITH_MAX>(part, part_max, c0 + kFoldBatch,
-                                     static_cast<int>(min(static_cast<int64_t>(kFoldBatch), count - c0 - kFoldBatch)), n, i,
-                                     live, g - 32 / kFoldOutputs, kRows - 32 / kFoldOutputs, tile[(b + 1) & 1],
-                                     tile_max[(b + 1) & 1]);
+    for (int64_t c0 = 0; c0 < count; c0 += kFoldRoundMax) {
+        const int nc = static_cast<int>(min(static_cast<int64_t>(kFoldRoundMax), count - c0));
+        __syncthreads();
+        for (int c = g; c < nc; c += kRows) {
+            tile[c * kFoldOutputs + o] = live ? __ldcs(part + (c0 + c) * n + i) : PT(0);
+            if (WITH_MAX) tile_max[c * kFoldOutputs + o] = live ? __ldcs(part_max + (c0 + c) * n + i) : 0.0f;
+        }
+        __syncthreads();
         if (adder) {
-            const PT *t = tile[b & 1];
-            const float *tm = tile_max[b & 1];
 #pragma unroll 8
             for (int c = 0; c < nc; ++c) {
                 if (PER_SLAB == 1) {
-                    s = __dadd_rn(s, static_cast<double>(t[c * kFoldOutputs + o]));
+                    s = __dadd_rn(s, static_cast<double>(tile[c * kFoldOutputs + o]));
                 } else {
-                    slab = __dadd_rn(slab, static_cast<double>(t[c * kFoldOutputs + o]));
+                    slab = __dadd_rn(slab, static_cast<double>(tile[c * kFoldOutputs + o]));
                     if ((c % PER_SLAB) == PER_SLAB - 1 || c0 + c == count - 1) {
                         s = __dadd_rn(s, slab);
                         slab = 0.0;
                     }
                 }
-                if (WITH_MAX) a = fmaxf(a, tm[c * kFoldOutputs + o]);
+                if (WITH_MAX) a = fmaxf(a, tile_max[c * kFoldOutputs + o]);
             }
         }
-        __syncthreads();
     }
     if (adder && live) {
         total[i] = s;
         if (WITH_MAX) vmax[i] = a;
     }
+}
+
+// Launch of fold_partials as a programmatic dependent of the kernel that wrote the partials.
+template <typename PT, int PER_SLAB, bool WITH_MAX>
+cudaError_t launch_fold(const PT *part, const float *part_max, int64_t count, int64_t n, double *total, float *vmax,
+                        cudaStream_t st) {
+    const size_t smem = fold_smem_bytes<PT, WITH_MAX>(count);
+    if (smem > 48 * 1024) {
+        const cudaError_t e = cudaFuncSetAttribute(fold_partials<PT, PER_SLAB, WITH_MAX>,
+                                                   cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
+        if (e != cudaSuccess) return e;
+    }
+    return launch_dependent(fold_partials<PT, PER_SLAB, WITH_MAX>,
+                            dim3(static_cast<unsigned>((n + kFoldOutputs - 1) / kFoldOutputs)), dim3(kFoldThreads), smem, st,
+                            part, part_max, count, n, total, vmax);
 }
 
 }  // namespace pq

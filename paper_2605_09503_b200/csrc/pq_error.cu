@@ -187,10 +187,7 @@ group_error_gather(const uint16_t *__restrict__ T, int64_t rows, int64_t K, int6
 
 template <typename PT, int PER_SLAB>
 pq_status fold(const void *part, int64_t count, int64_t n, double *err, cudaStream_t st) {
-    PQ_CUDA_OK(pq::launch_dependent(pq::fold_partials<PT, PER_SLAB, false>,
-                                    dim3(static_cast<unsigned>(pq_ceil_div(n, pq::kFoldOutputs))), dim3(pq::kFoldThreads),
-                                    0, st, static_cast<const PT *>(part), static_cast<const float *>(nullptr), count, n,
-                                    err, static_cast<float *>(nullptr)));
+    PQ_CUDA_OK((pq::launch_fold<PT, PER_SLAB, false>(static_cast<const PT *>(part), nullptr, count, n, err, nullptr, st)));
     return pq_launch_status();
 }
 

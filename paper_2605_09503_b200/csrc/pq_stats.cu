@@ -121,9 +121,7 @@ extern "C" pq_status pq_calib_stats(const void *T, int64_t rows, int64_t K, int6
     double *slab_sum = static_cast<double *>(ws);
     float *slab_max = reinterpret_cast<float *>(slab_sum + slabs * K);
     calib_stats_slab<<<grid, kStatsThreads, 0, st>>>(static_cast<const uint16_t *>(T), rows, K, ld, slab_sum, slab_max);
-    PQ_CUDA_OK(pq::launch_dependent(pq::fold_partials<double, 1, true>, dim3(static_cast<unsigned>(pq_ceil_div(K, pq::kFoldOutputs))),
-                                    dim3(pq::kFoldThreads), 0, st, static_cast<const double *>(slab_sum),
-                                    static_cast<const float *>(slab_max), slabs, K, sumsq, amax));
+    PQ_CUDA_OK((pq::launch_fold<double, 1, true>(slab_sum, slab_max, slabs, K, sumsq, amax, st)));
     return pq_launch_status();
 }
 
