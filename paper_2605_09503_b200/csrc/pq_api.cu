@@ -27,8 +27,12 @@ extern "C" size_t pq_workspace_bytes(int op, int64_t rows, int64_t K, int64_t N,
     switch (op) {
         case PQ_OP_CALIB_STATS: return round256(static_cast<size_t>(slabs) * K * (sizeof(double) + sizeof(float)));
         case PQ_OP_SELECT_PERM: return round256(static_cast<size_t>(P > 0 ? P : 1) * K * sizeof(uint64_t));
-        case PQ_OP_GROUP_ERROR:
-            return round256(static_cast<size_t>(chunks) * (P > 0 ? P : 1) * (K / 16 + 1) * sizeof(float));
+        case PQ_OP_GROUP_ERROR: {
+            // fp32 chunk partials of P candidate orders, or fp64 slab sums of the original order
+            const size_t by_chunk = static_cast<size_t>(chunks) * (P > 0 ? P : 1) * (K / 16 + 1) * sizeof(float);
+            const size_t by_slab = static_cast<size_t>(slabs) * (K / 16 + 1) * sizeof(double);
+            return round256(by_chunk > by_slab ? by_chunk : by_slab);
+        }
         case PQ_OP_QUANT_WEIGHT: return 256;
         case PQ_OP_GEMM: return 256;
         default: return 0;

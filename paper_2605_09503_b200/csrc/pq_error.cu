@@ -40,19 +40,30 @@ __device__ __forceinline__ float group_sse_lane(const float (&x)[8], float ts, f
 
 // ---------------------------------------------------------------- original order
 constexpr int kDirectThreads = 128;
-constexpr int kDirectRows = 8;  // rows in flight per thread (2 x 16 bytes each)
+constexpr int kDirectRows = 4;  // rows in flight per thread (2 x 16 bytes each)
+
+// Decode scale d = sf * ts and its reciprocal for each of the 256 scale bytes (they depend on the
+// byte only): built once per block, so a group costs one division, one convert and one 8-byte
+// shared-memory load instead of a second convert, a multiply and an IEEE reciprocal.
+__device__ __forceinline__ void build_scale_table(float2 *table, float ts) {
+    for (int b = threadIdx.x; b < 256; b += blockDim.x) {
+        const float d = __fmul_rn(pq::e4m3_to_f32(static_cast<uint32_t>(b)), ts);
+        table[b] = make_float2(d, d > 0.0f ? __frcp_rn(d) : 0.0f);
+    }
+}
 
 // Error of one row's 16 channels held by this lane; TEAM16 = group / 16 adjacent lanes share a group.
+// c6 = 6 * ts (NVFP4 only).
 template <int KIND, int TEAM16>
-__device__ __forceinline__ float row_sse16(const uint4 &lo, const uint4 &hi, float ts, float Qf) {
+__device__ __forceinline__ float row_sse16(const uint4 &lo, const uint4 &hi, float c6, const float2 *table, float Qf) {
     float xa[8], xb[8];
     pq::unpack8(lo, xa);
     pq::unpack8(hi, xb);
     const float amax = pq::team_max<TEAM16>(fmaxf(pq::absmax8(xa), pq::absmax8(xb)));
     float qa[8], qb[8], d, r;
     if (KIND == 0) {
-        uint32_t sf8;
-        pq::nvfp4_scale(amax, ts, sf8, d, r);
+        const float2 dr = table[pq::f32_to_e4m3(__fdiv_rn(amax, c6))];
+        d = dr.x, r = dr.y;
         pq::nvfp4_levels_abs(xa, r, qa);
         pq::nvfp4_levels_abs(xb, r, qb);
     } else {
@@ -73,10 +84,11 @@ static_assert(kDirectRuns == 16, "a warp holds two chunks of 16 runs");
 // partials of a group meet in shared memory and one thread adds them in fp64 in chunk order;
 // the workspace receives fp64 slab sums [slab][K/g].
 template <int KIND, int TEAM16>
-__global__ void __launch_bounds__(kDirectThreads)
+__global__ void __launch_bounds__(kDirectThreads, 8)
 group_error_direct(const uint16_t *__restrict__ T, int64_t rows, int64_t K, int64_t ld,
                    const float *__restrict__ ts_ptr, float Qf, double *__restrict__ slab_part /*[slabs, K/g]*/) {
     __shared__ float part_s[kSlabChunks][kDirectRuns];
+    __shared__ float2 scale_table[KIND == 0 ? 256 : 1];
     pq::dependents_may_launch();
     const int runs = static_cast<int>(K >> 4);  // K % (16 * TEAM16) == 0
     const int c = threadIdx.x / kDirectRuns, j = threadIdx.x % kDirectRuns;
@@ -88,6 +100,11 @@ group_error_direct(const uint16_t *__restrict__ T, int64_t rows, int64_t K, int6
     const bool live = run < runs && r0 < rows;
     const int n = live ? static_cast<int>(min(static_cast<int64_t>(PQ_CHUNK_ROWS), rows - r0)) : 0;
     const float ts = (KIND == 0) ? __ldg(ts_ptr) : 1.0f;
+    const float c6 = __fmul_rn(6.0f, ts);
+    if (KIND == 0) {
+        build_scale_table(scale_table, ts);
+        __syncthreads();
+    }
     const uint16_t *p = T + (live ? r0 * ld + static_cast<int64_t>(run) * 16 : 0);
     float acc = 0.0f;
 #pragma unroll 1
@@ -103,7 +120,7 @@ group_error_direct(const uint16_t *__restrict__ T, int64_t rows, int64_t K, int6
         }
         // rows past the end are all-zero groups: their error is +0.0 and adding it changes nothing
 #pragma unroll
-        for (int u = 0; u < kDirectRows; ++u) acc = __fadd_rn(acc, row_sse16<KIND, TEAM16>(lo[u], hi[u], ts, Qf));
+        for (int u = 0; u < kDirectRows; ++u) acc = __fadd_rn(acc, row_sse16<KIND, TEAM16>(lo[u], hi[u], c6, scale_table, Qf));
     }
     part_s[c][j] = acc;
     __syncthreads();

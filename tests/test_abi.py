@@ -46,6 +46,9 @@ def test_status_strings_and_sizes(L):
     assert binding.sf_bytes(130, 512, binding.PQ_SF_TCGEN05) == 2 * 8 * 512
     assert binding.sf_bytes(130, 500, binding.PQ_SF_LINEAR) == 0
     assert binding.workspace_bytes(binding.OP_CALIB_STATS, 4608, 3072) == 36 * 3072 * (8 + 4)
+    # group error: fp32 per (chunk, order, group) for candidate orders, fp64 per (slab, group) otherwise
+    assert binding.workspace_bytes(binding.OP_GROUP_ERROR, 5, 4096, 0, 1) >= 1 * 256 * 8
+    assert binding.workspace_bytes(binding.OP_GROUP_ERROR, 4608, 3072, 0, 6) >= 288 * 6 * 192 * 4
     assert binding.workspace_bytes(binding.OP_GROUP_ERROR, 130, 512, 0, 7) >= 3 * 7 * 32 * 4
     assert binding.workspace_bytes(binding.OP_GEMM, 128, 64, 128) >= 4
     assert binding.workspace_bytes(99, 1, 1) == 0

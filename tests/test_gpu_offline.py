@@ -209,3 +209,26 @@ def test_fakequant_int_bit_exact(bits, group, rows, K, with_perm):
         B.pq_fakequant_int(dev(x), (1, bits, group), ident, a)
         B.pq_fakequant_int(dev(x), (1, bits, group), None, b)
         assert torch.equal(a.view(torch.int16), b.view(torch.int16))
+
+
+@pytest.mark.parametrize("rows,K", [(5, 4096), (16, 512), (17, 512), (129, 3072), (300, 1024)])
+def test_workspaces_are_not_overrun(rows, K):
+    """The reductions write only inside the bytes pq_workspace_bytes asks for (guard words behind them stay)."""
+    x = dev(inputs.activations(small_cfg(rows, K), 5, 0))
+    ts = dev(torch.tensor([0.02], dtype=torch.float32))
+    perms = dev(torch.stack([torch.randperm(K) for _ in range(3)]).to(torch.int32))
+
+    def guarded(op, P=0):
+        need = B.workspace_bytes(op, rows, K, 0, P)
+        buf = torch.full((need + 4096,), 0xA5, dtype=torch.uint8, device=DEV)
+        return buf, buf[:need], need
+
+    buf, ws, need = guarded(B.OP_CALIB_STATS)
+    B.pq_calib_stats(x, torch.zeros(K, dtype=torch.float64, device=DEV), torch.zeros(K, dtype=torch.float32, device=DEV), ws)
+    assert bool((buf[need:] == 0xA5).all())
+    for fmt in FORMATS:
+        for pm, P in ((None, 1), (perms, 3)):
+            buf, ws, need = guarded(B.OP_GROUP_ERROR, P)
+            err = torch.zeros(P, K // fmt[2], dtype=torch.float64, device=DEV)
+            B.pq_group_error(x, fmt, ts, pm, err, ws)
+            assert bool((buf[need:] == 0xA5).all())
