@@ -15,19 +15,27 @@
 namespace {
 
 constexpr int kQuantThreads = 256;
-#ifndef PQ_ACT_THREADS
-#define PQ_ACT_THREADS 256
-#endif
-constexpr int kActThreads = PQ_ACT_THREADS;  // activation quantizer
+constexpr int kTileRows = 8;                    // blocks of the streaming kernels: 32 lanes along K x 8 rows
+constexpr int kActThreads = 32 * kTileRows;     // activation quantizer
+constexpr unsigned kGridYMax = 65535;
+
+// Row block of a (x = column chunk, y/z = row block) grid; y alone is limited to 65535 blocks.
+__device__ __forceinline__ int64_t row_block_index() {
+    return static_cast<int64_t>(blockIdx.z) * kGridYMax + blockIdx.y;
+}
+inline dim3 tile_grid(int64_t col_chunks, int64_t row_blocks) {
+    const int64_t z = pq_ceil_div(row_blocks, kGridYMax);
+    return dim3(static_cast<unsigned>(col_chunks), static_cast<unsigned>(row_blocks < kGridYMax ? row_blocks : kGridYMax),
+                static_cast<unsigned>(z));
+}
 
 // ---------------------------------------------------------------- activations (no gather)
 // One thread per 16-channel group: a 32-byte load (one 256-bit instruction when the tensor is
 // 32-byte aligned), the group's absmax, scale and codes in registers, an 8-byte store of codes.
 // The scale bytes of four adjacent groups are collected with shuffles into one 32-bit store
 // (adjacent in both scale layouts).  The index space covers the rows padded to a multiple of 128
-// in the tensor-core layout; padding rows only write zero scale bytes.  A block owns 256
-// consecutive groups of the flat (row, group) space, so its starting row and group need one
-// 64-bit division per block and each thread a 32-bit one.
+// in the tensor-core layout; padding rows only write zero scale bytes.  A block owns 8 rows x 32
+// consecutive groups (a warp = 1 KB of one row), so no thread divides anything.
 template <bool WIDE>
 __device__ __forceinline__ void load_group(const uint16_t *p, uint4 &lo, uint4 &hi) {
     if (WIDE) {
@@ -46,13 +54,9 @@ quant_nvfp4_kernel(const uint16_t *__restrict__ X, int64_t rows, int64_t rows_pa
                    int64_t ld, const float *__restrict__ ts_ptr, uint8_t *__restrict__ codes,
                    uint8_t *__restrict__ sf) {
     const uint32_t gpr = static_cast<uint32_t>(K >> 4);  // groups per row
-    const int64_t first = static_cast<int64_t>(blockIdx.x) * kActThreads;
-    const int64_t row0 = first / gpr;
-    const uint32_t g0 = static_cast<uint32_t>(first - row0 * gpr) + threadIdx.x;
-    const uint32_t dr = g0 / gpr;
-    const int64_t row = row0 + dr;
-    const uint32_t g = g0 - dr * gpr;
-    const bool in_range = row < rows_pad, live = row < rows;
+    const uint32_t g = blockIdx.x * 32u + threadIdx.x;
+    const int64_t row = row_block_index() * kTileRows + threadIdx.y;
+    const bool in_range = row < rows_pad && g < gpr, live = row < rows && g < gpr;
     // This kernel is launched as a programmatic dependent of whatever precedes it in the stream:
     // its blocks may become resident while that kernel's last blocks run, and wait here until it
     // has completed and its writes are visible (ordinary stream order from here on).  In turn a
@@ -91,20 +95,21 @@ quant_nvfp4_kernel(const uint16_t *__restrict__ X, int64_t rows, int64_t rows_pa
 }
 
 // ---------------------------------------------------------------- weights
+// blockDim (32, 8): lane = 8 adjacent channels, threadIdx.y + blockIdx.y strides over the rows.
 __global__ void amax_all_kernel(const uint16_t *__restrict__ W, int64_t rows, int64_t K, int64_t ld,
                                 unsigned int *__restrict__ amax_bits) {
-    const int64_t oct_per_row = K >> 3;
-    const int64_t total = rows * oct_per_row;
+    const int64_t oct = static_cast<int64_t>(blockIdx.x) * 32 + threadIdx.x;
     float a = 0.0f;
-    for (int64_t idx = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x; idx < total;
-         idx += static_cast<int64_t>(gridDim.x) * blockDim.x) {
-        const int64_t row = idx / oct_per_row, oct = idx - row * oct_per_row;
-        float x[8];
-        pq::unpack8(__ldg(reinterpret_cast<const uint4 *>(W + row * ld + oct * 8)), x);
-        a = fmaxf(a, pq::absmax8(x));
+    if (oct * 8 < K) {
+        for (int64_t row = static_cast<int64_t>(blockIdx.y) * kTileRows + threadIdx.y; row < rows;
+             row += static_cast<int64_t>(gridDim.y) * kTileRows) {
+            float x[8];
+            pq::unpack8(__ldg(reinterpret_cast<const uint4 *>(W + row * ld + oct * 8)), x);
+            a = fmaxf(a, pq::absmax8(x));
+        }
     }
     for (int m = 16; m; m >>= 1) a = fmaxf(a, __shfl_xor_sync(0xFFFFFFFFu, a, m));
-    if ((threadIdx.x & 31) == 0 && a > 0.0f) atomicMax(amax_bits, __float_as_uint(a));
+    if (threadIdx.x == 0 && a > 0.0f) atomicMax(amax_bits, __float_as_uint(a));
 }
 
 __global__ void weight_scale_kernel(const unsigned int *__restrict__ amax_bits, float *ts) {
@@ -193,29 +198,24 @@ __device__ __forceinline__ uint4 fakequant8(const float (&x)[8], float Qf) {
     return make_uint4(w[0], w[1], w[2], w[3]);
 }
 
+// blockDim (32, 8): a warp = 32 adjacent octets (512 bytes) of one row; teams never straddle a
+// warp (K % (8 TEAM) == 0 and 32 % TEAM == 0), dead lanes carry zeros through the shuffles.
 template <int TEAM>
 __global__ void __launch_bounds__(kQuantThreads)
 fakequant_int_kernel(const uint16_t *__restrict__ T, int64_t rows, int64_t K, int64_t ld, float Qf,
                      uint16_t *__restrict__ out, int64_t ldo) {
-    const int64_t oct_per_row = K >> 3;
-    const int64_t total = rows * oct_per_row;
-    const int64_t stride = static_cast<int64_t>(gridDim.x) * kQuantThreads;
-    const int64_t warp_first = (static_cast<int64_t>(blockIdx.x) * kQuantThreads + threadIdx.x) & ~31ll;
-    for (int64_t base = warp_first; base < total; base += stride) {
-        const int64_t idx = base + (threadIdx.x & 31);
-        const bool live = idx < total;
-        const int64_t row = live ? idx / oct_per_row : 0;
-        const int64_t oct = live ? idx - row * oct_per_row : 0;
-        float x[8];
-        if (live) {
-            pq::unpack8(__ldcs(reinterpret_cast<const uint4 *>(T + row * ld + oct * 8)), x);
-        } else {
+    const int64_t oct = static_cast<int64_t>(blockIdx.x) * 32 + threadIdx.x;
+    const int64_t row = row_block_index() * kTileRows + threadIdx.y;
+    const bool live = row < rows && oct * 8 < K;
+    float x[8];
+    if (live) {
+        pq::unpack8(__ldcs(reinterpret_cast<const uint4 *>(T + row * ld + oct * 8)), x);
+    } else {
 #pragma unroll
-            for (int i = 0; i < 8; ++i) x[i] = 0.0f;
-        }
-        const uint4 o = fakequant8<TEAM>(x, Qf);
-        if (live) __stcs(reinterpret_cast<uint4 *>(out + row * ldo + oct * 8), o);
+        for (int i = 0; i < 8; ++i) x[i] = 0.0f;
     }
+    const uint4 o = fakequant8<TEAM>(x, Qf);
+    if (live) __stcs(reinterpret_cast<uint4 *>(out + row * ldo + oct * 8), o);
 }
 
 template <int TEAM>
@@ -288,9 +288,9 @@ extern "C" pq_status pq_quant_act_nvfp4(const void *X, int64_t M, int64_t K, int
     // 256-bit loads need 32-byte aligned groups
     const bool wide = (reinterpret_cast<uintptr_t>(X) & 31u) == 0 && ld % 16 == 0;
     const int64_t rows_idx = sf_layout == PQ_SF_TCGEN05 ? pq_ceil_div(M, 128) * 128 : M;
-    const int64_t blocks = pq_ceil_div(rows_idx * (K / 16), kActThreads);
-    PQ_REQUIRE(blocks < (1ll << 31), PQ_ERR_SHAPE);
-    const unsigned grid = static_cast<unsigned>(blocks);
+    PQ_REQUIRE(K / 16 <= 32ll * 0x7FFFFFFF && rows_idx / kTileRows < static_cast<int64_t>(kGridYMax) * 65535, PQ_ERR_SHAPE);
+    const dim3 grid = tile_grid(pq_ceil_div(K / 16, 32), pq_ceil_div(rows_idx, kTileRows));
+    const dim3 block(32, kTileRows);
     // The quantizer's blocks should be able to run on an SM beside a GEMM CTA (the batched linear
     // path overlaps the two kernels): ask for the GEMM's shared-memory carve-out, otherwise an SM
     // has to drain before it can switch between the two configurations.
@@ -302,11 +302,11 @@ extern "C" pq_status pq_quant_act_nvfp4(const void *X, int64_t M, int64_t K, int
         carveout_set = true;
     }
     if (sf_layout == PQ_SF_TCGEN05) {
-        if (wide) PQ_CUDA_OK(pq::launch_dependent(quant_nvfp4_kernel<PQ_SF_TCGEN05, true>, dim3(grid), dim3(kActThreads), 0, st, x, M, rows_idx, K, ld, ts_x, codes, sf));
-        else PQ_CUDA_OK(pq::launch_dependent(quant_nvfp4_kernel<PQ_SF_TCGEN05, false>, dim3(grid), dim3(kActThreads), 0, st, x, M, rows_idx, K, ld, ts_x, codes, sf));
+        if (wide) PQ_CUDA_OK(pq::launch_dependent(quant_nvfp4_kernel<PQ_SF_TCGEN05, true>, grid, block, 0, st, x, M, rows_idx, K, ld, ts_x, codes, sf));
+        else PQ_CUDA_OK(pq::launch_dependent(quant_nvfp4_kernel<PQ_SF_TCGEN05, false>, grid, block, 0, st, x, M, rows_idx, K, ld, ts_x, codes, sf));
     } else {
-        if (wide) PQ_CUDA_OK(pq::launch_dependent(quant_nvfp4_kernel<PQ_SF_LINEAR, true>, dim3(grid), dim3(kActThreads), 0, st, x, M, rows_idx, K, ld, ts_x, codes, sf));
-        else PQ_CUDA_OK(pq::launch_dependent(quant_nvfp4_kernel<PQ_SF_LINEAR, false>, dim3(grid), dim3(kActThreads), 0, st, x, M, rows_idx, K, ld, ts_x, codes, sf));
+        if (wide) PQ_CUDA_OK(pq::launch_dependent(quant_nvfp4_kernel<PQ_SF_LINEAR, true>, grid, block, 0, st, x, M, rows_idx, K, ld, ts_x, codes, sf));
+        else PQ_CUDA_OK(pq::launch_dependent(quant_nvfp4_kernel<PQ_SF_LINEAR, false>, grid, block, 0, st, x, M, rows_idx, K, ld, ts_x, codes, sf));
     }
     return pq_launch_status();
 }
@@ -327,7 +327,15 @@ extern "C" pq_status pq_quant_weight(const void *Wt, int64_t N, int64_t K, int64
     const uint16_t *w = static_cast<const uint16_t *>(Wt);
     unsigned int *amax_bits = static_cast<unsigned int *>(ws);
     PQ_CUDA_OK(cudaMemsetAsync(amax_bits, 0, sizeof(unsigned int), st));
-    amax_all_kernel<<<grid_for(N * (K / 8), 256, 8), 256, 0, st>>>(w, N, K, ld, amax_bits);
+    {
+        // column chunks x enough row strides to fill the GPU (8 blocks per SM)
+        const int64_t chunks = pq_ceil_div(K / 8, 32);
+        const int64_t want_y = pq_ceil_div(grid_for(N * (K / 8), 256, 8), chunks);
+        const int64_t max_y = pq_ceil_div(N, kTileRows);
+        const int64_t gy = want_y < max_y ? (want_y > 0 ? want_y : 1) : max_y;
+        amax_all_kernel<<<dim3(static_cast<unsigned>(chunks), static_cast<unsigned>(gy < kGridYMax ? gy : kGridYMax)),
+                          dim3(32, kTileRows), 0, st>>>(w, N, K, ld, amax_bits);
+    }
     weight_scale_kernel<<<1, 1, 0, st>>>(amax_bits, ts_w);
     if (!perm) return pq_quant_act_nvfp4(Wt, N, K, ld, ts_w, codes, sf, sf_layout, stream);
 
@@ -361,13 +369,14 @@ extern "C" pq_status pq_fakequant_int(const void *T, int64_t rows, int64_t K, in
     const float Qf = static_cast<float>((1 << (fmt.bits - 1)) - 1);
     const size_t smem = static_cast<size_t>(K) * 2;
     const int grid_g = static_cast<int>(rows < 148 * 8 ? rows : 148 * 8);
-    const int grid = grid_for(rows * (K / 8), kQuantThreads, 16);
+    PQ_REQUIRE(rows / kTileRows < static_cast<int64_t>(kGridYMax) * 65535, PQ_ERR_SHAPE);
+    const dim3 grid = tile_grid(pq_ceil_div(K / 8, 32), pq_ceil_div(rows, kTileRows));
 #define PQ_FQ_CASE(TEAM)                                                                              \
     if (perm) {                                                                                       \
         if (allow_smem(fakequant_int_gather_kernel<TEAM>, smem) != PQ_OK) return PQ_ERR_CUDA;         \
         fakequant_int_gather_kernel<TEAM><<<grid_g, kQuantThreads, smem, st>>>(t, rows, K, ld, perm, Qf, o, ldo); \
     } else {                                                                                          \
-        fakequant_int_kernel<TEAM><<<grid, kQuantThreads, 0, st>>>(t, rows, K, ld, Qf, o, ldo);        \
+        fakequant_int_kernel<TEAM><<<grid, dim3(32, kTileRows), 0, st>>>(t, rows, K, ld, Qf, o, ldo); \
     }
     switch (fmt.group) {
         case 16: PQ_FQ_CASE(2) break;
