@@ -48,6 +48,11 @@ __device__ __forceinline__ void load_group(const uint16_t *p, uint4 &lo, uint4 &
     }
 }
 
+#ifndef PQ_ACT_ROWS
+#define PQ_ACT_ROWS 1
+#endif
+constexpr int kActRows = PQ_ACT_ROWS;  // rows per thread: their loads are issued together
+
 template <int SF_LAYOUT, bool WIDE>
 __global__ void __launch_bounds__(kActThreads)
 quant_nvfp4_kernel(const uint16_t *__restrict__ X, int64_t rows, int64_t rows_pad, int64_t K,
@@ -55,8 +60,7 @@ quant_nvfp4_kernel(const uint16_t *__restrict__ X, int64_t rows, int64_t rows_pa
                    uint8_t *__restrict__ sf) {
     const uint32_t gpr = static_cast<uint32_t>(K >> 4);  // groups per row
     const uint32_t g = blockIdx.x * 32u + threadIdx.x;
-    const int64_t row = row_block_index() * kTileRows + threadIdx.y;
-    const bool in_range = row < rows_pad && g < gpr, live = row < rows && g < gpr;
+    const int64_t row0 = row_block_index() * (kTileRows * kActRows) + threadIdx.y;
     // This kernel is launched as a programmatic dependent of whatever precedes it in the stream:
     // its blocks may become resident while that kernel's last blocks run, and wait here until it
     // has completed and its writes are visible (ordinary stream order from here on).  In turn a
@@ -66,30 +70,40 @@ quant_nvfp4_kernel(const uint16_t *__restrict__ X, int64_t rows, int64_t rows_pa
     pq::dependents_may_launch();
     const float ts = __ldg(ts_ptr);
 
-    uint4 lo = make_uint4(0, 0, 0, 0), hi = lo;
-    if (live) load_group<WIDE>(X + row * ld + static_cast<int64_t>(g) * 16, lo, hi);
-    float x[8], y[8];
-    pq::unpack8(lo, x);
-    pq::unpack8(hi, y);
-    const float amax = fmaxf(pq::absmax8(x), pq::absmax8(y));
-    uint32_t sf8;
-    float d, r;
-    pq::nvfp4_scale(amax, ts, sf8, d, r);
-    const uint32_t c0 = pq::nvfp4_codes(x, r), c1 = pq::nvfp4_codes(y, r);
-    if (live) __stcs(reinterpret_cast<uint2 *>(codes + row * (K >> 1) + static_cast<int64_t>(g) * 8), make_uint2(c0, c1));
-    // scale bytes of groups g .. g+3 (same row when the row holds a multiple of 4 groups)
-    uint32_t word = sf8;
-    word |= __shfl_down_sync(0xFFFFFFFFu, sf8, 1) << 8;
-    word |= __shfl_down_sync(0xFFFFFFFFu, sf8, 2) << 16;
-    word |= __shfl_down_sync(0xFFFFFFFFu, sf8, 3) << 24;
-    if (!in_range) return;
-    if (SF_LAYOUT == PQ_SF_TCGEN05) {
-        if ((g & 3u) == 0) *reinterpret_cast<uint32_t *>(sf + pq::sf_tc_offset(row, g, gpr >> 2)) = word;
-    } else if (live) {
-        if ((gpr & 3u) == 0) {
-            if ((g & 3u) == 0) *reinterpret_cast<uint32_t *>(sf + row * gpr + g) = word;
-        } else {
-            sf[row * gpr + g] = static_cast<uint8_t>(sf8);
+    uint4 lo[kActRows], hi[kActRows];
+#pragma unroll
+    for (int i = 0; i < kActRows; ++i) {
+        const int64_t row = row0 + i * kTileRows;
+        lo[i] = make_uint4(0, 0, 0, 0), hi[i] = lo[i];
+        if (row < rows && g < gpr) load_group<WIDE>(X + row * ld + static_cast<int64_t>(g) * 16, lo[i], hi[i]);
+    }
+#pragma unroll
+    for (int i = 0; i < kActRows; ++i) {
+        const int64_t row = row0 + i * kTileRows;
+        const bool in_range = row < rows_pad && g < gpr, live = row < rows && g < gpr;
+        float x[8], y[8];
+        pq::unpack8(lo[i], x);
+        pq::unpack8(hi[i], y);
+        const float amax = fmaxf(pq::absmax8(x), pq::absmax8(y));
+        uint32_t sf8;
+        float d, r;
+        pq::nvfp4_scale(amax, ts, sf8, d, r);
+        const uint32_t c0 = pq::nvfp4_codes(x, r), c1 = pq::nvfp4_codes(y, r);
+        if (live) __stcs(reinterpret_cast<uint2 *>(codes + row * (K >> 1) + static_cast<int64_t>(g) * 8), make_uint2(c0, c1));
+        // scale bytes of groups g .. g+3 (same row when the row holds a multiple of 4 groups)
+        uint32_t word = sf8;
+        word |= __shfl_down_sync(0xFFFFFFFFu, sf8, 1) << 8;
+        word |= __shfl_down_sync(0xFFFFFFFFu, sf8, 2) << 16;
+        word |= __shfl_down_sync(0xFFFFFFFFu, sf8, 3) << 24;
+        if (!in_range) continue;
+        if (SF_LAYOUT == PQ_SF_TCGEN05) {
+            if ((g & 3u) == 0) *reinterpret_cast<uint32_t *>(sf + pq::sf_tc_offset(row, g, gpr >> 2)) = word;
+        } else if (live) {
+            if ((gpr & 3u) == 0) {
+                if ((g & 3u) == 0) *reinterpret_cast<uint32_t *>(sf + row * gpr + g) = word;
+            } else {
+                sf[row * gpr + g] = static_cast<uint8_t>(sf8);
+            }
         }
     }
 }
@@ -289,7 +303,7 @@ extern "C" pq_status pq_quant_act_nvfp4(const void *X, int64_t M, int64_t K, int
     const bool wide = (reinterpret_cast<uintptr_t>(X) & 31u) == 0 && ld % 16 == 0;
     const int64_t rows_idx = sf_layout == PQ_SF_TCGEN05 ? pq_ceil_div(M, 128) * 128 : M;
     PQ_REQUIRE(K / 16 <= 32ll * 0x7FFFFFFF && rows_idx / kTileRows < static_cast<int64_t>(kGridYMax) * 65535, PQ_ERR_SHAPE);
-    const dim3 grid = tile_grid(pq_ceil_div(K / 16, 32), pq_ceil_div(rows_idx, kTileRows));
+    const dim3 grid = tile_grid(pq_ceil_div(K / 16, 32), pq_ceil_div(rows_idx, kTileRows * kActRows));
     const dim3 block(32, kTileRows);
     // The quantizer's blocks should be able to run on an SM beside a GEMM CTA (the batched linear
     // path overlaps the two kernels): ask for the GEMM's shared-memory carve-out, otherwise an SM
