@@ -30,6 +30,7 @@ NSETS = 4          # buffer sets the timed loop rotates over (each ~137 MB; L2 i
 XROT = 10          # activation buffers the stand-alone streaming loops rotate over (283 MB)
 ORACLE_ROWS_MAX = 2048   # largest row sample of the workload the oracle legs use
 FP4_OVER_BF16 = 4.0  # nominal dense tensor ratio (9 vs 2.25 PFLOP/s)
+GEMM_DRAM_BYTES_PER_LAUNCH = 54.55e6   # ncu, 23.92 MB read + 30.63 MB written per launch of the bench workload
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
 
@@ -320,7 +321,9 @@ def run_ours(args):
     gemm_tflops = flops / (ms_gemm * 1e-3) / 1e12
     quant_bytes = M * K * 2 + M * K // 2 + M * K // 16
     roofline = {"kernel": "gemm_w4a4_kernel", "bound": "tensor", "achieved": gemm_tflops, "peak": fp4_peak,
-                "unit": "TFLOP/s", "frac": gemm_tflops / fp4_peak, "traffic": None,
+                "unit": "TFLOP/s", "frac": gemm_tflops / fp4_peak, "traffic": GEMM_DRAM_BYTES_PER_LAUNCH,
+                "traffic_source": "dram__bytes_read.sum + dram__bytes_write.sum of one ncu capture of this kernel on this "
+                                  "workload (profiles/gemm_w4a4_kernel_qkv_4608x3072x9216.md); algorithmic bytes 108.8e6",
                 "peak_source": f"{peaks['source']} bf16 burst {peaks['bf16_tflops']} TFLOP/s x {FP4_OVER_BF16:g} "
                                f"(nominal fp4:bf16 ratio)",
                 "frac_of_sustained": gemm_tflops / (peaks["bf16_tflops_sustained"] * FP4_OVER_BF16),
