@@ -709,13 +709,15 @@ pq_status gemm_launch(const uint8_t *xq, const uint8_t *sfx, const float *ts_x, 
     cfg.dynamicSmemBytes = kSmemBytes;
     cfg.stream = st;
     // Programmatic dependent launch: the kernel may start (barrier set-up, tensor-memory allocation,
-    // tensor-map prefetch) while the quantizer in front of it drains; it waits for that kernel's
-    // results with griddepcontrol.wait before touching global memory.
+    // tensor-map prefetch) while the kernel in front of it in the stream drains (the quantizer, or
+    // the previous GEMM of a chain of layers); it waits for that kernel to complete with
+    // griddepcontrol.wait before touching global memory, so stream order is what the caller sees.
     cudaLaunchAttribute attr;
     attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr.val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = &attr;
-    cfg.numAttrs = programmatic ? 1 : 0;
+    cfg.numAttrs = 1;
+    (void)programmatic;
     PQ_CUDA_OK(cudaLaunchKernelEx(&cfg, gemm_w4a4_kernel, map_a, map_b, map_y, p));
     return PQ_OK;
 }
