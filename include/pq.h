@@ -258,6 +258,21 @@ pq_status pq_linear_w4a4_host(const void *X_host, int64_t M, int64_t K, const fl
                               const uint8_t *sfw, const float *ts_w, int64_t N, void *Y_dev,
                               void *Y_host, void *ws, size_t ws_bytes, void *stream);
 
+/* pq_linear_w4a4_host for n independent batches: uploads, the runtime path and downloads run on
+ * three internal streams ordered by events, so the copies of neighbouring batches overlap each
+ * other (PCIe is full duplex) and the kernels.  Batch i uses staging buffers X_dev[i % n_sets] and
+ * Y_dev[i % n_sets]; one set of intermediates xq / sfx serves all batches (the kernels of different
+ * batches run in order).  Results are those of n calls of pq_linear_w4a4_host.
+ *   X_host, Y_host : HOST arrays of n HOST pointers (bf16 [M, K] / [M, N] contiguous, pinned).
+ *   X_dev, Y_dev   : HOST arrays of n_sets device staging buffers, 2 <= n_sets <= 8.
+ * Ordering and the internal streams as for pq_linear_w4a4_batched; the caller synchronises
+ * `stream` before reading the Y_host buffers. */
+pq_status pq_linear_w4a4_host_batched(int n, const void *const *X_host, int64_t M, int64_t K,
+                                      const float *ts_x, void *const *X_dev, void *const *Y_dev,
+                                      int n_sets, uint8_t *xq, uint8_t *sfx, const uint8_t *wq,
+                                      const uint8_t *sfw, const float *ts_w, int64_t N,
+                                      void *const *Y_host, void *ws, size_t ws_bytes, void *stream);
+
 /* Integer fake-quant of Eq. 1-2 (quantize, dequantize, round to bf16), optional gather.
  *   T : bf16 [rows, K], ld.  out : bf16 [rows, K], ldo.  perm : int32 [K] or NULL.
  *   fmt.kind must be 1; K % fmt.group == 0; K <= 16384 when perm != NULL. */

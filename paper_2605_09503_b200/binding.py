@@ -53,6 +53,8 @@ _SIGNATURES = {
                               _vp, _sz, _vp]),
     "pq_linear_w4a4_batched": (_int, [_int, _vp, _i64, _i64, _i64, _vp, _vp, _vp, _int, _vp, _vp, _vp, _i64, _vp, _i64,
                                       _vp, _sz, _vp]),
+    "pq_linear_w4a4_host_batched": (_int, [_int, _vp, _i64, _i64, _vp, _vp, _vp, _int, _vp, _vp, _vp, _vp, _vp, _i64, _vp,
+                                           _vp, _sz, _vp]),
     "pq_linear_w4a4_host": (_int, [_vp, _i64, _i64, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _i64, _vp, _vp,
                                    _vp, _sz, _vp]),
     "pq_fakequant_int": (_int, [_vp, _i64, _i64, _i64, pq_format, _vp, _vp, _i64, _vp]),
@@ -231,6 +233,25 @@ def pq_linear_w4a4_batched(Xs, ts_x, xqs, sfxs, wq, sfw, ts_w, Ys, ws):
     _check("pq_linear_w4a4_batched", lib().pq_linear_w4a4_batched(
         n, arr(Xs), M, K, Xs[0].stride(0), _p(ts_x), arr(xqs), arr(sfxs), n_sets, _p(wq), _p(sfw), _p(ts_w), N,
         arr(Ys), Ys[0].stride(0), w, wb, _stream()))
+
+
+def pq_linear_w4a4_host_batched(X_hosts, ts_x, X_devs, Y_devs, xq, sfx, wq, sfw, ts_w, Y_hosts, ws):
+    """n host batches in, n host batches out; uploads, kernels and downloads of neighbouring batches overlap."""
+    n, n_sets = len(X_hosts), len(X_devs)
+    assert len(Y_hosts) == n and len(Y_devs) == n_sets
+    M, K = X_hosts[0].shape
+    N = wq.shape[0]
+    for x, y in zip(X_hosts, Y_hosts):
+        assert not x.is_cuda and not y.is_cuda and x.is_contiguous() and y.is_contiguous()
+        assert x.dtype == torch.bfloat16 and y.dtype == torch.bfloat16 and x.shape == (M, K) and y.shape == (M, N)
+    for x, y in zip(X_devs, Y_devs):
+        _bf16(x)
+        assert x.shape == (M, K) and x.is_contiguous() and y.shape == (M, N) and y.is_contiguous() and y.is_cuda
+    arr = lambda ts: (C.c_void_p * len(ts))(*[t.data_ptr() for t in ts])
+    w, wb = _ws(ws)
+    _check("pq_linear_w4a4_host_batched", lib().pq_linear_w4a4_host_batched(
+        n, arr(X_hosts), M, K, _p(ts_x), arr(X_devs), arr(Y_devs), n_sets, _p(xq), _p(sfx), _p(wq), _p(sfw), _p(ts_w),
+        N, arr(Y_hosts), w, wb, _stream()))
 
 
 def pq_linear_w4a4_host(X_host, ts_x, X_dev, xq, sfx, wq, sfw, ts_w, Y_dev, Y_host, ws):

@@ -758,9 +758,9 @@ constexpr int kMaxSets = 8, kMaxPipeDevices = 64;
 // Two internal streams and the events that order them, created once per device (host objects,
 // no device memory).
 struct Pipe {
-    cudaStream_t q = nullptr, g = nullptr;
-    cudaEvent_t fork = nullptr, join_q = nullptr, join_g = nullptr;
-    cudaEvent_t q_done[kMaxSets] = {}, g_done[kMaxSets] = {};
+    cudaStream_t q = nullptr, g = nullptr, up = nullptr, down = nullptr;
+    cudaEvent_t fork = nullptr, join_q = nullptr, join_g = nullptr, join_up = nullptr, join_down = nullptr;
+    cudaEvent_t q_done[kMaxSets] = {}, g_done[kMaxSets] = {}, up_done[kMaxSets] = {}, down_done[kMaxSets] = {};
     bool ready = false;
 };
 
@@ -773,10 +773,13 @@ Pipe *pipe_for_current_device() {
     Pipe &p = pipes[dev];
     if (!p.ready) {
         bool ok = cudaStreamCreateWithFlags(&p.q, cudaStreamNonBlocking) == cudaSuccess &&
-                  cudaStreamCreateWithFlags(&p.g, cudaStreamNonBlocking) == cudaSuccess;
+                  cudaStreamCreateWithFlags(&p.g, cudaStreamNonBlocking) == cudaSuccess &&
+                  cudaStreamCreateWithFlags(&p.up, cudaStreamNonBlocking) == cudaSuccess &&
+                  cudaStreamCreateWithFlags(&p.down, cudaStreamNonBlocking) == cudaSuccess;
         auto make = [&](cudaEvent_t *e) { ok = ok && cudaEventCreateWithFlags(e, cudaEventDisableTiming) == cudaSuccess; };
-        make(&p.fork), make(&p.join_q), make(&p.join_g);
-        for (int i = 0; i < kMaxSets; ++i) make(&p.q_done[i]), make(&p.g_done[i]);
+        make(&p.fork), make(&p.join_q), make(&p.join_g), make(&p.join_up), make(&p.join_down);
+        for (int i = 0; i < kMaxSets; ++i)
+            make(&p.q_done[i]), make(&p.g_done[i]), make(&p.up_done[i]), make(&p.down_done[i]);
         if (!ok) {
             (void)cudaGetLastError();
             return nullptr;
@@ -827,6 +830,59 @@ extern "C" pq_status pq_linear_w4a4_batched(int n, const void *const *X, int64_t
                   cudaEventRecord(pipe->join_g, pipe->g) == cudaSuccess &&
                   cudaStreamWaitEvent(user, pipe->join_q, 0) == cudaSuccess &&
                   cudaStreamWaitEvent(user, pipe->join_g, 0) == cudaSuccess;
+    if (!joined) {
+        (void)cudaGetLastError();
+        return rc == PQ_OK ? PQ_ERR_CUDA : rc;
+    }
+    return rc;
+}
+
+extern "C" pq_status pq_linear_w4a4_host_batched(int n, const void *const *X_host, int64_t M, int64_t K,
+                                                 const float *ts_x, void *const *X_dev, void *const *Y_dev, int n_sets,
+                                                 uint8_t *xq, uint8_t *sfx, const uint8_t *wq, const uint8_t *sfw,
+                                                 const float *ts_w, int64_t N, void *const *Y_host, void *ws,
+                                                 size_t ws_bytes, void *stream) {
+    PQ_REQUIRE(X_host && X_dev && Y_dev && Y_host, PQ_ERR_NULL);
+    PQ_REQUIRE(n >= 1 && n_sets >= 2 && n_sets <= kMaxSets && M > 0 && K > 0 && N > 0, PQ_ERR_SHAPE);
+    for (int i = 0; i < n; ++i) PQ_REQUIRE(X_host[i] && Y_host[i], PQ_ERR_NULL);
+    for (int s = 0; s < n_sets; ++s) PQ_REQUIRE(X_dev[s] && Y_dev[s], PQ_ERR_NULL);
+    Pipe *pipe = pipe_for_current_device();
+    if (!pipe) return PQ_ERR_CUDA;
+    cudaStream_t user = static_cast<cudaStream_t>(stream), up = pipe->up, run = pipe->g, down = pipe->down;
+    const size_t x_bytes = static_cast<size_t>(M) * K * 2, y_bytes = static_cast<size_t>(M) * N * 2;
+    PQ_CUDA_OK(cudaEventRecord(pipe->fork, user));
+    PQ_CUDA_OK(cudaStreamWaitEvent(up, pipe->fork, 0));
+    PQ_CUDA_OK(cudaStreamWaitEvent(run, pipe->fork, 0));
+    PQ_CUDA_OK(cudaStreamWaitEvent(down, pipe->fork, 0));
+    pq_status rc = PQ_OK;
+    auto cuda_ok = [&](cudaError_t e) {
+        if (e != cudaSuccess && rc == PQ_OK) rc = PQ_ERR_CUDA;
+        return rc == PQ_OK;
+    };
+    for (int i = 0; i < n && rc == PQ_OK; ++i) {
+        const int s = i % n_sets;
+        // upload: the staging buffer is free once the quantizer of its previous batch has read it
+        if (i >= n_sets && !cuda_ok(cudaStreamWaitEvent(up, pipe->q_done[s], 0))) break;
+        if (!cuda_ok(cudaMemcpyAsync(X_dev[s], X_host[i], x_bytes, cudaMemcpyHostToDevice, up))) break;
+        if (!cuda_ok(cudaEventRecord(pipe->up_done[s], up))) break;
+        // compute: needs the upload, and the output buffer's previous download to have finished
+        if (!cuda_ok(cudaStreamWaitEvent(run, pipe->up_done[s], 0))) break;
+        if (i >= n_sets && !cuda_ok(cudaStreamWaitEvent(run, pipe->down_done[s], 0))) break;
+        rc = pq_quant_act_nvfp4(X_dev[s], M, K, K, ts_x, xq, sfx, PQ_SF_TCGEN05, run);
+        if (rc != PQ_OK || !cuda_ok(cudaEventRecord(pipe->q_done[s], run))) break;
+        rc = gemm_launch(xq, sfx, ts_x, wq, sfw, ts_w, M, N, K, Y_dev[s], N, ws, ws_bytes, run, true);
+        if (rc != PQ_OK || !cuda_ok(cudaEventRecord(pipe->g_done[s], run))) break;
+        // download
+        if (!cuda_ok(cudaStreamWaitEvent(down, pipe->g_done[s], 0))) break;
+        if (!cuda_ok(cudaMemcpyAsync(Y_host[i], Y_dev[s], y_bytes, cudaMemcpyDeviceToHost, down))) break;
+        if (!cuda_ok(cudaEventRecord(pipe->down_done[s], down))) break;
+    }
+    const bool joined = cudaEventRecord(pipe->join_up, up) == cudaSuccess &&
+                        cudaEventRecord(pipe->join_g, run) == cudaSuccess &&
+                        cudaEventRecord(pipe->join_down, down) == cudaSuccess &&
+                        cudaStreamWaitEvent(user, pipe->join_up, 0) == cudaSuccess &&
+                        cudaStreamWaitEvent(user, pipe->join_g, 0) == cudaSuccess &&
+                        cudaStreamWaitEvent(user, pipe->join_down, 0) == cudaSuccess;
     if (!joined) {
         (void)cudaGetLastError();
         return rc == PQ_OK ? PQ_ERR_CUDA : rc;

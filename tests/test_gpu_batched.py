@@ -83,3 +83,25 @@ def test_batched_rejects_bad_arguments():
     Ys = [torch.empty(M, N, dtype=torch.bfloat16, device="cuda") for _ in range(2)]
     with pytest.raises(B.PqError):
         B.pq_linear_w4a4_batched(Xs, ts_x, one, sf, wq, sfw, ts_w, Ys, ws)      # a single set of intermediates
+
+
+def test_host_batched_equals_one_by_one():
+    M, K, N, n = 384, 256, 320, 5
+    Xs, ts_x, wq, sfw, ts_w = _layer(M, K, N, n, seed=11)
+    ws = B.workspace(B.OP_GEMM, M, K, N)
+    xq = torch.empty(M, K // 2, dtype=torch.uint8, device="cuda")
+    sfx = torch.empty(B.sf_bytes(M, K, 1), dtype=torch.uint8, device="cuda")
+    ref = []
+    for x in Xs:
+        y = torch.empty(M, N, dtype=torch.bfloat16, device="cuda")
+        B.pq_linear_w4a4(x, ts_x, xq, sfx, wq, sfw, ts_w, y, ws)
+        ref.append(y.cpu())
+    xh = [x.cpu().pin_memory() for x in Xs]
+    yh = [torch.zeros(M, N, dtype=torch.bfloat16).pin_memory() for _ in range(n)]
+    xd = [torch.empty(M, K, dtype=torch.bfloat16, device="cuda") for _ in range(2)]
+    yd = [torch.empty(M, N, dtype=torch.bfloat16, device="cuda") for _ in range(2)]
+    B.pq_linear_w4a4_host_batched(xh, ts_x, xd, yd, xq, sfx, wq, sfw, ts_w, yh, ws)
+    torch.cuda.synchronize()
+    assert B.pq_device_status(ws) == B.PQ_OK
+    for y, r in zip(yh, ref):
+        assert torch.equal(y.view(torch.int16), r.view(torch.int16))
