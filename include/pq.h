@@ -273,6 +273,34 @@ pq_status pq_linear_w4a4_host_batched(int n, const void *const *X_host, int64_t 
                                       const uint8_t *sfw, const float *ts_w, int64_t N,
                                       void *const *Y_host, void *ws, size_t ws_bytes, void *stream);
 
+/* Machine probes (no counterpart in the paper: they measure the GPU, not the method).  The GEMM's tile
+ * shape is bounded by how many operand bytes an SM can take in from L2 per MMA cycle and by how fast
+ * it can write a finished tile; these two calls measure both rates so that the roofline argument can
+ * be re-checked on any machine.
+ *   pq_probe_sm_ingest: `ctas` CTAs (one per SM when ctas <= SM count) each stream iters x 32 KB from
+ *     the region [src, src + region_bytes) (device memory; keep it below the L2 size and touch it
+ *     once to measure L2 -> SM) into shared memory with bulk copies, 6 in flight.  cycles[0] = SM clock
+ *     cycles of the slowest CTA, so bytes per clock per SM = iters * 32768 / cycles[0].
+ *     region_bytes: a multiple of 32768, >= 65536.  status: device int, PQ_OK or PQ_ERR_TIMEOUT.
+ *     sm_select: 0 = every CTA works; 1 = only CTAs that landed on an SM with an even id (one SM of
+ *     each pair of neighbouring SMs); 2 = only CTAs on SMs whose id / 2 is even (both SMs of every
+ *     other pair): with ctas = SM count, 1 and 2 keep half of the SMs busy in two different patterns,
+ *     which tells a per-SM-pair limit from a global one.
+ *   pq_probe_sm_store: `ctas` CTAs of four warps each write iters x 2048 bytes (512 contiguous bytes
+ *     per warp instruction) to disjoint parts of dst (>= ctas * iters * 2048 bytes).  cycles[0] as above.
+ * Both are asynchronous on `stream`; cycles / status are device words the calls reset first. */
+pq_status pq_probe_sm_ingest(const void *src, size_t region_bytes, int ctas, int iters, int sm_select,
+                             unsigned long long *cycles, int *status, void *stream);
+pq_status pq_probe_sm_store(void *dst, size_t dst_bytes, int ctas, int iters,
+                            unsigned long long *cycles, void *stream);
+/*   pq_probe_sm_forward: CTA pairs (clusters of two, ctas even); both CTAs stream iters x 32 KB from
+ *     L2 as above (4 copies in flight) while, if fwd_iters > 0, the first CTA of each pair also pushes
+ *     fwd_iters x 32 KB of its own shared memory into the second one's (2 in flight).  cycles[0] =
+ *     slowest L2 stream, cycles[1] = slowest forwarding loop: comparing cycles[0] with and without
+ *     forwarding tells whether shared-to-shared copies inside a cluster use the path from L2. */
+pq_status pq_probe_sm_forward(const void *src, size_t region_bytes, int ctas, int iters, int fwd_iters,
+                              unsigned long long *cycles, int *status, void *stream);
+
 /* Integer fake-quant of Eq. 1-2 (quantize, dequantize, round to bf16), optional gather.
  *   T : bf16 [rows, K], ld.  out : bf16 [rows, K], ldo.  perm : int32 [K] or NULL.
  *   fmt.kind must be 1; K % fmt.group == 0; K <= 16384 when perm != NULL. */
