@@ -58,3 +58,39 @@ def test_timing_reduction_and_sharding_across_two_ranks():
         assert worst == 15.0                         # max over ranks, seen by both
         assert rows == 4608
         assert abs(agg - 2 * 100.0 / 15e-3) < 1e-6
+
+
+def _calib_worker(rank, world, port, out):
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK=str(rank), WORLD_SIZE=str(world))
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    try:
+        g = torch.Generator().manual_seed(100 + rank)
+        # partials built so that the order of the additions shows in the last bits
+        sumsq = torch.rand(64, generator=g, dtype=torch.float64) * (1e12 if rank == 0 else 1e-3)
+        amax = torch.rand(64, generator=g, dtype=torch.float32) * (rank + 1)
+        err = torch.rand(3, 8, generator=g, dtype=torch.float64) * 10.0 ** (3 * rank)
+        S, A, rows, (E,) = sharding.combine_calibration(sumsq, amax, 1000 + rank, [err])
+        out.put((rank, sumsq, amax, err, S, A, rows, E))
+    finally:
+        dist.destroy_process_group()
+
+
+def test_calibration_partials_combine_in_rank_order():
+    world = 3
+    ctx = mp.get_context("spawn")
+    out = ctx.Queue()
+    port = _free_port()
+    procs = [ctx.Process(target=_calib_worker, args=(r, world, port, out)) for r in range(world)]
+    for p in procs:
+        p.start()
+    got = sorted((out.get(timeout=120) for _ in procs), key=lambda t: t[0])
+    for p in procs:
+        p.join(timeout=60)
+        assert p.exitcode == 0
+    S_want = (got[0][1] + got[1][1]) + got[2][1]                 # rank order, written out
+    E_want = (got[0][3] + got[1][3]) + got[2][3]
+    A_want = torch.maximum(torch.maximum(got[0][2], got[1][2]), got[2][2])
+    for _, _, _, _, S, A, rows, E in got:
+        assert torch.equal(S, S_want) and torch.equal(E, E_want) and torch.equal(A, A_want)
+        assert rows == 1000 + 1001 + 1002
+    assert not torch.equal(S_want, got[0][1] + (got[1][1] + got[2][1]))   # the case does depend on the order
