@@ -16,6 +16,9 @@
  *     (group absmax / 6 expressed in units of the tensor scale), one fp32 tensor scale.
  *   - Channel second moments (Assumption 3.1, Sec. 3.3), the joint criterion (Eq. 9), the
  *     descending sort (Prop. 3.2), the calibration error (Eq. 3) and the acceptance rule (Eq. 10).
+ *   - The producer of App. C (RMSNorm or adaptive LayerNorm with the channel reordering absorbed)
+ *     with the NVFP4 quantizer attached: row statistics in fp32 over the original channel order,
+ *     summed in the fixed 32-lane order stated at lane_order_sum.
  *
  * Pins: see tests/test_oracle_*.py.  Every function here is pinned by hand-computed values,
  * closed forms, brute force on tiny inputs or an independent library routine, except the
@@ -361,6 +364,77 @@ int pqo_quant_nvfp4(const uint16_t *T, int64_t rows, int64_t K, int64_t ld, cons
         }
     }
     return 0;
+}
+
+/* ------------------------------------------------------------------ fused norm + reorder + quantize */
+
+/* Sum over a row in the order a 32-lane row walk gives: element i belongs to lane (i / 8) % 32,
+ * each lane adds its elements in ascending i, the 32 lane partials are then combined by a
+ * butterfly (strides 16, 8, 4, 2, 1; every lane ends with the same value).
+ * mode 0: sum of v[i];  mode 1: sum of v[i]^2 by fused multiply-add. */
+static float lane_order_sum(const float *v, int64_t K, int mode) {
+    float p[32], q[32];
+    for (int l = 0; l < 32; ++l) p[l] = 0.0f;
+    for (int64_t i = 0; i < K; ++i) {
+        int l = (int)((i / 8) % 32);
+        p[l] = mode ? fmaf(v[i], v[i], p[l]) : p[l] + v[i];
+    }
+    for (int m = 16; m >= 1; m >>= 1) {
+        for (int l = 0; l < 32; ++l) q[l] = p[l] + p[l ^ m];
+        for (int l = 0; l < 32; ++l) p[l] = q[l];
+    }
+    return p[0];
+}
+
+/* Normalization with the channel reordering and the NVFP4 quantizer behind it (the absorbed
+ * permutation of App. C, with the quantizer of Eq. 8 attached): per row x of H
+ *   kind 0 (RMSNorm):            y_i = (x_i * inv) * a_i,                   inv = 1 / sqrt(mean(x^2) + eps)
+ *   kind 1 (adaptive LayerNorm): y_i = fma((x_i - mu) * inv, 1 + a_i, b_i), inv = 1 / sqrt(mean((x - mu)^2) + eps)
+ * (a = weight or modulation scale, b = modulation shift; statistics over the ORIGINAL channel order,
+ * so they do not depend on the permutation), then out_j = y_{perm[j]} and the NVFP4 groups of out.
+ * y_bf16 (optional) receives bf16(out), the tensor the unfused kernel of App. C would write.
+ * All arithmetic fp32, sums in lane order (lane_order_sum). */
+int pqo_norm_quant_nvfp4(const uint16_t *H, int64_t rows, int64_t K, int64_t ld, int kind, const float *a,
+                         const float *b, float eps, const int32_t *perm, float ts, uint8_t *codes,
+                         uint8_t *sf, uint16_t *y_bf16) {
+    if (!H || !a || !codes || !sf || rows <= 0 || K <= 0 || K % 16 != 0 || ld < K) return 1;
+    if (kind != 0 && kind != 1) return 1;
+    if (kind == 1 && !b) return 1;
+    int fail = 0;
+#pragma omp parallel for schedule(static)
+    for (int64_t t = 0; t < rows; ++t) {
+        float *x = (float *)malloc(sizeof(float) * (size_t)K * 2);
+        if (!x) {
+            fail = 1;
+            continue;
+        }
+        float *y = x + K;
+        for (int64_t i = 0; i < K; ++i) x[i] = pqo_bf16_to_f32(H[t * ld + i]);
+        if (kind == 0) {
+            float ms = lane_order_sum(x, K, 1) / (float)K;
+            float inv = 1.0f / sqrtf(ms + eps);
+            for (int64_t i = 0; i < K; ++i) y[i] = (x[i] * inv) * a[i];
+        } else {
+            float mu = lane_order_sum(x, K, 0) / (float)K;
+            for (int64_t i = 0; i < K; ++i) y[i] = x[i] - mu;      /* centred values, reused below */
+            float var = lane_order_sum(y, K, 1) / (float)K;
+            float inv = 1.0f / sqrtf(var + eps);
+            for (int64_t i = 0; i < K; ++i) y[i] = fmaf(y[i] * inv, 1.0f + a[i], b[i]);
+        }
+        for (int64_t k = 0; k < K / 16; ++k) {
+            float g[16], d;
+            uint8_t code[16], sf8;
+            for (int j = 0; j < 16; ++j) g[j] = y[perm ? perm[k * 16 + j] : k * 16 + j];
+            nvfp4_group(g, 16, ts, &sf8, &d, code);
+            sf[t * (K / 16) + k] = sf8;
+            for (int j = 0; j < 16; j += 2)
+                codes[t * (K / 2) + (k * 16 + j) / 2] = (uint8_t)(code[j] | (code[j + 1] << 4));
+            if (y_bf16)
+                for (int j = 0; j < 16; ++j) y_bf16[t * K + k * 16 + j] = pqo_f32_to_bf16(g[j]);
+        }
+        free(x);
+    }
+    return fail;
 }
 
 /* Decode one NVFP4 tensor back to fp32: value * (scale * ts), both products in fp32. */

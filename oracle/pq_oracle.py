@@ -49,6 +49,7 @@ def _declare(L):
     L.pqo_error_weight.argtypes = [_P, _i64]
     L.pqo_quant_nvfp4.argtypes = [_P, _i64, _i64, _i64, _P, C.c_float, _P, _P]
     L.pqo_dequant_nvfp4.argtypes = [_P, _P, C.c_float, _i64, _i64, _P]
+    L.pqo_norm_quant_nvfp4.argtypes = [_P, _i64, _i64, _i64, C.c_int, _P, _P, C.c_float, _P, C.c_float, _P, _P, _P]
     L.pqo_fakequant_int.argtypes = [_P, _i64, _i64, _i64, C.c_int, C.c_int, _P, _P, _i64]
     L.pqo_gemm_ref_one.restype = C.c_double
     L.pqo_gemm_ref_one.argtypes = [_P, _P, C.c_float, _P, _P, C.c_float, _i64, _i64, _i64]
@@ -194,6 +195,22 @@ def quant_nvfp4(T, ts, perm=None):
     _check(lib().pqo_quant_nvfp4(_ptr(T), rows, K, K, _ptr(perm), C.c_float(ts), _ptr(codes),
                                  _ptr(sf)), "quant_nvfp4")
     return codes, sf
+
+
+def norm_quant_nvfp4(H, kind, a, b, eps, ts, perm=None):
+    """Fused normalization (0 = RMSNorm with weight a, 1 = adaptive LayerNorm with scale a, shift b),
+    reordering and NVFP4 quantization -> (codes, scale bytes [rows, K/16], bf16 bits of the reordered output)."""
+    H = _bf16(H)
+    rows, K = H.shape
+    perm = _perm(perm, K)
+    a = np.ascontiguousarray(a, dtype=np.float32)
+    b = None if b is None else np.ascontiguousarray(b, dtype=np.float32)
+    codes = np.empty((rows, K // 2), dtype=np.uint8)
+    sf = np.empty((rows, K // 16), dtype=np.uint8)
+    y = np.empty((rows, K), dtype=np.uint16)
+    _check(lib().pqo_norm_quant_nvfp4(_ptr(H), rows, K, K, kind, _ptr(a), _ptr(b), C.c_float(eps), _ptr(perm),
+                                      C.c_float(ts), _ptr(codes), _ptr(sf), _ptr(y)), "norm_quant_nvfp4")
+    return codes, sf, y
 
 
 def dequant_nvfp4(codes, sf, ts):
