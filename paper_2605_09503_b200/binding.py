@@ -59,6 +59,8 @@ _SIGNATURES = {
                                    _vp, _sz, _vp]),
     "pq_fakequant_int": (_int, [_vp, _i64, _i64, _i64, pq_format, _vp, _vp, _i64, _vp]),
     "pq_sf_to_linear": (_int, [_vp, _i64, _i64, _vp, _vp]),
+    "pq_norm_quant_nvfp4": (_int, [_vp, _i64, _i64, _i64, _int, _vp, _vp, C.c_float, _vp, _vp, _vp, _vp, _int, _vp,
+                                   _vp]),
     "pq_device_status": (_int, [_vp, _vp]),
     "pq_probe_sm_ingest": (_int, [_vp, _sz, _int, _int, _int, _vp, _vp, _vp]),
     "pq_probe_sm_store": (_int, [_vp, _sz, _int, _int, _vp, _vp]),
@@ -284,6 +286,19 @@ def pq_fakequant_int(T, fmt, perm, out):
 
 def pq_sf_to_linear(sf_tc, rows, K, sf_linear):
     _check("pq_sf_to_linear", lib().pq_sf_to_linear(_p(sf_tc), rows, K, _p(sf_linear), _stream()))
+
+
+NORM_RMS, NORM_ADALN = 0, 1
+
+
+def pq_norm_quant_nvfp4(H, kind, a, b, eps, perm, ts_x, codes, sf, sf_layout, y_out=None):
+    _bf16(H)
+    M, K = H.shape
+    assert a.dtype == torch.float32 and a.numel() == K and (b is None or (b.dtype == torch.float32 and b.numel() == K))
+    assert perm is None or (perm.dtype == torch.int32 and perm.numel() == K)
+    assert y_out is None or (y_out.dtype == torch.bfloat16 and y_out.shape == (M, K) and y_out.is_contiguous())
+    _check("pq_norm_quant_nvfp4", lib().pq_norm_quant_nvfp4(_p(H), M, K, H.stride(0), kind, _p(a), _p(b), eps, _p(perm),
+                                                            _p(ts_x), _p(codes), _p(sf), sf_layout, _p(y_out), _stream()))
 
 
 def pq_probe_sm_ingest(src, ctas, iters, sm_select=0):
