@@ -429,6 +429,15 @@ def run_ours(args):
                   rows * K * 4)
             del fq, xq_b, sfx_b
         del big
+        # fused producer: adaptive LayerNorm / RMSNorm + reordering + quantizer (reads 2 B, writes 0.5625 B per element)
+        av = 0.2 * torch.randn(K, device=dev)
+        bv = torch.randn(K, device=dev)
+        order = cal.perms[5].contiguous()
+        for kind, name in ((B.NORM_ADALN, "norm_quant_adaln"), (B.NORM_RMS, "norm_quant_rms")):
+            stage(name, graph_loop(torch, lambda i: B.pq_norm_quant_nvfp4(xs[i % XROT], kind, av, bv, 1e-6, order, cal.ts_x,
+                                                                          xq_rot[i % XROT], sfx_rot[i % XROT],
+                                                                          B.PQ_SF_TCGEN05), it),
+                  quant_bytes, bound="L1 / shared memory (gather through the permutation)")
         ws_err = B.workspace(B.OP_GROUP_ERROR, M, K, 0, 6)
         e6 = torch.zeros(6, K // 16, dtype=torch.float64, device=dev)
         ms = graph_loop(torch, lambda i: B.pq_group_error(xs[i % XROT], pipeline.NVFP4, cal.ts_x, cal.perms, e6, ws_err),
