@@ -23,7 +23,7 @@
  * Pins: see tests/test_oracle_*.py.  Every function here is pinned by hand-computed values,
  * closed forms, brute force on tiny inputs or an independent library routine, except the
  * behaviour of the whole pipeline on real-model activations ("parity unpinned": no weights,
- * calibration data or authors' code exist in this build; only synthetic stand-ins).
+ * calibration data or authors' code are available here; only synthetic stand-ins).
  */
 #include <math.h>
 #include <stdint.h>
@@ -387,12 +387,14 @@ static float lane_order_sum(const float *v, int64_t K, int mode) {
 }
 
 /* Normalization with the channel reordering and the NVFP4 quantizer behind it (the absorbed
- * permutation of App. C, with the quantizer of Eq. 8 attached): per row x of H
- *   kind 0 (RMSNorm):            y_i = (x_i * inv) * a_i,                   inv = 1 / sqrt(mean(x^2) + eps)
- *   kind 1 (adaptive LayerNorm): y_i = fma((x_i - mu) * inv, 1 + a_i, b_i), inv = 1 / sqrt(mean((x - mu)^2) + eps)
- * (a = weight or modulation scale, b = modulation shift; statistics over the ORIGINAL channel order,
- * so they do not depend on the permutation), then out_j = y_{perm[j]} and the NVFP4 groups of out.
- * y_bf16 (optional) receives bf16(out), the tensor the unfused kernel of App. C would write.
+ * permutation of App. C, with the quantizer of Eq. 8 attached): per row x of H and output position j
+ * reading channel c = perm[j]
+ *   kind 0 (RMSNorm):            out_j = (x_c * inv) * a_j,                   inv = 1 / sqrt(mean(x^2) + eps)
+ *   kind 1 (adaptive LayerNorm): out_j = fma((x_c - mu) * inv, 1 + a_j, b_j), inv = 1 / sqrt(mean((x - mu)^2) + eps)
+ * a (weight or modulation scale) and b (modulation shift) are indexed by OUTPUT position: they
+ * arrive reordered, (1 + Ps) and Pb of App. C.  The statistics run over the ORIGINAL channel order,
+ * so they do not depend on the permutation.  Then the NVFP4 groups of out.  y_bf16 (optional)
+ * receives bf16(out), the tensor the unfused kernel of App. C would write.
  * All arithmetic fp32, sums in lane order (lane_order_sum). */
 int pqo_norm_quant_nvfp4(const uint16_t *H, int64_t rows, int64_t K, int64_t ld, int kind, const float *a,
                          const float *b, float eps, const int32_t *perm, float ts, uint8_t *codes,
@@ -409,22 +411,24 @@ int pqo_norm_quant_nvfp4(const uint16_t *H, int64_t rows, int64_t K, int64_t ld,
             continue;
         }
         float *y = x + K;
+        float mu = 0.0f, inv;
         for (int64_t i = 0; i < K; ++i) x[i] = pqo_bf16_to_f32(H[t * ld + i]);
         if (kind == 0) {
             float ms = lane_order_sum(x, K, 1) / (float)K;
-            float inv = 1.0f / sqrtf(ms + eps);
-            for (int64_t i = 0; i < K; ++i) y[i] = (x[i] * inv) * a[i];
+            inv = 1.0f / sqrtf(ms + eps);
         } else {
-            float mu = lane_order_sum(x, K, 0) / (float)K;
-            for (int64_t i = 0; i < K; ++i) y[i] = x[i] - mu;      /* centred values, reused below */
+            mu = lane_order_sum(x, K, 0) / (float)K;
+            for (int64_t i = 0; i < K; ++i) y[i] = x[i] - mu;
             float var = lane_order_sum(y, K, 1) / (float)K;
-            float inv = 1.0f / sqrtf(var + eps);
-            for (int64_t i = 0; i < K; ++i) y[i] = fmaf(y[i] * inv, 1.0f + a[i], b[i]);
+            inv = 1.0f / sqrtf(var + eps);
         }
         for (int64_t k = 0; k < K / 16; ++k) {
             float g[16], d;
             uint8_t code[16], sf8;
-            for (int j = 0; j < 16; ++j) g[j] = y[perm ? perm[k * 16 + j] : k * 16 + j];
+            for (int j = 0; j < 16; ++j) {
+                int64_t pos = k * 16 + j, c = perm ? perm[pos] : pos;
+                g[j] = (kind == 0) ? (x[c] * inv) * a[pos] : fmaf((x[c] - mu) * inv, 1.0f + a[pos], b[pos]);
+            }
             nvfp4_group(g, 16, ts, &sf8, &d, code);
             sf[t * (K / 16) + k] = sf8;
             for (int j = 0; j < 16; j += 2)

@@ -198,8 +198,9 @@ def quant_nvfp4(T, ts, perm=None):
 
 
 def norm_quant_nvfp4(H, kind, a, b, eps, ts, perm=None):
-    """Fused normalization (0 = RMSNorm with weight a, 1 = adaptive LayerNorm with scale a, shift b),
-    reordering and NVFP4 quantization -> (codes, scale bytes [rows, K/16], bf16 bits of the reordered output)."""
+    """Fused normalization (0 = RMSNorm with weight a, 1 = adaptive LayerNorm with scale a, shift b; a and b
+    indexed by output position), reordering and NVFP4 quantization
+    -> (codes, scale bytes [rows, K/16], bf16 bits of the reordered output)."""
     H = _bf16(H)
     rows, K = H.shape
     perm = _perm(perm, K)

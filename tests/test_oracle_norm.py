@@ -69,8 +69,15 @@ def test_permutation_is_a_gather_of_the_unpermuted_result():
         c0, s0, y0 = O.norm_quant_nvfp4(xb, kind, a, b, 1e-5, 0.02)
         ci, si, yi = O.norm_quant_nvfp4(xb, kind, a, b, 1e-5, 0.02, perm=np.arange(K, dtype=np.int32))
         assert np.array_equal(c0, ci) and np.array_equal(s0, si) and np.array_equal(y0, yi)     # identity order
-        cp, sp, yp = O.norm_quant_nvfp4(xb, kind, a, b, 1e-5, 0.02, perm=perm)
+        # the parameters travel with their channels (they are indexed by output position)
+        cp, sp, yp = O.norm_quant_nvfp4(xb, kind, a[perm], b[perm], 1e-5, 0.02, perm=perm)
         assert np.array_equal(yp, y0[:, perm])               # same statistics, channels read through the order
+        # and parameters left in place act on whatever channel lands at their position
+        cq, sq, yq = O.norm_quant_nvfp4(xb, kind, np.ones(K, np.float32) if kind == 0 else np.zeros(K, np.float32),
+                                        np.zeros(K, np.float32), 1e-5, 0.02, perm=perm)
+        c1, s1, y1 = O.norm_quant_nvfp4(xb, kind, np.ones(K, np.float32) if kind == 0 else np.zeros(K, np.float32),
+                                        np.zeros(K, np.float32), 1e-5, 0.02)
+        assert np.array_equal(yq, y1[:, perm])
 
 
 def test_lane_order_of_the_row_sums():
