@@ -275,15 +275,16 @@ pq_status pq_linear_w4a4_host_batched(int n, const void *const *X_host, int64_t 
 
 /* The producer in front of a quantized linear layer, fused (App. C: the channel reordering absorbed
  * into the normalization kernel; here the NVFP4 quantizer of Eq. 8 is attached as well, so the
- * normalized activations are never written in bf16).  Per token row x of H, in fp32:
- *   PQ_NORM_RMS  : y_i = (x_i * inv) * a_i,                    inv = 1 / sqrt(mean_i(x_i^2) + eps)
- *   PQ_NORM_ADALN: y_i = fma((x_i - mu) * inv, 1 + a_i, b_i),  inv = 1 / sqrt(mean_i((x_i - mu)^2) + eps)
- * (a = RMSNorm weight or modulation scale, b = modulation shift, one vector per call; IEEE division
- * and square root).  The row sums run over the ORIGINAL channel order (so they do not depend on the
- * permutation): element i is added by lane (i / 8) % 32 in ascending i, the 32 lane sums meet in a
- * butterfly of strides 16, 8, 4, 2, 1.  Then out_j = y_{perm[j]} (perm == NULL: identity) is
- * quantized in groups of 16 exactly as pq_quant_act_nvfp4 quantizes a bf16 tensor holding out,
- * except that out keeps its fp32 precision.
+ * normalized activations are never written in bf16).  Per token row x of H and output position j
+ * reading channel c = perm[j] (perm == NULL: c = j), in fp32:
+ *   PQ_NORM_RMS  : out_j = (x_c * inv) * a_j,                    inv = 1 / sqrt(mean_i(x_i^2) + eps)
+ *   PQ_NORM_ADALN: out_j = fma((x_c - mu) * inv, 1 + a_j, b_j),  inv = 1 / sqrt(mean_i((x_i - mu)^2) + eps)
+ * a (RMSNorm weight or modulation scale) and b (modulation shift) are indexed by OUTPUT position: they
+ * arrive reordered, the (1 + Ps) and Pb of App. C; one vector each per call; IEEE division and square
+ * root.  The row sums run over the ORIGINAL channel order (so they do not depend on the permutation):
+ * element i is added by lane (i / 8) % 32 in ascending i, the 32 lane sums meet in a butterfly of strides
+ * 16, 8, 4, 2, 1.  out is quantized in groups of 16 exactly as pq_quant_act_nvfp4 quantizes a bf16
+ * tensor holding out, except that out keeps its fp32 precision.
  *   H : bf16 [M, K], ld.  K % 16 == 0 (K % 64 == 0 for PQ_SF_TCGEN05), K <= 32768.
  *   a, b : device fp32 [K], 16-byte aligned (b may be NULL for PQ_NORM_RMS).  perm : int32 [K] or NULL.
  *   codes, sf : as pq_quant_act_nvfp4.  y_out : bf16 [M, K] contiguous or NULL; receives bf16(out),

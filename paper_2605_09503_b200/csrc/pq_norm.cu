@@ -4,11 +4,14 @@
 //
 // One warp per token row.  The row is read once with coalesced 16-byte loads (lane l owns the
 // octets l, l + 32, ...: the summation order of the row statistics is this walk followed by a
-// butterfly over the lanes, and does not depend on the permutation), kept in shared memory in
-// fp32, normalized and modulated in place; then each lane takes 16-channel groups of the OUTPUT
-// order, gathers their values from shared memory through the permutation and quantizes them like
-// the stand-alone quantizer (8-byte code store, scale bytes of four neighbouring groups merged into
-// one 32-bit store).  Optionally the reordered bf16 tensor of the unfused kernel is written too.
+// butterfly over the lanes, and does not depend on the permutation) and kept in shared memory as
+// bf16; then each lane takes four consecutive positions of the OUTPUT order (a quarter of a group),
+// gathers their channels from shared memory through the permutation, normalizes them with the
+// scale / shift of the output positions (the parameters arrive reordered: one contiguous 16-byte
+// load per lane, like the indices) and quantizes them like the stand-alone quantizer (the four
+// lanes of a group share the absmax by shuffles; 2-byte code stores, coalesced; scale bytes of four
+// neighbouring groups merged into one 32-bit store).  The normalized values exist only in registers, in fp32.  Optionally the
+// reordered bf16 tensor of the unfused kernel is written too.
 #include "pq_common.cuh"
 
 namespace {
@@ -22,183 +25,27 @@ __device__ __forceinline__ float lane_butterfly(float p) {
     return p;
 }
 
-// Quantize the 16 values (x, y) of output group g of `row` and store codes, scale byte (merged over
-// four neighbouring lanes) and, optionally, the bf16 values.  Called by whole warps.
-template <int SF_LAYOUT>
-__device__ __forceinline__ void quantize_and_store(const float (&x)[8], const float (&y)[8], int64_t row, int g, int gpr,
-                                                   int K, bool live, bool have, float ts, uint8_t *__restrict__ codes,
-                                                   uint8_t *__restrict__ sf, uint16_t *__restrict__ y_out) {
-        const float amax = fmaxf(pq::absmax8(x), pq::absmax8(y));
-        uint32_t sf8;
-        float d, r;
-        pq::nvfp4_scale(amax, ts, sf8, d, r);
-        const uint32_t c0 = pq::nvfp4_codes(x, r), c1 = pq::nvfp4_codes(y, r);
-        if (live && have) {
-            __stcs(reinterpret_cast<uint2 *>(codes + row * (K >> 1) + g * 8), make_uint2(c0, c1));
-            if (y_out) {
-                uint32_t w[8];
-#pragma unroll
-                for (int e = 0; e < 4; ++e) {
-                    w[e] = __bfloat16_as_ushort(__float2bfloat16_rn(x[2 * e])) |
-                           (static_cast<uint32_t>(__bfloat16_as_ushort(__float2bfloat16_rn(x[2 * e + 1]))) << 16);
-                    w[4 + e] = __bfloat16_as_ushort(__float2bfloat16_rn(y[2 * e])) |
-                               (static_cast<uint32_t>(__bfloat16_as_ushort(__float2bfloat16_rn(y[2 * e + 1]))) << 16);
-                }
-                uint4 *dst = reinterpret_cast<uint4 *>(y_out + row * K + g * 16);
-                dst[0] = make_uint4(w[0], w[1], w[2], w[3]);
-                dst[1] = make_uint4(w[4], w[5], w[6], w[7]);
-            }
-        }
-        // scale bytes of groups g .. g+3 (padding rows write zeros)
-        uint32_t word = sf8;
-        word |= __shfl_down_sync(0xFFFFFFFFu, sf8, 1) << 8;
-        word |= __shfl_down_sync(0xFFFFFFFFu, sf8, 2) << 16;
-        word |= __shfl_down_sync(0xFFFFFFFFu, sf8, 3) << 24;
-        if (!have) return;
-        if (SF_LAYOUT == PQ_SF_TCGEN05) {
-            if ((g & 3) == 0) *reinterpret_cast<uint32_t *>(sf + pq::sf_tc_offset(row, g, gpr >> 2)) = word;
-        } else if (live) {
-            if ((gpr & 3) == 0) {
-                if ((g & 3) == 0) *reinterpret_cast<uint32_t *>(sf + row * gpr + g) = word;
-            } else {
-                sf[row * gpr + g] = static_cast<uint8_t>(sf8);
-            }
-        }
-}
-
-// Shared-memory layout of a row of fp32 values: the two 16-byte halves of octet o live at float4
-// index o and octs + o, so that a warp's 16-byte accesses (lane = octet) are contiguous and free of
-// bank conflicts.  Channel c = 8 o + e sits at float index 4 ((e >> 2) octs + o) + (e & 3).
-__device__ __forceinline__ int swz(int c, int octs) { return (((c >> 2) & 1) * octs + (c >> 3)) * 4 + (c & 3); }
-
-// Rows of up to 8 * 32 * REG_OCTS channels: the lane keeps its octets as packed bf16 in registers,
-// so the statistics and the scaling read no memory; only the finished fp32 row goes to shared
-// memory, for the gather.
-template <int KIND, int SF_LAYOUT, int REG_OCTS>
-__global__ void __launch_bounds__(32 * kMaxRowsPerBlock)
-norm_quant_reg_kernel(const uint16_t *__restrict__ H, int64_t rows, int64_t rows_pad, int K, int64_t ld,
-                      const float *__restrict__ a, const float *__restrict__ b, float eps,
-                      const int32_t *__restrict__ perm, const float *__restrict__ ts_ptr,
-                      uint8_t *__restrict__ codes, uint8_t *__restrict__ sf, uint16_t *__restrict__ y_out) {
-    extern __shared__ __align__(16) float row_s[];  // [warps][K], swizzled
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int64_t row = static_cast<int64_t>(blockIdx.x) * (blockDim.x >> 5) + warp;
-    if (row >= rows_pad) return;  // whole warps only
-    const bool live = row < rows;
-    float *ys = row_s + static_cast<size_t>(warp) * K;
-    const int octs = K >> 3, gpr = K >> 4;
-    const float ts = __ldg(ts_ptr);
-
-    if (live) {
-        const uint16_t *src = H + row * ld;
-        uint4 v[REG_OCTS];
-#pragma unroll
-        for (int u = 0; u < REG_OCTS; ++u) {
-            const int o = lane + 32 * u;
-            v[u] = o < octs ? __ldcs(reinterpret_cast<const uint4 *>(src + o * 8)) : make_uint4(0, 0, 0, 0);
-        }
-        float p = 0.0f;
-#pragma unroll
-        for (int u = 0; u < REG_OCTS; ++u) {
-            if (lane + 32 * u < octs) {
-                float x[8];
-                pq::unpack8(v[u], x);
-#pragma unroll
-                for (int e = 0; e < 8; ++e) p = KIND == 0 ? __fmaf_rn(x[e], x[e], p) : __fadd_rn(p, x[e]);
-            }
-        }
-        p = lane_butterfly(p);
-        float inv, mu = 0.0f;
-        if (KIND == 0) {
-            inv = __fdiv_rn(1.0f, __fsqrt_rn(__fadd_rn(__fdiv_rn(p, static_cast<float>(K)), eps)));
-        } else {
-            mu = __fdiv_rn(p, static_cast<float>(K));
-            float q = 0.0f;
-#pragma unroll
-            for (int u = 0; u < REG_OCTS; ++u) {
-                if (lane + 32 * u < octs) {
-                    float x[8];
-                    pq::unpack8(v[u], x);
-#pragma unroll
-                    for (int e = 0; e < 8; ++e) {
-                        const float d = __fsub_rn(x[e], mu);
-                        q = __fmaf_rn(d, d, q);
-                    }
-                }
-            }
-            q = lane_butterfly(q);
-            inv = __fdiv_rn(1.0f, __fsqrt_rn(__fadd_rn(__fdiv_rn(q, static_cast<float>(K)), eps)));
-        }
-#pragma unroll
-        for (int u = 0; u < REG_OCTS; ++u) {
-            const int o = lane + 32 * u;
-            if (o < octs) {
-                float x[8], y[8];
-                pq::unpack8(v[u], x);
-                const float4 a0 = __ldg(reinterpret_cast<const float4 *>(a + o * 8)), a1 = __ldg(reinterpret_cast<const float4 *>(a + o * 8) + 1);
-                const float w[8] = {a0.x, a0.y, a0.z, a0.w, a1.x, a1.y, a1.z, a1.w};
-                if (KIND == 0) {
-#pragma unroll
-                    for (int e = 0; e < 8; ++e) y[e] = __fmul_rn(__fmul_rn(x[e], inv), w[e]);
-                } else {
-                    const float4 b0 = __ldg(reinterpret_cast<const float4 *>(b + o * 8)), b1 = __ldg(reinterpret_cast<const float4 *>(b + o * 8) + 1);
-                    const float sh[8] = {b0.x, b0.y, b0.z, b0.w, b1.x, b1.y, b1.z, b1.w};
-#pragma unroll
-                    for (int e = 0; e < 8; ++e)
-                        y[e] = __fmaf_rn(__fmul_rn(__fsub_rn(x[e], mu), inv), __fadd_rn(1.0f, w[e]), sh[e]);
-                }
-                reinterpret_cast<float4 *>(ys)[o] = make_float4(y[0], y[1], y[2], y[3]);
-                reinterpret_cast<float4 *>(ys)[octs + o] = make_float4(y[4], y[5], y[6], y[7]);
-            }
-        }
-    }
-    __syncwarp();
-
-    for (int g0 = 0; g0 < gpr; g0 += 32) {
-        const int g = g0 + lane;
-        const bool have = g < gpr;
-        float x[8], y[8];
-#pragma unroll
-        for (int e = 0; e < 8; ++e) x[e] = 0.0f, y[e] = 0.0f;
-        if (live && have) {
-            if (perm) {
-                const int4 *pi = reinterpret_cast<const int4 *>(perm + g * 16);
-                const int4 i0 = __ldg(pi), i1 = __ldg(pi + 1), i2 = __ldg(pi + 2), i3 = __ldg(pi + 3);
-                x[0] = ys[swz(i0.x, octs)], x[1] = ys[swz(i0.y, octs)], x[2] = ys[swz(i0.z, octs)], x[3] = ys[swz(i0.w, octs)];
-                x[4] = ys[swz(i1.x, octs)], x[5] = ys[swz(i1.y, octs)], x[6] = ys[swz(i1.z, octs)], x[7] = ys[swz(i1.w, octs)];
-                y[0] = ys[swz(i2.x, octs)], y[1] = ys[swz(i2.y, octs)], y[2] = ys[swz(i2.z, octs)], y[3] = ys[swz(i2.w, octs)];
-                y[4] = ys[swz(i3.x, octs)], y[5] = ys[swz(i3.y, octs)], y[6] = ys[swz(i3.z, octs)], y[7] = ys[swz(i3.w, octs)];
-            } else {
-                const float4 *v4 = reinterpret_cast<const float4 *>(ys);
-                const float4 u0 = v4[2 * g], u1 = v4[octs + 2 * g], u2 = v4[2 * g + 1], u3 = v4[octs + 2 * g + 1];
-                x[0] = u0.x, x[1] = u0.y, x[2] = u0.z, x[3] = u0.w, x[4] = u1.x, x[5] = u1.y, x[6] = u1.z, x[7] = u1.w;
-                y[0] = u2.x, y[1] = u2.y, y[2] = u2.z, y[3] = u2.w, y[4] = u3.x, y[5] = u3.y, y[6] = u3.z, y[7] = u3.w;
-            }
-        }
-        quantize_and_store<SF_LAYOUT>(x, y, row, g, gpr, K, live, have, ts, codes, sf, y_out);
-    }
-}
-
 template <int KIND, int SF_LAYOUT>
 __global__ void __launch_bounds__(32 * kMaxRowsPerBlock)
 norm_quant_kernel(const uint16_t *__restrict__ H, int64_t rows, int64_t rows_pad, int K, int64_t ld,
                   const float *__restrict__ a, const float *__restrict__ b, float eps,
                   const int32_t *__restrict__ perm, const float *__restrict__ ts_ptr, uint8_t *__restrict__ codes,
                   uint8_t *__restrict__ sf, uint16_t *__restrict__ y_out) {
-    extern __shared__ __align__(16) float row_s[];  // [warps][K]
+    extern __shared__ __align__(16) uint16_t row_s[];  // [warps][K] bf16 bit patterns
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int64_t row = static_cast<int64_t>(blockIdx.x) * (blockDim.x >> 5) + warp;
     if (row >= rows_pad) return;  // whole warps only
     const bool live = row < rows;
-    float *ys = row_s + static_cast<size_t>(warp) * K;
+    uint16_t *xs = row_s + static_cast<size_t>(warp) * K;
     const int octs = K >> 3, gpr = K >> 4;
     const float ts = __ldg(ts_ptr);
+    float inv = 0.0f, mu = 0.0f;
 
     if (live) {
-        // ---- the row, once: fp32 copy in shared memory, first statistic
+        // ---- the row, once: a copy in shared memory (for the gather) and the first statistic;
+        // four loads in flight per lane and step, sums in ascending octet order
         const uint16_t *src = H + row * ld;
         float p = 0.0f;
-        // four loads in flight per lane and step (the sums still run in ascending octet order)
         for (int o0 = lane; o0 < octs; o0 += 128) {
             uint4 v[4];
 #pragma unroll
@@ -210,82 +57,108 @@ norm_quant_kernel(const uint16_t *__restrict__ H, int64_t rows, int64_t rows_pad
             for (int u = 0; u < 4; ++u) {
                 const int o = o0 + 32 * u;
                 if (o >= octs) break;
+                reinterpret_cast<uint4 *>(xs)[o] = v[u];
                 float x[8];
                 pq::unpack8(v[u], x);
-                reinterpret_cast<float4 *>(ys + o * 8)[0] = make_float4(x[0], x[1], x[2], x[3]);
-                reinterpret_cast<float4 *>(ys + o * 8)[1] = make_float4(x[4], x[5], x[6], x[7]);
 #pragma unroll
                 for (int e = 0; e < 8; ++e) p = KIND == 0 ? __fmaf_rn(x[e], x[e], p) : __fadd_rn(p, x[e]);
             }
         }
         p = lane_butterfly(p);
-        float inv, mu = 0.0f;
         if (KIND == 0) {
             inv = __fdiv_rn(1.0f, __fsqrt_rn(__fadd_rn(__fdiv_rn(p, static_cast<float>(K)), eps)));
         } else {
             mu = __fdiv_rn(p, static_cast<float>(K));
             float q = 0.0f;
             for (int o = lane; o < octs; o += 32) {  // the lane re-reads what it wrote
-                float4 *v = reinterpret_cast<float4 *>(ys + o * 8);
-                float4 u0 = v[0], u1 = v[1];
-                float d[8] = {u0.x, u0.y, u0.z, u0.w, u1.x, u1.y, u1.z, u1.w};
+                float x[8];
+                pq::unpack8(reinterpret_cast<const uint4 *>(xs)[o], x);
 #pragma unroll
                 for (int e = 0; e < 8; ++e) {
-                    d[e] = __fsub_rn(d[e], mu);
-                    q = __fmaf_rn(d[e], d[e], q);
+                    const float d = __fsub_rn(x[e], mu);
+                    q = __fmaf_rn(d, d, q);
                 }
-                v[0] = make_float4(d[0], d[1], d[2], d[3]);
-                v[1] = make_float4(d[4], d[5], d[6], d[7]);
             }
             q = lane_butterfly(q);
             inv = __fdiv_rn(1.0f, __fsqrt_rn(__fadd_rn(__fdiv_rn(q, static_cast<float>(K)), eps)));
         }
-        // ---- scale / modulation, in place, original channel order (coalesced parameter loads)
-        for (int o = lane; o < octs; o += 32) {
-            float4 *v = reinterpret_cast<float4 *>(ys + o * 8);
-            const float4 u0 = v[0], u1 = v[1];
-            const float4 a0 = __ldg(reinterpret_cast<const float4 *>(a + o * 8)), a1 = __ldg(reinterpret_cast<const float4 *>(a + o * 8) + 1);
-            const float x[8] = {u0.x, u0.y, u0.z, u0.w, u1.x, u1.y, u1.z, u1.w};
-            const float w[8] = {a0.x, a0.y, a0.z, a0.w, a1.x, a1.y, a1.z, a1.w};
-            float y[8];
-            if (KIND == 0) {
-#pragma unroll
-                for (int e = 0; e < 8; ++e) y[e] = __fmul_rn(__fmul_rn(x[e], inv), w[e]);
-            } else {
-                const float4 b0 = __ldg(reinterpret_cast<const float4 *>(b + o * 8)), b1 = __ldg(reinterpret_cast<const float4 *>(b + o * 8) + 1);
-                const float sh[8] = {b0.x, b0.y, b0.z, b0.w, b1.x, b1.y, b1.z, b1.w};
-#pragma unroll
-                for (int e = 0; e < 8; ++e) y[e] = __fmaf_rn(__fmul_rn(x[e], inv), __fadd_rn(1.0f, w[e]), sh[e]);
-            }
-            v[0] = make_float4(y[0], y[1], y[2], y[3]);
-            v[1] = make_float4(y[4], y[5], y[6], y[7]);
-        }
     }
     __syncwarp();
 
-    // ---- output order: gather, quantize, store
-    for (int g0 = 0; g0 < gpr; g0 += 32) {
-        const int g = g0 + lane;
-        const bool have = g < gpr;
-        float x[8], y[8];
-#pragma unroll
-        for (int e = 0; e < 8; ++e) x[e] = 0.0f, y[e] = 0.0f;
+    // ---- output order, four positions per lane (so that the permutation indices and the parameters
+    // are read with one contiguous 16-byte load per lane): gather, normalize, quantize; the four
+    // lanes of a group share its absmax through two shuffles and each derive the scale.
+    const int quads = K >> 2;
+    for (int q0 = 0; q0 < quads; q0 += 32) {
+        const int q = q0 + lane;           // positions 4q .. 4q+3, group q >> 2
+        const bool have = q < quads;
+        float out[4] = {0.0f, 0.0f, 0.0f, 0.0f};
         if (live && have) {
+            float v[4];
             if (perm) {
-                const int4 *pi = reinterpret_cast<const int4 *>(perm + g * 16);
-                const int4 i0 = __ldg(pi), i1 = __ldg(pi + 1), i2 = __ldg(pi + 2), i3 = __ldg(pi + 3);
-                x[0] = ys[i0.x], x[1] = ys[i0.y], x[2] = ys[i0.z], x[3] = ys[i0.w];
-                x[4] = ys[i1.x], x[5] = ys[i1.y], x[6] = ys[i1.z], x[7] = ys[i1.w];
-                y[0] = ys[i2.x], y[1] = ys[i2.y], y[2] = ys[i2.z], y[3] = ys[i2.w];
-                y[4] = ys[i3.x], y[5] = ys[i3.y], y[6] = ys[i3.z], y[7] = ys[i3.w];
+                const int4 idx = __ldg(reinterpret_cast<const int4 *>(perm) + q);
+                v[0] = pq::bf16_bits_to_f32(xs[idx.x]), v[1] = pq::bf16_bits_to_f32(xs[idx.y]);
+                v[2] = pq::bf16_bits_to_f32(xs[idx.z]), v[3] = pq::bf16_bits_to_f32(xs[idx.w]);
             } else {
-                const float4 *v = reinterpret_cast<const float4 *>(ys + g * 16);
-                const float4 u0 = v[0], u1 = v[1], u2 = v[2], u3 = v[3];
-                x[0] = u0.x, x[1] = u0.y, x[2] = u0.z, x[3] = u0.w, x[4] = u1.x, x[5] = u1.y, x[6] = u1.z, x[7] = u1.w;
-                y[0] = u2.x, y[1] = u2.y, y[2] = u2.z, y[3] = u2.w, y[4] = u3.x, y[5] = u3.y, y[6] = u3.z, y[7] = u3.w;
+                const uint2 w = reinterpret_cast<const uint2 *>(xs)[q];
+                v[0] = __uint_as_float(w.x << 16), v[1] = __uint_as_float(w.x & 0xFFFF0000u);
+                v[2] = __uint_as_float(w.y << 16), v[3] = __uint_as_float(w.y & 0xFFFF0000u);
+            }
+            const float4 a4 = __ldg(reinterpret_cast<const float4 *>(a) + q);
+            const float w[4] = {a4.x, a4.y, a4.z, a4.w};
+            if (KIND == 0) {
+#pragma unroll
+                for (int j = 0; j < 4; ++j) out[j] = __fmul_rn(__fmul_rn(v[j], inv), w[j]);
+            } else {
+                const float4 b4 = __ldg(reinterpret_cast<const float4 *>(b) + q);
+                const float sh[4] = {b4.x, b4.y, b4.z, b4.w};
+#pragma unroll
+                for (int j = 0; j < 4; ++j)
+                    out[j] = __fmaf_rn(__fmul_rn(__fsub_rn(v[j], mu), inv), __fadd_rn(1.0f, w[j]), sh[j]);
             }
         }
-        quantize_and_store<SF_LAYOUT>(x, y, row, g, gpr, K, live, have, ts, codes, sf, y_out);
+        float amax = fmaxf(fmaxf(fabsf(out[0]), fabsf(out[1])), fmaxf(fabsf(out[2]), fabsf(out[3])));
+        amax = fmaxf(amax, __shfl_xor_sync(0xFFFFFFFFu, amax, 1));
+        amax = fmaxf(amax, __shfl_xor_sync(0xFFFFFFFFu, amax, 2));
+        uint32_t sf8;
+        float d, r;
+        pq::nvfp4_scale(amax, ts, sf8, d, r);
+        uint16_t c16;
+        asm("{\n"
+            ".reg .b8 lo, hi;\n"
+            "cvt.rn.satfinite.e2m1x2.f32 lo, %2, %1;\n"
+            "cvt.rn.satfinite.e2m1x2.f32 hi, %4, %3;\n"
+            "mov.b16 %0, {lo, hi};\n"
+            "}\n"
+            : "=h"(c16)
+            : "f"(__fmul_rn(out[0], r)), "f"(__fmul_rn(out[1], r)), "f"(__fmul_rn(out[2], r)), "f"(__fmul_rn(out[3], r)));
+        if (live && have) {
+            *reinterpret_cast<uint16_t *>(codes + row * (K >> 1) + q * 2) = c16;
+            if (y_out) {
+                const uint32_t w0 = __bfloat16_as_ushort(__float2bfloat16_rn(out[0])) |
+                                    (static_cast<uint32_t>(__bfloat16_as_ushort(__float2bfloat16_rn(out[1]))) << 16);
+                const uint32_t w1 = __bfloat16_as_ushort(__float2bfloat16_rn(out[2])) |
+                                    (static_cast<uint32_t>(__bfloat16_as_ushort(__float2bfloat16_rn(out[3]))) << 16);
+                reinterpret_cast<uint2 *>(y_out + row * K)[q] = make_uint2(w0, w1);
+            }
+        }
+        // scale bytes: the first lane of each group holds its byte; four neighbouring groups sit in
+        // lanes l, l + 4, l + 8, l + 12 (padding rows write zeros)
+        uint32_t word = sf8;
+        word |= __shfl_down_sync(0xFFFFFFFFu, sf8, 4) << 8;
+        word |= __shfl_down_sync(0xFFFFFFFFu, sf8, 8) << 16;
+        word |= __shfl_down_sync(0xFFFFFFFFu, sf8, 12) << 24;
+        if (!have || (q & 3) != 0) continue;
+        const int g = q >> 2;
+        if (SF_LAYOUT == PQ_SF_TCGEN05) {
+            if ((g & 3) == 0) *reinterpret_cast<uint32_t *>(sf + pq::sf_tc_offset(row, g, gpr >> 2)) = word;
+        } else if (live) {
+            if ((gpr & 3) == 0) {
+                if ((g & 3) == 0) *reinterpret_cast<uint32_t *>(sf + row * gpr + g) = word;
+            } else {
+                sf[row * gpr + g] = static_cast<uint8_t>(sf8);
+            }
+        }
     }
 }
 
@@ -293,23 +166,16 @@ template <int KIND, int SF_LAYOUT>
 pq_status launch(const uint16_t *H, int64_t M, int64_t rows_pad, int K, int64_t ld, const float *a, const float *b,
                  float eps, const int32_t *perm, const float *ts, uint8_t *codes, uint8_t *sf, uint16_t *y_out,
                  cudaStream_t st) {
-    int warps = static_cast<int>(kSmemBudget / (static_cast<size_t>(K) * 4));
+    // one warp per row, the row as bf16 in shared memory: 8 rows per block up to 12800 channels
+    int warps = static_cast<int>(kSmemBudget / (static_cast<size_t>(K) * 2));
     if (warps > kMaxRowsPerBlock) warps = kMaxRowsPerBlock;
     if (warps < 1) return PQ_ERR_SHAPE;
-    const size_t smem = static_cast<size_t>(warps) * K * 4;
+    const size_t smem = static_cast<size_t>(warps) * K * 2;
     if (smem > 48 * 1024)
         PQ_CUDA_OK(cudaFuncSetAttribute(norm_quant_kernel<KIND, SF_LAYOUT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                         static_cast<int>(smem)));
     const int64_t blocks = pq_ceil_div(rows_pad, warps);
     PQ_REQUIRE(blocks < (1ll << 31), PQ_ERR_SHAPE);
-    if (K <= 8 * 32 * 16) {  // up to 4096 channels: the row stays in registers as packed bf16
-        if (smem > 48 * 1024)
-            PQ_CUDA_OK(cudaFuncSetAttribute(norm_quant_reg_kernel<KIND, SF_LAYOUT, 16>,
-                                            cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)));
-        norm_quant_reg_kernel<KIND, SF_LAYOUT, 16><<<static_cast<unsigned>(blocks), warps * 32, smem, st>>>(
-            H, M, rows_pad, K, ld, a, b, eps, perm, ts, codes, sf, y_out);
-        return pq_launch_status();
-    }
     norm_quant_kernel<KIND, SF_LAYOUT><<<static_cast<unsigned>(blocks), warps * 32, smem, st>>>(
         H, M, rows_pad, K, ld, a, b, eps, perm, ts, codes, sf, y_out);
     return pq_launch_status();
