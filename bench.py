@@ -415,7 +415,8 @@ def run_ours(args):
 
         def stage(name, ms, nbytes, **extra):
             gbs = nbytes / ms / 1e6
-            stages[name] = {"ms": ms, "GB/s": gbs, "frac_hbm": gbs / hbm, "bytes": nbytes, **extra}
+            stages[name] = {"ms": ms, "GB/s": gbs, "frac_hbm": gbs / hbm, "frac_hbm_nominal_8000": gbs / 8000.0,
+                            "bytes": nbytes, **extra}
 
         big = [torch.cat(xs[0:8]), torch.cat(xs[2:10])]          # 2 x 226 MB
         for tag, src, rows in (("", xs, M), ("_8batches", big, 8 * M)):
