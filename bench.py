@@ -316,17 +316,19 @@ def run_ours(args):
     # ---- the same loop held for about 1.5 s: the 1 kW power cap engages after a few hundred steps and
     # the SM clock settles near 1.6 GHz; this figure goes with the sustained peak, the headline (a few
     # hundred steps unless --steps says otherwise) with the burst peak
-    sustained_steps = 20000
-    for i in range(3):
-        step(i)
-    barrier()
-    a2, b2 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    a2.record()
-    for i in range(sustained_steps):
-        step(i)
-    b2.record()
-    barrier()
-    ms_sustained = max_over_ranks(a2.elapsed_time(b2) / sustained_steps)
+    sustained_steps = 20000 if args.steps >= 100 else 0      # skipped in short (profiling) runs
+    ms_sustained = None
+    if sustained_steps:
+        for i in range(3):
+            step(i)
+        barrier()
+        a2, b2 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a2.record()
+        for i in range(sustained_steps):
+            step(i)
+        b2.record()
+        barrier()
+        ms_sustained = max_over_ranks(a2.elapsed_time(b2) / sustained_steps)
 
     # ---- the two kernels of the step on their own (same launch configuration, same rotation)
     iters = max(20, min(args.steps, 200))
@@ -350,7 +352,7 @@ def run_ours(args):
               "gemm_w4a4": {"ms": ms_gemm, "TFLOP/s": gemm_tflops},
               "linear_incl_quant": {"ms": ms_step, "TFLOP/s": flops / (ms_step * 1e-3) / 1e12,
                                     "frac_fp4_peak": flops / (ms_step * 1e-3) / 1e12 / fp4_peak},
-              "linear_incl_quant_sustained": {
+              "linear_incl_quant_sustained": None if ms_sustained is None else {
                   "ms": ms_sustained, "steps": sustained_steps, "TFLOP/s": flops / (ms_sustained * 1e-3) / 1e12,
                   "frac_fp4_sustained_peak": flops / (ms_sustained * 1e-3) / 1e12
                                              / (peaks["bf16_tflops_sustained"] * FP4_OVER_BF16)}}
