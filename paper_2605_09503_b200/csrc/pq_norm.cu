@@ -5,11 +5,11 @@
 // One warp per token row.  The row is read once with coalesced 16-byte loads (lane l owns the
 // octets l, l + 32, ...: the summation order of the row statistics is this walk followed by a
 // butterfly over the lanes, and does not depend on the permutation) and kept in shared memory as
-// bf16; then each lane takes four consecutive positions of the OUTPUT order (a quarter of a group),
+// bf16; then each lane takes eight consecutive positions of the OUTPUT order (half a group),
 // gathers their channels from shared memory through the permutation, normalizes them with the
-// scale / shift of the output positions (the parameters arrive reordered: one contiguous 16-byte
-// load per lane, like the indices) and quantizes them like the stand-alone quantizer (the four
-// lanes of a group share the absmax by shuffles; 2-byte code stores, coalesced; scale bytes of four
+// scale / shift of the output positions (the parameters arrive reordered: two contiguous 16-byte
+// loads per lane, like the indices) and quantizes them like the stand-alone quantizer (the two
+// lanes of a group share the absmax by a shuffle; 4-byte code stores, coalesced; scale bytes of four
 // neighbouring groups merged into one 32-bit store).  The normalized values exist only in registers, in fp32.  Optionally the
 // reordered bf16 tensor of the unfused kernel is written too.
 #include "pq_common.cuh"
@@ -17,6 +17,9 @@
 namespace {
 
 constexpr int kMaxRowsPerBlock = 8;
+#ifndef PQ_NORM_POS
+#define PQ_NORM_POS 8
+#endif
 constexpr size_t kSmemBudget = 200 * 1024;
 
 __device__ __forceinline__ float lane_butterfly(float p) {
@@ -85,71 +88,93 @@ norm_quant_kernel(const uint16_t *__restrict__ H, int64_t rows, int64_t rows_pad
     }
     __syncwarp();
 
-    // ---- output order, four positions per lane (so that the permutation indices and the parameters
-    // are read with one contiguous 16-byte load per lane): gather, normalize, quantize; the four
-    // lanes of a group share its absmax through two shuffles and each derive the scale.
-    const int quads = K >> 2;
-    for (int q0 = 0; q0 < quads; q0 += 32) {
-        const int q = q0 + lane;           // positions 4q .. 4q+3, group q >> 2
-        const bool have = q < quads;
-        float out[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+    // ---- output order, POS = 4 or 8 consecutive positions per lane (a quarter or half of a group;
+    // the indices and parameters of a lane are one or two contiguous 16-byte loads): gather,
+    // normalize, quantize; the lanes of a group share its absmax by shuffles and each derive the scale.
+    constexpr int POS = PQ_NORM_POS, LPG = 16 / POS;  // lanes per group
+    const int slots = K / POS;
+    for (int q0 = 0; q0 < slots; q0 += 32) {
+        const int q = q0 + lane;           // positions POS q .. POS q + POS - 1, group q / LPG
+        const bool have = q < slots;
+        float out[POS];
+#pragma unroll
+        for (int j = 0; j < POS; ++j) out[j] = 0.0f;
         if (live && have) {
-            float v[4];
-            if (perm) {
-                const int4 idx = __ldg(reinterpret_cast<const int4 *>(perm) + q);
-                v[0] = pq::bf16_bits_to_f32(xs[idx.x]), v[1] = pq::bf16_bits_to_f32(xs[idx.y]);
-                v[2] = pq::bf16_bits_to_f32(xs[idx.z]), v[3] = pq::bf16_bits_to_f32(xs[idx.w]);
-            } else {
-                const uint2 w = reinterpret_cast<const uint2 *>(xs)[q];
-                v[0] = __uint_as_float(w.x << 16), v[1] = __uint_as_float(w.x & 0xFFFF0000u);
-                v[2] = __uint_as_float(w.y << 16), v[3] = __uint_as_float(w.y & 0xFFFF0000u);
+            float v[POS], w[POS];
+#pragma unroll
+            for (int h = 0; h < POS / 4; ++h) {
+                if (perm) {
+                    const int4 idx = __ldg(reinterpret_cast<const int4 *>(perm) + q * (POS / 4) + h);
+                    v[4 * h + 0] = pq::bf16_bits_to_f32(xs[idx.x]), v[4 * h + 1] = pq::bf16_bits_to_f32(xs[idx.y]);
+                    v[4 * h + 2] = pq::bf16_bits_to_f32(xs[idx.z]), v[4 * h + 3] = pq::bf16_bits_to_f32(xs[idx.w]);
+                } else {
+                    const uint2 u = reinterpret_cast<const uint2 *>(xs)[q * (POS / 4) + h];
+                    v[4 * h + 0] = __uint_as_float(u.x << 16), v[4 * h + 1] = __uint_as_float(u.x & 0xFFFF0000u);
+                    v[4 * h + 2] = __uint_as_float(u.y << 16), v[4 * h + 3] = __uint_as_float(u.y & 0xFFFF0000u);
+                }
+                const float4 a4 = __ldg(reinterpret_cast<const float4 *>(a) + q * (POS / 4) + h);
+                w[4 * h + 0] = a4.x, w[4 * h + 1] = a4.y, w[4 * h + 2] = a4.z, w[4 * h + 3] = a4.w;
             }
-            const float4 a4 = __ldg(reinterpret_cast<const float4 *>(a) + q);
-            const float w[4] = {a4.x, a4.y, a4.z, a4.w};
             if (KIND == 0) {
 #pragma unroll
-                for (int j = 0; j < 4; ++j) out[j] = __fmul_rn(__fmul_rn(v[j], inv), w[j]);
+                for (int j = 0; j < POS; ++j) out[j] = __fmul_rn(__fmul_rn(v[j], inv), w[j]);
             } else {
-                const float4 b4 = __ldg(reinterpret_cast<const float4 *>(b) + q);
-                const float sh[4] = {b4.x, b4.y, b4.z, b4.w};
+                float sh[POS];
 #pragma unroll
-                for (int j = 0; j < 4; ++j)
+                for (int h = 0; h < POS / 4; ++h) {
+                    const float4 b4 = __ldg(reinterpret_cast<const float4 *>(b) + q * (POS / 4) + h);
+                    sh[4 * h + 0] = b4.x, sh[4 * h + 1] = b4.y, sh[4 * h + 2] = b4.z, sh[4 * h + 3] = b4.w;
+                }
+#pragma unroll
+                for (int j = 0; j < POS; ++j)
                     out[j] = __fmaf_rn(__fmul_rn(__fsub_rn(v[j], mu), inv), __fadd_rn(1.0f, w[j]), sh[j]);
             }
         }
-        float amax = fmaxf(fmaxf(fabsf(out[0]), fabsf(out[1])), fmaxf(fabsf(out[2]), fabsf(out[3])));
-        amax = fmaxf(amax, __shfl_xor_sync(0xFFFFFFFFu, amax, 1));
-        amax = fmaxf(amax, __shfl_xor_sync(0xFFFFFFFFu, amax, 2));
+        float amax = 0.0f;
+#pragma unroll
+        for (int j = 0; j < POS; ++j) amax = fmaxf(amax, fabsf(out[j]));
+#pragma unroll
+        for (int m = 1; m < LPG; m <<= 1) amax = fmaxf(amax, __shfl_xor_sync(0xFFFFFFFFu, amax, m));
         uint32_t sf8;
         float d, r;
         pq::nvfp4_scale(amax, ts, sf8, d, r);
-        uint16_t c16;
-        asm("{\n"
-            ".reg .b8 lo, hi;\n"
-            "cvt.rn.satfinite.e2m1x2.f32 lo, %2, %1;\n"
-            "cvt.rn.satfinite.e2m1x2.f32 hi, %4, %3;\n"
-            "mov.b16 %0, {lo, hi};\n"
-            "}\n"
-            : "=h"(c16)
-            : "f"(__fmul_rn(out[0], r)), "f"(__fmul_rn(out[1], r)), "f"(__fmul_rn(out[2], r)), "f"(__fmul_rn(out[3], r)));
+        uint32_t cw = 0;
+#pragma unroll
+        for (int h = 0; h < POS / 4; ++h) {
+            uint16_t c16;
+            asm("{\n"
+                ".reg .b8 lo, hi;\n"
+                "cvt.rn.satfinite.e2m1x2.f32 lo, %2, %1;\n"
+                "cvt.rn.satfinite.e2m1x2.f32 hi, %4, %3;\n"
+                "mov.b16 %0, {lo, hi};\n"
+                "}\n"
+                : "=h"(c16)
+                : "f"(__fmul_rn(out[4 * h], r)), "f"(__fmul_rn(out[4 * h + 1], r)), "f"(__fmul_rn(out[4 * h + 2], r)),
+                  "f"(__fmul_rn(out[4 * h + 3], r)));
+            cw |= static_cast<uint32_t>(c16) << (16 * h);
+        }
         if (live && have) {
-            *reinterpret_cast<uint16_t *>(codes + row * (K >> 1) + q * 2) = c16;
+            uint8_t *cdst = codes + row * (K >> 1) + q * (POS / 2);
+            if (POS == 4) *reinterpret_cast<uint16_t *>(cdst) = static_cast<uint16_t>(cw);
+            else *reinterpret_cast<uint32_t *>(cdst) = cw;
             if (y_out) {
-                const uint32_t w0 = __bfloat16_as_ushort(__float2bfloat16_rn(out[0])) |
-                                    (static_cast<uint32_t>(__bfloat16_as_ushort(__float2bfloat16_rn(out[1]))) << 16);
-                const uint32_t w1 = __bfloat16_as_ushort(__float2bfloat16_rn(out[2])) |
-                                    (static_cast<uint32_t>(__bfloat16_as_ushort(__float2bfloat16_rn(out[3]))) << 16);
-                reinterpret_cast<uint2 *>(y_out + row * K)[q] = make_uint2(w0, w1);
+                uint32_t yw[POS / 2];
+#pragma unroll
+                for (int j = 0; j < POS / 2; ++j)
+                    yw[j] = __bfloat16_as_ushort(__float2bfloat16_rn(out[2 * j])) |
+                            (static_cast<uint32_t>(__bfloat16_as_ushort(__float2bfloat16_rn(out[2 * j + 1]))) << 16);
+                if (POS == 4) reinterpret_cast<uint2 *>(y_out + row * K)[q] = make_uint2(yw[0], yw[1]);
+                else reinterpret_cast<uint4 *>(y_out + row * K)[q] = make_uint4(yw[0], yw[1], yw[POS / 2 - 2], yw[POS / 2 - 1]);
             }
         }
-        // scale bytes: the first lane of each group holds its byte; four neighbouring groups sit in
-        // lanes l, l + 4, l + 8, l + 12 (padding rows write zeros)
+        // scale bytes: the first lane of each group holds its byte; four neighbouring groups sit LPG
+        // lanes apart (padding rows write zeros)
         uint32_t word = sf8;
-        word |= __shfl_down_sync(0xFFFFFFFFu, sf8, 4) << 8;
-        word |= __shfl_down_sync(0xFFFFFFFFu, sf8, 8) << 16;
-        word |= __shfl_down_sync(0xFFFFFFFFu, sf8, 12) << 24;
-        if (!have || (q & 3) != 0) continue;
-        const int g = q >> 2;
+        word |= __shfl_down_sync(0xFFFFFFFFu, sf8, LPG) << 8;
+        word |= __shfl_down_sync(0xFFFFFFFFu, sf8, 2 * LPG) << 16;
+        word |= __shfl_down_sync(0xFFFFFFFFu, sf8, 3 * LPG) << 24;
+        if (!have || (q % LPG) != 0) continue;
+        const int g = q / LPG;
         if (SF_LAYOUT == PQ_SF_TCGEN05) {
             if ((g & 3) == 0) *reinterpret_cast<uint32_t *>(sf + pq::sf_tc_offset(row, g, gpr >> 2)) = word;
         } else if (live) {
