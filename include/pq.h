@@ -213,7 +213,11 @@ pq_status pq_quant_act_nvfp4(const void *X, int64_t M, int64_t K, int64_t ld, co
  *        caller zeroes it once (cudaMemset) before the first GEMM that uses it; the kernel only
  *        ever writes a non-zero code there.
  * Every device-side wait is bounded; if one expires the kernel records PQ_ERR_TIMEOUT in the
- * status word (read it with pq_device_status) and returns. */
+ * status word (read it with pq_device_status) and returns.
+ * Launch: the kernel (like the activation quantizer) is launched as a programmatic dependent of
+ * the kernel before it in `stream`: its set-up may overlap that kernel's last thread blocks, and
+ * it waits for that kernel to complete before it reads or writes global memory, so what the
+ * caller observes is ordinary stream order. */
 pq_status pq_gemm_w4a4(const uint8_t *xq, const uint8_t *sfx, const float *ts_x, const uint8_t *wq,
                        const uint8_t *sfw, const float *ts_w, int64_t M, int64_t N, int64_t K,
                        void *Y, int64_t ldy, void *ws, size_t ws_bytes, void *stream);
