@@ -88,6 +88,11 @@ const char *pq_status_string(pq_status s);
 /* Library version as major*100 + minor. */
 int pq_version(void);
 
+/* Text of the last CUDA runtime failure behind a PQ_ERR_CUDA returned to this host thread
+ * ("<cuda error name>: <failed call> (line N)"), or "" if there was none.  The pointer stays valid;
+ * the text is overwritten by the next failure on the same thread. */
+const char *pq_last_error_detail(void);
+
 /* Bytes of scratch the given entry point needs for these sizes (rows = M / T / N as the entry
  * point calls it, P = number of candidate orders, ignored elsewhere).  Never fails; unknown op
  * returns 0.  The workspace must be 256-byte aligned. */

@@ -61,6 +61,7 @@ _SIGNATURES = {
     "pq_sf_to_linear": (_int, [_vp, _i64, _i64, _vp, _vp]),
     "pq_norm_quant_nvfp4": (_int, [_vp, _i64, _i64, _i64, _int, _vp, _vp, C.c_float, _vp, _vp, _vp, _vp, _int, _vp,
                                    _vp]),
+    "pq_last_error_detail": (C.c_char_p, []),
     "pq_device_status": (_int, [_vp, _vp]),
     "pq_probe_sm_ingest": (_int, [_vp, _sz, _int, _int, _int, _vp, _vp, _vp]),
     "pq_probe_sm_store": (_int, [_vp, _sz, _int, _int, _vp, _vp]),
@@ -91,7 +92,12 @@ def status_string(code):
 
 def _check(name, code):
     if code != PQ_OK:
-        raise PqError(name, code, status_string(code))
+        detail = status_string(code)
+        if code == 6:   # PQ_ERR_CUDA: say which call failed
+            extra = lib().pq_last_error_detail()
+            if extra:
+                detail += " -- " + extra.decode()
+        raise PqError(name, code, detail)
 
 
 def _stream():

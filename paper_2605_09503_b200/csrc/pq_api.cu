@@ -1,4 +1,6 @@
 // Entry points that launch no kernel: status strings, version, workspace sizing.
+#include <cstdio>
+
 #include "pq_common.cuh"
 
 extern "C" const char *pq_status_string(pq_status s) {
@@ -16,6 +18,15 @@ extern "C" const char *pq_status_string(pq_status s) {
 }
 
 extern "C" int pq_version(void) { return 1; }
+
+// Last CUDA failure seen by this host thread, as text: "<cuda error name>: <call> (line N)".
+static thread_local char g_last_error[256] = "";
+
+void pq_note_cuda_error(cudaError_t err, const char *what, int line) {
+    snprintf(g_last_error, sizeof(g_last_error), "%s: %.180s (line %d)", cudaGetErrorName(err), what, line);
+}
+
+extern "C" const char *pq_last_error_detail(void) { return g_last_error; }
 
 static size_t round256(size_t b) { return (b + 255) / 256 * 256; }
 

@@ -17,19 +17,27 @@
         if (!(cond)) return (code); \
     } while (0)
 
-#define PQ_CUDA_OK(expr)                          \
-    do {                                          \
-        if ((expr) != cudaSuccess) {              \
-            (void)cudaGetLastError();             \
-            return PQ_ERR_CUDA;                   \
-        }                                         \
+// Records which CUDA call failed (readable through pq_last_error_detail) -- defined in pq_api.cu.
+void pq_note_cuda_error(cudaError_t err, const char *what, int line);
+
+#define PQ_CUDA_OK(expr)                                     \
+    do {                                                     \
+        const cudaError_t pq_err_ = (expr);                  \
+        if (pq_err_ != cudaSuccess) {                        \
+            pq_note_cuda_error(pq_err_, #expr, __LINE__);    \
+            (void)cudaGetLastError();                        \
+            return PQ_ERR_CUDA;                              \
+        }                                                    \
     } while (0)
 
 static inline bool pq_aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 static inline bool pq_aligned256(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 255u) == 0; }
 
 static inline pq_status pq_launch_status() {
-    return cudaGetLastError() == cudaSuccess ? PQ_OK : PQ_ERR_CUDA;
+    const cudaError_t e = cudaGetLastError();
+    if (e == cudaSuccess) return PQ_OK;
+    pq_note_cuda_error(e, "kernel launch", 0);
+    return PQ_ERR_CUDA;
 }
 
 static inline int64_t pq_ceil_div(int64_t a, int64_t b) { return (a + b - 1) / b; }

@@ -20,8 +20,9 @@
 //   warps 6..13  scale-factor stagers: read the stage's scale blocks from shared memory and write
 //                them into one of three scale slots in tensor memory with tcgen05.st (one warp per
 //                lane quadrant; two sets of four warps take alternate K iterations).
-// 192 divides every FLUX output width (3072, 9216, 12288) and leaves room in the 512 tensor-memory
-// columns for two accumulators (384) plus three scale slots (3 x 40).
+// 256 divides every FLUX output width (3072, 9216, 12288).  The 512 tensor-memory columns hold one
+// 256-column accumulator plus four scale slots (4 x 48); the epilogue warps pull the accumulator
+// into registers as packed bf16 within a few hundred cycles and store it from there.
 //
 // Measurements on B200 behind these choices:
 //   - a tcgen05.cp of one 512-byte scale block occupies the tensor pipe for about 80 cycles and
@@ -55,27 +56,28 @@
 
 namespace {
 
-constexpr int BM = 256, BM_CTA = 128, BN = 192, BN_CTA = BN / 2, BK = 256;
+constexpr int BM = 256, BM_CTA = 128, BN = 256, BN_CTA = BN / 2, BK = 256;
 constexpr int kStages = 5;
 constexpr int kABytes = BM_CTA * BK / 2;   // 16384
-constexpr int kBBytes = BN_CTA * BK / 2;   // 12288
+constexpr int kBBytes = BN_CTA * BK / 2;   // 16384
 constexpr int kSfBlock = 512;              // 128 rows x 4 groups
 constexpr int kSfaBytes = 4 * kSfBlock;    // 4 K-blocks of one 128-row block
 constexpr int kSfbBytes = 2 * kSfaBytes;   // two 128-row blocks
-constexpr int kStageBytes = kABytes + kBBytes + kSfaBytes + kSfbBytes;  // 34816 = 34 * 1024
+constexpr int kStageBytes = kABytes + kBBytes + kSfaBytes + kSfbBytes;  // 38912 = 38 * 1024
 constexpr int kEpiBox = 32 * 128;          // 32 rows x 64 bf16, one TMA store
-constexpr int kEpiBytes = 4 * 2 * kEpiBox; // two boxes per epilogue warp
-constexpr int kThreads = 448;              // producer, MMA issuer, 4 epilogue and 8 stager warps
+constexpr int kEpiWarps = 8;               // lane quadrant x column half of the accumulator
+constexpr int kEpiBytes = kEpiWarps * kEpiBox;      // one staging box per epilogue warp: 32 KB
+constexpr int kFirstStager = 2 + kEpiWarps;
+constexpr int kThreads = 32 * (kFirstStager + 8);   // producer, MMA issuer, 8 epilogue and 8 stager warps
 constexpr int kTmemCols = 512;
-constexpr uint32_t kAccStride = BN;        // accumulator b starts at column b * 192
-// Three scale slots follow the accumulators.  A slot holds the scales of one stage: per 64-channel
-// K block 4 columns of A scales (128 rows) and 6 columns of B scales (192 rows).
-constexpr int kSfSlots = 3;
-constexpr uint32_t kSfSlotCol0 = 2 * BN, kSfSlotCols = 4 * (4 + 6), kSfbOfs = 16;
+// One 256-column accumulator, then four scale slots.  A slot holds the scales of one stage: per
+// 64-channel K block 4 columns of A scales (128 rows) and 8 columns of B scales (256 rows).
+constexpr int kSfSlots = 4;
+constexpr uint32_t kSfSlotCol0 = BN, kSfSlotCols = 4 * (4 + 8), kSfbOfs = 16;
 static_assert(kSfSlotCol0 + kSfSlots * kSfSlotCols <= 512, "tensor memory columns");
 constexpr long long kWaitCycles = 4000000000ll;  // about two seconds of SM clock per wait
-// barriers: stage_full[S] sf_ready[S] stage_free[S] acc_full[2] acc_empty[2]
-constexpr int kNumBars = 3 * kStages + 4;
+// barriers: stage_full[S] sf_ready[S] stage_free[S] acc_full acc_empty
+constexpr int kNumBars = 3 * kStages + 2;
 constexpr size_t kSmemBytes = kStages * kStageBytes + kEpiBytes + 1024 /*alignment slack*/ + 8 * kNumBars + 64;
 
 struct GemmParams {
@@ -243,6 +245,15 @@ __device__ __forceinline__ void tc_ld32(uint32_t taddr, uint32_t (&v)[32]) {
         : "r"(taddr)
         : "memory");
 }
+__device__ __forceinline__ void tc_ld16(uint32_t taddr, uint32_t (&v)[16]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];\n"
+        : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
+          "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15])
+        : "r"(taddr)
+        : "memory");
+}
 __device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tc_st4(uint32_t taddr, const uint4 &v) {
     asm volatile("tcgen05.st.sync.aligned.32x32b.x4.b32 [%0], {%1, %2, %3, %4};" ::"r"(taddr), "r"(v.x), "r"(v.y),
@@ -252,16 +263,10 @@ __device__ __forceinline__ void tc_st4(uint32_t taddr, const uint4 &v) {
 __device__ __forceinline__ void tc_st2(uint32_t taddr, uint32_t a, uint32_t b) {
     asm volatile("tcgen05.st.sync.aligned.32x32b.x2.b32 [%0], {%1, %2};" ::"r"(taddr), "r"(a), "r"(b) : "memory");
 }
-// Six columns of B scales of one K block: the 32-row words of the tile's 192 rows, picked from the
-// two 128-row blocks the tile touches (`mid`: the tile starts in the middle of the first block).
-__device__ __forceinline__ void stage_b_scales(uint32_t taddr, const uint4 &b0, const uint4 &b1, bool mid) {
-    if (mid) {
-        tc_st4(taddr, make_uint4(b0.z, b0.w, b1.x, b1.y));
-        tc_st2(taddr + 4, b1.z, b1.w);
-    } else {
-        tc_st4(taddr, b0);
-        tc_st2(taddr + 4, b1.x, b1.y);
-    }
+// Eight columns of B scales of one K block: the two 128-row blocks of the tile's 256 rows.
+__device__ __forceinline__ void stage_b_scales(uint32_t taddr, const uint4 &b0, const uint4 &b1) {
+    tc_st4(taddr, b0);
+    tc_st4(taddr + 4, b1);
 }
 __device__ __forceinline__ void tc_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ uint4 lds128(uint32_t addr) {
@@ -295,10 +300,11 @@ __device__ __forceinline__ uint32_t pack_bf16(uint32_t lo_bits, uint32_t hi_bits
 }
 
 // ---------------------------------------------------------------- kernel
-// Register budget: with 112 registers per thread the four warps an SM sub-partition gets from
-// this CTA leave it 2048 registers, room for two warps of a 32-register kernel, so a 256-thread
-// block of the activation quantizer can run on the SM beside the GEMM (batched linear path).
-constexpr int kMaxRegs = 112;
+// Register budget: the register file is split over the four SM sub-partitions (16384 registers
+// each) and two of them receive five of this CTA's 18 warps: 5 x 32 x 96 = 15360 fits, 104 would not.
+// The 1024 registers left there take one warp of a 32-register kernel, so 128-thread blocks of
+// other kernels can still run on the SM beside the GEMM.
+constexpr int kMaxRegs = 96;
 __global__ void __cluster_dims__(2, 1, 1) __maxnreg__(kMaxRegs)
 gemm_w4a4_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                  const __grid_constant__ CUtensorMap map_y, const GemmParams p) {
@@ -314,8 +320,8 @@ gemm_w4a4_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
     auto stage_full_bar = [&](int s) { return bars + 8u * s; };
     auto sf_ready_bar = [&](int s) { return bars + 8u * (kStages + s); };     // scale blocks landed (own CTA)
     auto stage_free_bar = [&](int s) { return bars + 8u * (2 * kStages + s); };  // the stage's MMAs have run
-    auto acc_full_bar = [&](int b) { return bars + 8u * (3 * kStages + b); };
-    auto acc_empty_bar = [&](int b) { return bars + 8u * (3 * kStages + 2 + b); };  // leader's copy only
+    const uint32_t acc_full_bar = bars + 8u * (3 * kStages);
+    const uint32_t acc_empty_bar = bars + 8u * (3 * kStages + 1);  // leader's copy only
     uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars_ptr + 8 * kNumBars);
     volatile int *abort_flag = reinterpret_cast<volatile int *>(bars_ptr + 8 * kNumBars + 8);
 
@@ -329,10 +335,8 @@ gemm_w4a4_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
             mbar_init(sf_ready_bar(s), 1);
             mbar_init(stage_free_bar(s), 1);
         }
-        for (int b = 0; b < 2; ++b) {
-            mbar_init(acc_full_bar(b), 1);
-            mbar_init(acc_empty_bar(b), 8);  // 4 epilogue warps in each CTA
-        }
+        mbar_init(acc_full_bar, 1);
+        mbar_init(acc_empty_bar, 2 * kEpiWarps);  // the epilogue warps of both CTAs
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         prefetch_tensormap(&map_a);
@@ -412,10 +416,11 @@ gemm_w4a4_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
             uint32_t s = 0, ph = 0, t = 0, tcount = 0;
             bool ok = true;
             for (int tile = pair; tile < total_tiles && ok; tile += num_pairs, ++tcount) {
-                const uint32_t b = tcount & 1u, accpar = (tcount >> 1) & 1u;
-                ok = mbar_wait_warp(acc_empty_bar(b), accpar ^ 1u, abort_flag, p.status);
+                // the accumulator is free once the epilogue has read the previous tile out of it
+                ok = mbar_wait_warp(acc_empty_bar, (tcount & 1u) ^ 1u, abort_flag, p.status);
                 if (!ok) break;
-                const uint32_t d_tmem = tmem_base + b * kAccStride;
+                tc_fence_after();
+                const uint32_t d_tmem = tmem_base;
                 uint32_t acc = 0;
                 for (int kt = 0; kt < p.k_tiles; ++kt) {
                     ok = mbar_wait_warp(stage_full_bar(s), ph, abort_flag, p.status);
@@ -428,12 +433,12 @@ gemm_w4a4_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
                     if (elect_one()) {
                         if (kb_valid == 4) {
                             tc_mma_pair(d_tmem, da, db, kIdesc, sfa_t, sfb_t, acc);
-                            tc_mma_pair(d_tmem, da + 2, db + 2, kIdesc, sfa_t + 4, sfb_t + 6, 1u);
-                            tc_mma_pair(d_tmem, da + 4, db + 4, kIdesc, sfa_t + 8, sfb_t + 12, 1u);
-                            tc_mma_pair(d_tmem, da + 6, db + 6, kIdesc, sfa_t + 12, sfb_t + 18, 1u);
+                            tc_mma_pair(d_tmem, da + 2, db + 2, kIdesc, sfa_t + 4, sfb_t + 8, 1u);
+                            tc_mma_pair(d_tmem, da + 4, db + 4, kIdesc, sfa_t + 8, sfb_t + 16, 1u);
+                            tc_mma_pair(d_tmem, da + 6, db + 6, kIdesc, sfa_t + 12, sfb_t + 24, 1u);
                         } else {
                             for (int kk = 0; kk < kb_valid; ++kk)
-                                tc_mma_pair(d_tmem, da + 2 * kk, db + 2 * kk, kIdesc, sfa_t + 4 * kk, sfb_t + 6 * kk,
+                                tc_mma_pair(d_tmem, da + 2 * kk, db + 2 * kk, kIdesc, sfa_t + 4 * kk, sfb_t + 8 * kk,
                                             acc | static_cast<uint32_t>(kk));
                         }
                         // the stage (and its scale slot) is free in both CTAs once these MMAs have run
@@ -446,21 +451,20 @@ gemm_w4a4_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
                     ph ^= (s == 0) ? 1u : 0u;
                     t = (t + 1 == kSfSlots) ? 0u : t + 1;
                 }
-                if (ok && elect_one()) tc_commit_pair(acc_full_bar(b));  // the leader's epilogue passes it on
+                if (ok && elect_one()) tc_commit_pair(acc_full_bar);  // the leader's epilogue passes it on
                 __syncwarp();
             }
         }
-    } else if (warp >= 6) {
+    } else if (warp >= kFirstStager) {
         // ------------------------------------------------------------ scale-factor stagers
         // Two sets of four warps (one warp per tensor-memory lane quadrant) take alternate K
         // iterations, so a set has two stages' worth of MMA time for one stage of scales.
         const uint32_t q = warp & 3;  // tensor-memory lane quadrant this warp may write
-        const uint32_t set = static_cast<uint32_t>(warp - 6) >> 2;
+        const uint32_t set = static_cast<uint32_t>(warp - kFirstStager) >> 2;
         const uint32_t lane_ofs = (q * 32u) << 16;
         uint32_t it = 0;
         bool ok = true;
         for (int tile = pair; tile < total_tiles && ok; tile += num_pairs) {
-            const bool mid = (((tile / p.m_tiles) * BN) & 127) != 0;
             for (int kt = 0; kt < p.k_tiles; ++kt, ++it) {
                 if ((it & 1u) != set) continue;
                 const int s = it % kStages;
@@ -494,7 +498,7 @@ gemm_w4a4_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
 #pragma unroll
                     for (int kk = 0; kk < 4; ++kk) {
                         tc_st4(sf_t + 4 * kk, a[kk]);
-                        stage_b_scales(sf_t + kSfbOfs + 6 * kk, b0[kk], b1[kk], mid);
+                        stage_b_scales(sf_t + kSfbOfs + 8 * kk, b0[kk], b1[kk]);
                     }
                 } else {
                     for (int kk = 0; kk < kb_valid; ++kk) {
@@ -502,7 +506,7 @@ gemm_w4a4_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
                         const uint4 b0 = lds128(sf_s + kSfaBytes + kk * kSfBlock);
                         const uint4 b1 = lds128(sf_s + 2 * kSfaBytes + kk * kSfBlock);
                         tc_st4(sf_t + 4 * kk, a);
-                        stage_b_scales(sf_t + kSfbOfs + 6 * kk, b0, b1, mid);
+                        stage_b_scales(sf_t + kSfbOfs + 8 * kk, b0, b1);
                     }
                 }
                 tc_wait_st();
@@ -513,46 +517,47 @@ gemm_w4a4_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
         }
     } else {
         // ------------------------------------------------------------ epilogue
-        const int q = warp & 3;  // tensor-memory lane quadrant this warp may read
+        // Eight warps: lane quadrant q x column half h.  A warp reads its 32 rows x 128 columns
+        // out of tensor memory, scales and rounds them to bf16 and keeps them packed in 64
+        // registers; the accumulator goes back to the MMA issuer after those four loads (a few
+        // hundred cycles), and the two 64-column boxes leave through one staging box and TMA
+        // stores behind the next tile's main loop.
+        const int q = warp & 3;                // tensor-memory lane quadrant this warp may read
+        const int h = (warp - 2) >> 2;         // column half
         const float alpha = __fmul_rn(__ldg(p.ts_x), __ldg(p.ts_w));
-        const uint32_t my_epi = epi + static_cast<uint32_t>(q) * (2 * kEpiBox);
+        const uint32_t buf = epi + static_cast<uint32_t>(warp - 2) * kEpiBox;
         const uint32_t row_ofs = static_cast<uint32_t>(lane) * 128u, sw = static_cast<uint32_t>(lane & 7);
-        uint32_t tcount = 0, boxes = 0;
+        uint32_t tcount = 0;
         for (int tile = pair; tile < total_tiles; tile += num_pairs, ++tcount) {
             const int m_blk = tile % p.m_tiles, n_blk = tile / p.m_tiles;
-            const int m0 = m_blk * BM + static_cast<int>(rank) * BM_CTA + q * 32, n0 = n_blk * BN;
-            const uint32_t b = tcount & 1u, accpar = (tcount >> 1) & 1u;
-            const bool got = mbar_wait(acc_full_bar(b), accpar, abort_flag, p.status);
+            const int m0 = m_blk * BM + static_cast<int>(rank) * BM_CTA + q * 32, n0 = n_blk * BN + h * (BN / 2);
+            const bool got = mbar_wait(acc_full_bar, tcount & 1u, abort_flag, p.status);
             if (!__all_sync(0xFFFFFFFFu, got)) break;
-            if (rank == 0 && q == 0 && lane == 0) mbar_arrive_remote(acc_full_bar(b), 1);
+            if (rank == 0 && warp == 2 && lane == 0) mbar_arrive_remote(acc_full_bar, 1);
             tc_fence_after();
-            const uint32_t acc = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + b * kAccStride;
-#pragma unroll 1
-            for (int c = 0; c < BN / 64; ++c, ++boxes) {
-                uint32_t v[32], w[32];
-                tc_ld32(acc + c * 64, v);
-                tc_ld32(acc + c * 64 + 32, w);
+            const uint32_t acc = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + h * (BN / 2);
+            uint32_t pk[64];  // pk[8 c + i] = columns 16 c + 2 i, 16 c + 2 i + 1 of this lane's row
+#pragma unroll
+            for (int c = 0; c < 8; ++c) {
+                uint32_t v[16];
+                tc_ld16(acc + c * 16, v);
                 tc_wait_ld();
-                if (c == BN / 64 - 1) {
-                    // the whole accumulator has been read: hand it back to the MMA issuer
-                    tc_fence_before();
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive_leader(acc_empty_bar(b), rank);
-                }
-                const uint32_t buf = my_epi + (boxes & 1u) * kEpiBox;
-                // the TMA store that read this box two boxes ago must have finished reading it
-                if (lane == 0) bulk_wait_read<1>();
+#pragma unroll
+                for (int i = 0; i < 8; ++i) pk[8 * c + i] = pack_bf16(v[2 * i], v[2 * i + 1], alpha);
+            }
+            // this warp's part of the accumulator has been read: hand it back to the MMA issuer
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive_leader(acc_empty_bar, rank);
+#pragma unroll
+            for (int c = 0; c < 2; ++c) {
+                // the store that read the box before (previous chunk or previous tile) must be done with it
+                if (lane == 0) bulk_wait_read<0>();
                 __syncwarp();
 #pragma unroll
-                for (int i = 0; i < 4; ++i)
-                    sts128(buf + row_ofs + ((static_cast<uint32_t>(i) ^ sw) << 4), pack_bf16(v[8 * i], v[8 * i + 1], alpha),
-                           pack_bf16(v[8 * i + 2], v[8 * i + 3], alpha), pack_bf16(v[8 * i + 4], v[8 * i + 5], alpha),
-                           pack_bf16(v[8 * i + 6], v[8 * i + 7], alpha));
-#pragma unroll
-                for (int i = 0; i < 4; ++i)
-                    sts128(buf + row_ofs + ((static_cast<uint32_t>(i + 4) ^ sw) << 4),
-                           pack_bf16(w[8 * i], w[8 * i + 1], alpha), pack_bf16(w[8 * i + 2], w[8 * i + 3], alpha),
-                           pack_bf16(w[8 * i + 4], w[8 * i + 5], alpha), pack_bf16(w[8 * i + 6], w[8 * i + 7], alpha));
+                for (int i = 0; i < 8; ++i)
+                    sts128(buf + row_ofs + ((static_cast<uint32_t>(i) ^ sw) << 4), pk[32 * c + 4 * i], pk[32 * c + 4 * i + 1],
+                           pk[32 * c + 4 * i + 2], pk[32 * c + 4 * i + 3]);
                 fence_async_smem();
                 __syncwarp();
                 if (lane == 0) {
