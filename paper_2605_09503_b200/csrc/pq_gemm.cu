@@ -3,22 +3,25 @@
 //   Y[m,n] = bf16( ts_x*ts_w * sum_k (qx[m,k]*sfx[m,k/16]) * (qw[n,k]*sfw[n,k/16]) )
 //
 // Design.  Thread-block clusters of two CTAs (one per SM) work as a pair on output tiles of
-// 256 x 192, persistent over the tile list: tcgen05.mma.cta_group::2 lets each CTA hold 128 rows
+// 256 x 256, persistent over the tile list: tcgen05.mma.cta_group::2 lets each CTA hold 128 rows
 // of the accumulator while the B operand is split between the two shared memories, so a CTA
-// fetches 128 rows of X codes and only 96 rows of W codes per 256-channel K step -- a quarter
-// less L2->SM traffic than two independent 128 x 192 tiles.  Roles of the 14 warps of a CTA:
+// fetches 128 rows of X codes and 128 rows of W codes per 256-channel K step (38 KB with the
+// scales, for 512 cycles of MMA).  What bounds the main loop is the rate at which the SMs can take
+// operands in from L2 (about 70 bytes per clock each when all of them pull), so the tile is as
+// large as tensor memory allows.  Roles of the 18 warps of a CTA:
 //   warp 0       producer: TMA loads of the packed E2M1 operand tiles (128-byte swizzle) and bulk
 //                copies of the scale-factor blocks into a 5-stage shared-memory ring.  Operand
 //                loads of both CTAs signal the pair leader's barrier (cp.async.bulk.tensor with
 //                .cta_group::2).
 //   warp 1       (leader CTA) issues tcgen05.mma.kind::mxf4nvf4.block_scale, K = 64 per instruction,
-//                4 per stage, into one of two 192-column fp32 accumulators in tensor memory.
-//   warps 2..5   epilogue: tcgen05.ld the finished accumulator (own CTA's 128 rows), scale by
-//                ts_x*ts_w, round to bf16, stage 32 x 64 boxes in swizzled shared memory and write
-//                them with TMA stores (full 128-byte lines) -- overlapping the next tile's main
-//                loop through the second accumulator.
-//   warps 6..13  scale-factor stagers: read the stage's scale blocks from shared memory and write
-//                them into one of three scale slots in tensor memory with tcgen05.st (one warp per
+//                4 per stage, into the 256-column fp32 accumulator in tensor memory.
+//   warps 2..9   epilogue (lane quadrant x column half): tcgen05.ld the finished accumulator (own
+//                CTA's 128 rows) 16 columns at a time, scale by ts_x*ts_w, round to bf16 and keep the
+//                32 x 128 piece as 64 packed registers; hand the accumulator back; then stage 32 x 64
+//                boxes in swizzled shared memory and write them with TMA stores (full 128-byte
+//                lines) while the next tile's main loop runs.
+//   warps 10..17 scale-factor stagers: read the stage's scale blocks from shared memory and write
+//                them into one of four scale slots in tensor memory with tcgen05.st (one warp per
 //                lane quadrant; two sets of four warps take alternate K iterations).
 // 256 divides every FLUX output width (3072, 9216, 12288).  The 512 tensor-memory columns hold one
 // 256-column accumulator plus four scale slots (4 x 48); the epilogue warps pull the accumulator
@@ -41,8 +44,7 @@
 // block occupies 4 tensor-memory columns (row r of the block -> lane r%32, column r/32, the same
 // in all four lane quadrants), which is the layout the MMA reads: lane l of every stager warp
 // loads the 16 bytes at offset 16 l of the block and stores them as columns of its quadrant.
-// The 192 B-scale rows of a tile span two blocks; the stagers pick the six 32-row words that
-// belong to the tile (it may start in the middle of a block) and store them as 6 columns.
+// The 256 B-scale rows of a tile are two whole blocks: 8 columns per K block.
 //
 // Cross-CTA signalling uses plain remote mbarrier arrives and, for the completion of a stage's
 // MMAs, one tcgen05.commit per CTA (the leader's epilogue passes accumulator completions on).  Every wait on an mbarrier is bounded.  If one expires the CTA
@@ -537,13 +539,19 @@ gemm_w4a4_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
             tc_fence_after();
             const uint32_t acc = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + h * (BN / 2);
             uint32_t pk[64];  // pk[8 c + i] = columns 16 c + 2 i, 16 c + 2 i + 1 of this lane's row
+            // two loads in flight: chunk c + 1 is on its way while chunk c is scaled and packed
+            uint32_t va[16], vb[16];
+            tc_ld16(acc, va);
 #pragma unroll
-            for (int c = 0; c < 8; ++c) {
-                uint32_t v[16];
-                tc_ld16(acc + c * 16, v);
+            for (int c = 0; c < 8; c += 2) {
                 tc_wait_ld();
+                tc_ld16(acc + (c + 1) * 16, vb);
 #pragma unroll
-                for (int i = 0; i < 8; ++i) pk[8 * c + i] = pack_bf16(v[2 * i], v[2 * i + 1], alpha);
+                for (int i = 0; i < 8; ++i) pk[8 * c + i] = pack_bf16(va[2 * i], va[2 * i + 1], alpha);
+                tc_wait_ld();
+                if (c + 2 < 8) tc_ld16(acc + (c + 2) * 16, va);
+#pragma unroll
+                for (int i = 0; i < 8; ++i) pk[8 * (c + 1) + i] = pack_bf16(vb[2 * i], vb[2 * i + 1], alpha);
             }
             // this warp's part of the accumulator has been read: hand it back to the MMA issuer
             tc_fence_before();
