@@ -42,6 +42,10 @@ static inline pq_status pq_launch_status() {
 
 static inline int64_t pq_ceil_div(int64_t a, int64_t b) { return (a + b - 1) / b; }
 
+// pq_quant_act_nvfp4 with a choice of block shape (library-internal; defined in pq_quant.cu).
+pq_status pq_quant_act_nvfp4_shaped(const void *X, int64_t M, int64_t K, int64_t ld, const float *ts_x, uint8_t *codes,
+                                    uint8_t *sf, int sf_layout, int small_blocks, void *stream);
+
 #ifdef __CUDACC__
 
 namespace pq {

@@ -828,7 +828,8 @@ extern "C" pq_status pq_linear_w4a4_batched(int n, const void *const *X, int64_t
             const int s = i % n_sets;
             // the GEMM that last read this set of intermediates has to be done with it
             if (i >= n_sets && cudaStreamWaitEvent(pipe->q, pipe->g_done[s], 0) != cudaSuccess) rc = PQ_ERR_CUDA;
-            if (rc == PQ_OK) rc = pq_quant_act_nvfp4(X[i], M, K, ld, ts_x, xq[s], sfx[s], PQ_SF_TCGEN05, pipe->q);
+            // 128-thread blocks: they fit on an SM beside the GEMM's CTA
+            if (rc == PQ_OK) rc = pq_quant_act_nvfp4_shaped(X[i], M, K, ld, ts_x, xq[s], sfx[s], PQ_SF_TCGEN05, 1, pipe->q);
             if (rc == PQ_OK && cudaEventRecord(pipe->q_done[s], pipe->q) != cudaSuccess) rc = PQ_ERR_CUDA;
             if (rc == PQ_OK && cudaStreamWaitEvent(pipe->g, pipe->q_done[s], 0) != cudaSuccess) rc = PQ_ERR_CUDA;
         }

@@ -16,7 +16,9 @@ namespace {
 
 constexpr int kQuantThreads = 256;
 constexpr int kTileRows = 8;                    // blocks of the streaming kernels: 32 lanes along K x 8 rows
-constexpr int kActThreads = 32 * kTileRows;     // activation quantizer
+// The activation quantizer comes in two block shapes: 8 warps (best alone) and 4 warps, one per SM
+// sub-partition at 32 registers, which is what fits on an SM beside a GEMM CTA (batched linear path).
+constexpr int kActThreads = 32 * kTileRows;
 constexpr unsigned kGridYMax = 65535;
 
 // Row block of a (x = column chunk, y/z = row block) grid; y alone is limited to 65535 blocks.
@@ -34,7 +36,7 @@ inline dim3 tile_grid(int64_t col_chunks, int64_t row_blocks) {
 // 32-byte aligned), the group's absmax, scale and codes in registers, an 8-byte store of codes.
 // The scale bytes of four adjacent groups are collected with shuffles into one 32-bit store
 // (adjacent in both scale layouts).  The index space covers the rows padded to a multiple of 128
-// in the tensor-core layout; padding rows only write zero scale bytes.  A block owns 8 rows x 32
+// in the tensor-core layout; padding rows only write zero scale bytes.  A block owns 8 (or 4) rows x 32
 // consecutive groups (a warp = 1 KB of one row), so no thread divides anything.
 template <bool WIDE>
 __device__ __forceinline__ void load_group(const uint16_t *p, uint4 &lo, uint4 &hi) {
@@ -53,14 +55,14 @@ __device__ __forceinline__ void load_group(const uint16_t *p, uint4 &lo, uint4 &
 #endif
 constexpr int kActRows = PQ_ACT_ROWS;  // rows per thread: their loads are issued together
 
-template <int SF_LAYOUT, bool WIDE>
+template <int SF_LAYOUT, bool WIDE, int kActTileRows>
 __global__ void __launch_bounds__(kActThreads)
 quant_nvfp4_kernel(const uint16_t *__restrict__ X, int64_t rows, int64_t rows_pad, int64_t K,
                    int64_t ld, const float *__restrict__ ts_ptr, uint8_t *__restrict__ codes,
                    uint8_t *__restrict__ sf) {
     const uint32_t gpr = static_cast<uint32_t>(K >> 4);  // groups per row
     const uint32_t g = blockIdx.x * 32u + threadIdx.x;
-    const int64_t row0 = row_block_index() * (kTileRows * kActRows) + threadIdx.y;
+    const int64_t row0 = row_block_index() * (kActTileRows * kActRows) + threadIdx.y;
     // This kernel is launched as a programmatic dependent of whatever precedes it in the stream:
     // its blocks may become resident while that kernel's last blocks run, and wait here until it
     // has completed and its writes are visible (ordinary stream order from here on).  In turn a
@@ -73,13 +75,13 @@ quant_nvfp4_kernel(const uint16_t *__restrict__ X, int64_t rows, int64_t rows_pa
     uint4 lo[kActRows], hi[kActRows];
 #pragma unroll
     for (int i = 0; i < kActRows; ++i) {
-        const int64_t row = row0 + i * kTileRows;
+        const int64_t row = row0 + i * kActTileRows;
         lo[i] = make_uint4(0, 0, 0, 0), hi[i] = lo[i];
         if (row < rows && g < gpr) load_group<WIDE>(X + row * ld + static_cast<int64_t>(g) * 16, lo[i], hi[i]);
     }
 #pragma unroll
     for (int i = 0; i < kActRows; ++i) {
-        const int64_t row = row0 + i * kTileRows;
+        const int64_t row = row0 + i * kActTileRows;
         const bool in_range = row < rows_pad && g < gpr, live = row < rows && g < gpr;
         float x[8], y[8];
         pq::unpack8(lo[i], x);
@@ -289,9 +291,38 @@ extern "C" size_t pq_sf_bytes(int64_t rows, int64_t K, int sf_layout) {
     return 0;
 }
 
-extern "C" pq_status pq_quant_act_nvfp4(const void *X, int64_t M, int64_t K, int64_t ld,
-                                        const float *ts_x, uint8_t *codes, uint8_t *sf, int sf_layout,
-                                        void *stream) {
+namespace {
+template <int TILE_ROWS>
+pq_status quant_act_launch(const uint16_t *x, int64_t M, int64_t K, int64_t ld, const float *ts_x, uint8_t *codes,
+                           uint8_t *sf, int sf_layout, bool wide, cudaStream_t st) {
+    const int64_t rows_idx = sf_layout == PQ_SF_TCGEN05 ? pq_ceil_div(M, 128) * 128 : M;
+    PQ_REQUIRE(K / 16 <= 32ll * 0x7FFFFFFF && rows_idx / TILE_ROWS < static_cast<int64_t>(kGridYMax) * 65535, PQ_ERR_SHAPE);
+    const dim3 grid = tile_grid(pq_ceil_div(K / 16, 32), pq_ceil_div(rows_idx, TILE_ROWS * kActRows));
+    const dim3 block(32, TILE_ROWS);
+    // The quantizer's blocks should be able to run on an SM beside a GEMM CTA (the batched linear
+    // path overlaps the two kernels): ask for the GEMM's shared-memory carve-out, otherwise an SM
+    // has to drain before it can switch between the two configurations.
+    static bool carveout_set = false;
+    if (!carveout_set) {
+        cudaFuncSetAttribute(quant_nvfp4_kernel<PQ_SF_TCGEN05, true, TILE_ROWS>, cudaFuncAttributePreferredSharedMemoryCarveout, 100);
+        cudaFuncSetAttribute(quant_nvfp4_kernel<PQ_SF_TCGEN05, false, TILE_ROWS>, cudaFuncAttributePreferredSharedMemoryCarveout, 100);
+        (void)cudaGetLastError();
+        carveout_set = true;
+    }
+    if (sf_layout == PQ_SF_TCGEN05) {
+        if (wide) PQ_CUDA_OK(pq::launch_dependent(quant_nvfp4_kernel<PQ_SF_TCGEN05, true, TILE_ROWS>, grid, block, 0, st, x, M, rows_idx, K, ld, ts_x, codes, sf));
+        else PQ_CUDA_OK(pq::launch_dependent(quant_nvfp4_kernel<PQ_SF_TCGEN05, false, TILE_ROWS>, grid, block, 0, st, x, M, rows_idx, K, ld, ts_x, codes, sf));
+    } else {
+        if (wide) PQ_CUDA_OK(pq::launch_dependent(quant_nvfp4_kernel<PQ_SF_LINEAR, true, TILE_ROWS>, grid, block, 0, st, x, M, rows_idx, K, ld, ts_x, codes, sf));
+        else PQ_CUDA_OK(pq::launch_dependent(quant_nvfp4_kernel<PQ_SF_LINEAR, false, TILE_ROWS>, grid, block, 0, st, x, M, rows_idx, K, ld, ts_x, codes, sf));
+    }
+    return pq_launch_status();
+}
+}  // namespace
+
+// small_blocks != 0: 128-thread blocks, for running beside a GEMM (used by the batched linear path)
+pq_status pq_quant_act_nvfp4_shaped(const void *X, int64_t M, int64_t K, int64_t ld, const float *ts_x, uint8_t *codes,
+                                    uint8_t *sf, int sf_layout, int small_blocks, void *stream) {
     PQ_REQUIRE(X && ts_x && codes && sf, PQ_ERR_NULL);
     PQ_REQUIRE(sf_layout == PQ_SF_LINEAR || sf_layout == PQ_SF_TCGEN05, PQ_ERR_FORMAT);
     PQ_REQUIRE(M > 0 && K > 0 && K % 16 == 0 && ld >= K, PQ_ERR_SHAPE);
@@ -301,28 +332,14 @@ extern "C" pq_status pq_quant_act_nvfp4(const void *X, int64_t M, int64_t K, int
     const uint16_t *x = static_cast<const uint16_t *>(X);
     // 256-bit loads need 32-byte aligned groups
     const bool wide = (reinterpret_cast<uintptr_t>(X) & 31u) == 0 && ld % 16 == 0;
-    const int64_t rows_idx = sf_layout == PQ_SF_TCGEN05 ? pq_ceil_div(M, 128) * 128 : M;
-    PQ_REQUIRE(K / 16 <= 32ll * 0x7FFFFFFF && rows_idx / kTileRows < static_cast<int64_t>(kGridYMax) * 65535, PQ_ERR_SHAPE);
-    const dim3 grid = tile_grid(pq_ceil_div(K / 16, 32), pq_ceil_div(rows_idx, kTileRows * kActRows));
-    const dim3 block(32, kTileRows);
-    // The quantizer's blocks should be able to run on an SM beside a GEMM CTA (the batched linear
-    // path overlaps the two kernels): ask for the GEMM's shared-memory carve-out, otherwise an SM
-    // has to drain before it can switch between the two configurations.
-    static bool carveout_set = false;
-    if (!carveout_set) {
-        cudaFuncSetAttribute(quant_nvfp4_kernel<PQ_SF_TCGEN05, true>, cudaFuncAttributePreferredSharedMemoryCarveout, 100);
-        cudaFuncSetAttribute(quant_nvfp4_kernel<PQ_SF_TCGEN05, false>, cudaFuncAttributePreferredSharedMemoryCarveout, 100);
-        (void)cudaGetLastError();
-        carveout_set = true;
-    }
-    if (sf_layout == PQ_SF_TCGEN05) {
-        if (wide) PQ_CUDA_OK(pq::launch_dependent(quant_nvfp4_kernel<PQ_SF_TCGEN05, true>, grid, block, 0, st, x, M, rows_idx, K, ld, ts_x, codes, sf));
-        else PQ_CUDA_OK(pq::launch_dependent(quant_nvfp4_kernel<PQ_SF_TCGEN05, false>, grid, block, 0, st, x, M, rows_idx, K, ld, ts_x, codes, sf));
-    } else {
-        if (wide) PQ_CUDA_OK(pq::launch_dependent(quant_nvfp4_kernel<PQ_SF_LINEAR, true>, grid, block, 0, st, x, M, rows_idx, K, ld, ts_x, codes, sf));
-        else PQ_CUDA_OK(pq::launch_dependent(quant_nvfp4_kernel<PQ_SF_LINEAR, false>, grid, block, 0, st, x, M, rows_idx, K, ld, ts_x, codes, sf));
-    }
-    return pq_launch_status();
+    return small_blocks ? quant_act_launch<4>(x, M, K, ld, ts_x, codes, sf, sf_layout, wide, st)
+                        : quant_act_launch<kTileRows>(x, M, K, ld, ts_x, codes, sf, sf_layout, wide, st);
+}
+
+extern "C" pq_status pq_quant_act_nvfp4(const void *X, int64_t M, int64_t K, int64_t ld,
+                                        const float *ts_x, uint8_t *codes, uint8_t *sf, int sf_layout,
+                                        void *stream) {
+    return pq_quant_act_nvfp4_shaped(X, M, K, ld, ts_x, codes, sf, sf_layout, 0, stream);
 }
 
 extern "C" pq_status pq_quant_weight(const void *Wt, int64_t N, int64_t K, int64_t ld,
