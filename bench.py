@@ -459,7 +459,7 @@ def run_ours(args):
             stage(name, graph_loop(torch, lambda i: B.pq_norm_quant_nvfp4(xs[i % XROT], kind, av, bv, 1e-6, order, cal.ts_x,
                                                                           xq_rot[i % XROT], sfx_rot[i % XROT],
                                                                           B.PQ_SF_TCGEN05), it),
-                  quant_bytes, bound="L1 / shared memory (gather through the permutation)")
+                  quant_bytes, bound="instruction issue / latency (one wave of 16 warps per SM; 16-21 instructions per element)")
         ws_err = B.workspace(B.OP_GROUP_ERROR, M, K, 0, 6)
         e6 = torch.zeros(6, K // 16, dtype=torch.float64, device=dev)
         ms = graph_loop(torch, lambda i: B.pq_group_error(xs[i % XROT], pipeline.NVFP4, cal.ts_x, cal.perms, e6, ws_err),

@@ -2,16 +2,18 @@
 // the channel reordering absorbed into it, and the NVFP4 quantizer of the runtime path (Eq. 8)
 // attached, so the normalized activations never make a bf16 round trip through HBM.
 //
-// One warp per token row.  The row is read once with coalesced 16-byte loads (lane l owns the
+// A warp owns whole token rows.  A row is read once with coalesced 16-byte loads (lane l owns the
 // octets l, l + 32, ...: the summation order of the row statistics is this walk followed by a
 // butterfly over the lanes, and does not depend on the permutation) and kept in shared memory as
-// bf16; then each lane takes eight consecutive positions of the OUTPUT order (half a group),
-// gathers their channels from shared memory through the permutation, normalizes them with the
-// scale / shift of the output positions (the parameters arrive reordered: two contiguous 16-byte
-// loads per lane, like the indices) and quantizes them like the stand-alone quantizer (the two
-// lanes of a group share the absmax by a shuffle; 4-byte code stores, coalesced; scale bytes of four
-// neighbouring groups merged into one 32-bit store).  The normalized values exist only in registers, in fp32.  Optionally the
+// bf16; then the lanes walk the OUTPUT order, gather their channels from shared memory through the
+// permutation, normalize them with the scale / shift of the output positions (the parameters arrive
+// reordered: contiguous 16-byte loads per lane, like the indices) and quantize them like the
+// stand-alone quantizer (coalesced code stores; scale bytes of four neighbouring groups merged into
+// one 32-bit store).  The normalized values exist only in registers, in fp32.  Optionally the
 // reordered bf16 tensor of the unfused kernel is written too.
+//
+// Two kernels: rows of up to 6400 channels go four per warp (below, second kernel); wider rows one
+// per warp, eight positions per lane (first kernel).
 #include "pq_common.cuh"
 
 namespace {
@@ -187,11 +189,268 @@ norm_quant_kernel(const uint16_t *__restrict__ H, int64_t rows, int64_t rows_pad
     }
 }
 
+// ---- several rows per warp ----------------------------------------------------------------------
+// The same computation with the rows taken four (or two) at a time by a warp.  Their bf16 values sit
+// interleaved per channel in shared memory (8 or 4 bytes per channel), so one shared-memory load
+// gathers a channel for all rows of the warp, and the indices and parameters of an output position
+// are fetched once for them; a lane takes a whole group (16 output positions), so the scale is derived
+// once per group and nothing but the scale bytes crosses lanes.  The 16-byte chunks of an octet are
+// XOR-swizzled by bits of the octet index, which makes the transposing stores of the first phase
+// conflict-free.  The order of every floating-point operation is that of the one-row kernel.
+#ifndef PQ_NORM_ROWS
+#define PQ_NORM_ROWS 4
+#endif
+#ifndef PQ_NORM_WARPS
+#define PQ_NORM_WARPS 4
+#endif
+#ifndef PQ_NORM_SPLIT
+#define PQ_NORM_SPLIT 2
+#endif
+// kGroupWarps row groups per block, kSplit warps per row group: the first reads the rows and takes
+// the statistics, then all of them share the walk over the output order
+constexpr int kGroupRows = PQ_NORM_ROWS, kGroupWarps = PQ_NORM_WARPS, kSplit = PQ_NORM_SPLIT;
+static_assert(kGroupRows == 2 || kGroupRows == 4, "rows per warp");
+
+// 16-byte chunk k of octet o (R = 4: two channels per chunk, four chunks; R = 2: four channels, two chunks)
+template <int R>
+__device__ __forceinline__ int chunk_of(int o, int k) {
+    return R == 4 ? 4 * o + (k ^ ((o >> 1) & 3)) : 2 * o + (k ^ ((o >> 2) & 1));
+}
+template <int R>
+__device__ __forceinline__ int swizzled_channel(int c) {
+    return R == 4 ? c ^ (((c >> 4) & 3) << 1) : c ^ (((c >> 5) & 1) << 2);
+}
+// the rows of one channel: R = 4 in (x, y), R = 2 in x
+template <int R>
+__device__ __forceinline__ uint2 channel_rows(const uint16_t *xs, int c) {
+    if (R == 4) return reinterpret_cast<const uint2 *>(xs)[swizzled_channel<4>(c)];
+    return make_uint2(reinterpret_cast<const uint32_t *>(xs)[swizzled_channel<2>(c)], 0u);
+}
+__device__ __forceinline__ float row_value(const uint2 &g, int r) {
+    const uint32_t w = r < 2 ? g.x : g.y;
+    return __uint_as_float((r & 1) ? (w & 0xFFFF0000u) : (w << 16));
+}
+
+template <int KIND, int SF_LAYOUT>
+__global__ void __launch_bounds__(32 * kGroupWarps * kSplit, 2)
+norm_quant_grouped_kernel(const uint16_t *__restrict__ H, int64_t rows, int64_t rows_pad, int K, int64_t ld,
+                        const float *__restrict__ a, const float *__restrict__ b, float eps,
+                        const int32_t *__restrict__ perm, const float *__restrict__ ts_ptr,
+                        uint8_t *__restrict__ codes, uint8_t *__restrict__ sf, uint16_t *__restrict__ y_out) {
+    extern __shared__ __align__(16) uint16_t row_s[];  // [row groups][K][R rows] bf16 bit patterns
+    __shared__ float stat_s[kGroupWarps][2 * kGroupRows];
+    constexpr int R = kGroupRows;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int grp_in_block = warp % kGroupWarps, part = warp / kGroupWarps;
+    const int64_t row0 = (static_cast<int64_t>(blockIdx.x) * kGroupWarps + grp_in_block) * R;
+    const bool present = row0 < rows_pad;  // a row group past the end still joins the barrier
+    const int nlive =
+        present ? static_cast<int>(min(static_cast<int64_t>(R), max(static_cast<int64_t>(0), rows - row0))) : 0;
+    uint16_t *xs = row_s + static_cast<size_t>(grp_in_block) * K * R;
+    uint4 *xs4 = reinterpret_cast<uint4 *>(xs);
+    const int octs = K >> 3, gpr = K >> 4;
+    const float ts = __ldg(ts_ptr);
+    float inv[R], mu[R];
+#pragma unroll
+    for (int r = 0; r < R; ++r) inv[r] = 0.0f, mu[r] = 0.0f;
+
+    if (nlive > 0 && part == 0) {
+        // ---- the rows, once: interleaved copy in shared memory and the first statistic; three
+        // octets of each row in flight per lane, sums in ascending octet order
+        constexpr int U = 3;
+        float p[R];
+#pragma unroll
+        for (int r = 0; r < R; ++r) p[r] = 0.0f;
+        for (int o0 = lane; o0 < octs; o0 += 32 * U) {
+            uint4 v[U][R];
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                const int o = o0 + 32 * u;
+#pragma unroll
+                for (int r = 0; r < R; ++r)
+                    v[u][r] = (o < octs && r < nlive)
+                                  ? __ldcs(reinterpret_cast<const uint4 *>(H + (row0 + r) * ld + o * 8))
+                                  : make_uint4(0, 0, 0, 0);
+            }
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                const int o = o0 + 32 * u;
+                if (o >= octs) break;
+                const uint32_t *w0 = &v[u][0].x, *w1 = &v[u][1].x, *w2 = &v[u][R - 2].x, *w3 = &v[u][R - 1].x;
+                if (R == 4) {
+#pragma unroll
+                    for (int k = 0; k < 4; ++k)
+                        xs4[chunk_of<4>(o, k)] =
+                            make_uint4(__byte_perm(w0[k], w1[k], 0x5410), __byte_perm(w2[k], w3[k], 0x5410),
+                                       __byte_perm(w0[k], w1[k], 0x7632), __byte_perm(w2[k], w3[k], 0x7632));
+                } else {
+#pragma unroll
+                    for (int k = 0; k < 2; ++k)
+                        xs4[chunk_of<2>(o, k)] =
+                            make_uint4(__byte_perm(w0[2 * k], w1[2 * k], 0x5410), __byte_perm(w0[2 * k], w1[2 * k], 0x7632),
+                                       __byte_perm(w0[2 * k + 1], w1[2 * k + 1], 0x5410),
+                                       __byte_perm(w0[2 * k + 1], w1[2 * k + 1], 0x7632));
+                }
+#pragma unroll
+                for (int r = 0; r < R; ++r) {
+                    float x[8];
+                    pq::unpack8(v[u][r], x);
+#pragma unroll
+                    for (int e = 0; e < 8; ++e) p[r] = KIND == 0 ? __fmaf_rn(x[e], x[e], p[r]) : __fadd_rn(p[r], x[e]);
+                }
+            }
+        }
+#pragma unroll
+        for (int r = 0; r < R; ++r) p[r] = lane_butterfly(p[r]);
+        if (KIND == 0) {
+#pragma unroll
+            for (int r = 0; r < R; ++r)
+                if (r < nlive) inv[r] = __fdiv_rn(1.0f, __fsqrt_rn(__fadd_rn(__fdiv_rn(p[r], static_cast<float>(K)), eps)));
+        } else {
+            float q[R];
+#pragma unroll
+            for (int r = 0; r < R; ++r) mu[r] = __fdiv_rn(p[r], static_cast<float>(K)), q[r] = 0.0f;
+            for (int o = lane; o < octs; o += 32) {  // the lane re-reads what it wrote
+#pragma unroll
+                for (int k = 0; k < R; ++k) {  // R chunks per octet
+                    const uint4 c = xs4[chunk_of<R>(o, k)];
+                    const uint32_t cw[4] = {c.x, c.y, c.z, c.w};
+#pragma unroll
+                    for (int i = 0; i < 8 / R; ++i) {  // channels of the chunk, ascending
+                        const uint2 ch = R == 4 ? make_uint2(cw[2 * i], cw[2 * i + 1]) : make_uint2(cw[i], 0u);
+#pragma unroll
+                        for (int r = 0; r < R; ++r) {
+                            const float d0 = __fsub_rn(row_value(ch, r), mu[r]);
+                            q[r] = __fmaf_rn(d0, d0, q[r]);
+                        }
+                    }
+                }
+            }
+#pragma unroll
+            for (int r = 0; r < R; ++r) {
+                q[r] = lane_butterfly(q[r]);
+                if (r < nlive) inv[r] = __fdiv_rn(1.0f, __fsqrt_rn(__fadd_rn(__fdiv_rn(q[r], static_cast<float>(K)), eps)));
+            }
+        }
+    }
+    if (kSplit > 1) {
+        if (part == 0 && lane == 0) {
+#pragma unroll
+            for (int r = 0; r < R; ++r) stat_s[grp_in_block][r] = inv[r], stat_s[grp_in_block][R + r] = mu[r];
+        }
+        __syncthreads();
+#pragma unroll
+        for (int r = 0; r < R; ++r) inv[r] = stat_s[grp_in_block][r], mu[r] = stat_s[grp_in_block][R + r];
+    } else {
+        __syncwarp();
+    }
+    if (!present) return;
+
+    // ---- output order: one whole group (16 consecutive positions) per lane, for all rows of the warp;
+    // the indices and parameters are fetched once, the scale is derived once per group and row
+    constexpr int POS = 16;
+    const bool any_live = nlive > 0;
+    for (int q0 = 32 * part; q0 < gpr; q0 += 32 * kSplit) {
+        const int q = q0 + lane;  // group
+        const bool have = q < gpr;
+        uint2 g[POS];
+        float w[POS], sh[POS];
+#pragma unroll
+        for (int j = 0; j < POS; ++j) g[j] = make_uint2(0, 0), w[j] = 0.0f, sh[j] = 0.0f;
+        if (have && any_live) {
+#pragma unroll
+            for (int h = 0; h < POS / 4; ++h) {
+                const int j0 = POS * q + 4 * h;
+                int4 idx = make_int4(j0, j0 + 1, j0 + 2, j0 + 3);
+                if (perm) idx = __ldg(reinterpret_cast<const int4 *>(perm) + (POS / 4) * q + h);
+                g[4 * h + 0] = channel_rows<R>(xs, idx.x), g[4 * h + 1] = channel_rows<R>(xs, idx.y);
+                g[4 * h + 2] = channel_rows<R>(xs, idx.z), g[4 * h + 3] = channel_rows<R>(xs, idx.w);
+                const float4 a4 = __ldg(reinterpret_cast<const float4 *>(a) + (POS / 4) * q + h);
+                w[4 * h + 0] = a4.x, w[4 * h + 1] = a4.y, w[4 * h + 2] = a4.z, w[4 * h + 3] = a4.w;
+                if (KIND == 1) {
+                    const float4 b4 = __ldg(reinterpret_cast<const float4 *>(b) + (POS / 4) * q + h);
+                    sh[4 * h + 0] = b4.x, sh[4 * h + 1] = b4.y, sh[4 * h + 2] = b4.z, sh[4 * h + 3] = b4.w;
+                }
+            }
+            if (KIND == 1) {
+#pragma unroll
+                for (int j = 0; j < POS; ++j) w[j] = __fadd_rn(1.0f, w[j]);
+            }
+        }
+#pragma unroll
+        for (int r = 0; r < R; ++r) {
+            const int64_t row = row0 + r;
+            const bool live = r < nlive;  // rows past the end carry inv = mu = 0 and zeros in shared memory
+            float out[POS];
+            float amax = 0.0f;
+#pragma unroll
+            for (int j = 0; j < POS; ++j) {
+                const float v = row_value(g[j], r);
+                out[j] = KIND == 0 ? __fmul_rn(__fmul_rn(v, inv[r]), w[j])
+                                   : __fmaf_rn(__fmul_rn(__fsub_rn(v, mu[r]), inv[r]), w[j], sh[j]);
+                amax = fmaxf(amax, fabsf(out[j]));
+            }
+            if (!(live && have)) amax = 0.0f;  // nothing of such a row or group is stored but a zero scale byte
+            uint32_t sf8;
+            float d, rcp;
+            pq::nvfp4_scale(amax, ts, sf8, d, rcp);
+            if (live && have) {
+                float y[8];
+                uint2 cw;
+#pragma unroll
+                for (int j = 0; j < 8; ++j) y[j] = __fmul_rn(out[j], rcp);
+                cw.x = pq::f32x8_to_e2m1(y);
+#pragma unroll
+                for (int j = 0; j < 8; ++j) y[j] = __fmul_rn(out[8 + j], rcp);
+                cw.y = pq::f32x8_to_e2m1(y);
+                *reinterpret_cast<uint2 *>(codes + row * (K >> 1) + q * 8) = cw;
+                if (y_out) {
+                    uint32_t yw[POS / 2];
+#pragma unroll
+                    for (int j = 0; j < POS / 2; ++j)
+                        yw[j] = __bfloat16_as_ushort(__float2bfloat16_rn(out[2 * j])) |
+                                (static_cast<uint32_t>(__bfloat16_as_ushort(__float2bfloat16_rn(out[2 * j + 1]))) << 16);
+                    uint4 *ydst = reinterpret_cast<uint4 *>(y_out + row * K) + 2 * q;
+                    ydst[0] = make_uint4(yw[0], yw[1], yw[2], yw[3]);
+                    ydst[1] = make_uint4(yw[4], yw[5], yw[6], yw[7]);
+                }
+            }
+            // scale bytes: four neighbouring groups sit in neighbouring lanes (padding rows write zeros)
+            uint32_t word = sf8;
+            word |= __shfl_down_sync(0xFFFFFFFFu, sf8, 1) << 8;
+            word |= __shfl_down_sync(0xFFFFFFFFu, sf8, 2) << 16;
+            word |= __shfl_down_sync(0xFFFFFFFFu, sf8, 3) << 24;
+            if (!have || row >= rows_pad) continue;
+            if (SF_LAYOUT == PQ_SF_TCGEN05) {
+                if ((q & 3) == 0) *reinterpret_cast<uint32_t *>(sf + pq::sf_tc_offset(row, q, gpr >> 2)) = word;
+            } else if (live) {
+                if ((gpr & 3) == 0) {
+                    if ((q & 3) == 0) *reinterpret_cast<uint32_t *>(sf + row * gpr + q) = word;
+                } else {
+                    sf[row * gpr + q] = static_cast<uint8_t>(sf8);
+                }
+            }
+        }
+    }
+}
+
 template <int KIND, int SF_LAYOUT>
 pq_status launch(const uint16_t *H, int64_t M, int64_t rows_pad, int K, int64_t ld, const float *a, const float *b,
                  float eps, const int32_t *perm, const float *ts, uint8_t *codes, uint8_t *sf, uint16_t *y_out,
                  cudaStream_t st) {
-    // one warp per row, the row as bf16 in shared memory: 8 rows per block up to 12800 channels
+    // up to 6400 channels: four rows per warp, four warps per block (two blocks per SM at 3072 channels)
+    const size_t group_smem = static_cast<size_t>(kGroupWarps) * kGroupRows * K * 2;
+    if (group_smem <= kSmemBudget) {
+        if (group_smem > 40 * 1024)  // the kernel's static shared memory counts towards the 48 KB default limit
+            PQ_CUDA_OK(cudaFuncSetAttribute(norm_quant_grouped_kernel<KIND, SF_LAYOUT>,
+                                            cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(group_smem)));
+        const int64_t blocks = pq_ceil_div(rows_pad, kGroupWarps * kGroupRows);
+        PQ_REQUIRE(blocks < (1ll << 31), PQ_ERR_SHAPE);
+        norm_quant_grouped_kernel<KIND, SF_LAYOUT><<<static_cast<unsigned>(blocks), kGroupWarps * kSplit * 32, group_smem, st>>>(
+            H, M, rows_pad, K, ld, a, b, eps, perm, ts, codes, sf, y_out);
+        return pq_launch_status();
+    }
+    // wider rows: one warp per row, the row as bf16 in shared memory: 8 rows per block up to 12800 channels
     int warps = static_cast<int>(kSmemBudget / (static_cast<size_t>(K) * 2));
     if (warps > kMaxRowsPerBlock) warps = kMaxRowsPerBlock;
     if (warps < 1) return PQ_ERR_SHAPE;
