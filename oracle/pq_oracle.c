@@ -212,6 +212,35 @@ int pqo_calib_stats(const uint16_t *T, int64_t rows, int64_t K, int64_t ld, doub
     return 0;
 }
 
+/* Output-side calibration error, the other reading of "the quantization error on the
+ * calibration data" of Sec. 3.3 (acceptance rule, Eq. 10): per output column n
+ *     err[n] += sum_t (Yref[t,n] - Yq[t,n])^2
+ * with Yref the unquantized product in fp32 and Yq the bf16 output of the quantized layer.  The
+ * difference is one fp32 subtraction; the squares are summed over rows in chunks and slabs exactly
+ * as in pqo_calib_stats. */
+int pqo_output_error(const float *Yref, int64_t ld_ref, const uint16_t *Yq, int64_t ld_q, int64_t rows,
+                     int64_t N, double *err) {
+    if (!Yref || !Yq || !err || rows <= 0 || N <= 0 || ld_ref < N || ld_q < N) return 1;
+    for (int64_t s0 = 0; s0 < rows; s0 += PQO_SLAB) {
+        int64_t s1 = (s0 + PQO_SLAB < rows) ? s0 + PQO_SLAB : rows;
+#pragma omp parallel for schedule(static)
+        for (int64_t n = 0; n < N; ++n) {
+            double slab = 0.0;
+            for (int64_t r0 = s0; r0 < s1; r0 += PQO_CHUNK) {
+                int64_t r1 = (r0 + PQO_CHUNK < s1) ? r0 + PQO_CHUNK : s1;
+                float p = 0.0f;
+                for (int64_t t = r0; t < r1; ++t) {
+                    float d = Yref[t * ld_ref + n] - pqo_bf16_to_f32(Yq[t * ld_q + n]);
+                    p = fmaf(d, d, p);
+                }
+                slab += (double)p;
+            }
+            err[n] += slab;
+        }
+    }
+    return 0;
+}
+
 /* ------------------------------------------------------------------ permutation candidates */
 
 typedef struct {

@@ -42,6 +42,7 @@ def _declare(L):
     L.pqo_tensor_scale.argtypes = [_P, _i64]
     L.pqo_calib_stats.argtypes = [_P, _i64, _i64, _i64, _P, _P]
     L.pqo_select_perm.argtypes = [_P, _i64, _P, _i64, _i64, C.c_int, _P]
+    L.pqo_output_error.argtypes = [_P, _i64, _P, _i64, _i64, _i64, _P]
     L.pqo_group_error.argtypes = [_P, _i64, _i64, _i64, C.c_int, C.c_int, C.c_int, C.c_float, _P,
                                   C.c_int, _P]
     L.pqo_accept.argtypes = [_P, C.c_double, _P, C.c_double, C.c_int, _i64, C.c_double, _P, _P, _P]
@@ -133,6 +134,19 @@ def calib_stats(T, sumsq=None, amax=None):
         amax = np.zeros(K, dtype=np.float32)
     _check(lib().pqo_calib_stats(_ptr(T), rows, K, K, _ptr(sumsq), _ptr(amax)), "calib_stats")
     return sumsq, amax
+
+
+def output_error(Yref, Yq, err=None):
+    """Sec. 3.3 / Eq. 10, output-side reading: per output column the sum over rows of
+    (Yref - Yq)^2, Yref fp32 [rows, N], Yq bf16 bit patterns [rows, N]; accumulated into err (fp64 [N])."""
+    Yref = np.ascontiguousarray(Yref, dtype=np.float32)
+    Yq = _bf16(Yq)
+    rows, N = Yref.shape
+    assert Yq.shape == (rows, N)
+    if err is None:
+        err = np.zeros(N, dtype=np.float64)
+    _check(lib().pqo_output_error(_ptr(Yref), N, _ptr(Yq), N, rows, N, _ptr(err)), "output_error")
+    return err
 
 
 def select_perm(sumsq_a, rows_a, sumsq_w, rows_w, J=5):
