@@ -73,7 +73,8 @@ enum {
     PQ_OP_SELECT_PERM = 2,
     PQ_OP_GROUP_ERROR = 3,
     PQ_OP_QUANT_WEIGHT = 4,
-    PQ_OP_GEMM = 5
+    PQ_OP_GEMM = 5,
+    PQ_OP_OUTPUT_ERROR = 6
 };
 
 /* Row blocking of the sums in pq_calib_stats and pq_group_error (part of the arithmetic
@@ -170,6 +171,24 @@ pq_status pq_group_error(const void *T, int64_t rows, int64_t K, int64_t ld, pq_
                          const float *ts, const int32_t *perms, int P, double *err, void *ws,
                          size_t ws_bytes, void *stream);
 
+/* Output-side calibration error: "the quantization error on the calibration data" of Sec. 3.3
+ * (the E of the acceptance rule, Eq. 10) read on the layer's output instead of its inputs.  For
+ * every output column n
+ *     err[n] += sum_t (Yref[t,n] - Yq[t,n])^2
+ * Yref is the unquantized product X W^T in fp32 (any GEMM the caller trusts), Yq the bf16 output
+ * of the quantized layer (pq_linear_w4a4 with the candidate order applied to both operands).
+ * The difference is one fp32 subtraction; the squares are accumulated like pq_calib_stats: fp32
+ * fused multiply-add in row order inside a chunk of PQ_CHUNK_ROWS rows, chunks, slabs and the
+ * total in fp64 as stated at PQ_SLAB_ROWS.  sum_n err[n] of the original order and of each
+ * candidate are the E[p] of pq_accept (pass them as err_x with Kg = N and a zero err_w).
+ *   Yref : device fp32 [rows, N], ld_ref elements between rows (ld_ref % 4 == 0, 16-byte aligned).
+ *   Yq   : device bf16 [rows, N], ld_q (ld_q % 8 == 0, 16-byte aligned).  N % 8 == 0.
+ *   err  : device fp64 [N] in/out (the caller zeroes it before the first batch).
+ *   ws   : pq_workspace_bytes(PQ_OP_OUTPUT_ERROR, rows, N, 0, 0)  (N in the place of K). */
+pq_status pq_output_error(const float *Yref, int64_t ld_ref, const void *Yq, int64_t ld_q,
+                          int64_t rows, int64_t N, double *err, void *ws, size_t ws_bytes,
+                          void *stream);
+
 /* Relative-error weights for pq_accept: lambda[0] = 1 / sum_i sumsq_a[i], lambda[1] =
  * 1 / sum_i sumsq_w[i] (sequential fp64 sums in channel order).  lambda: device fp64 [2]. */
 pq_status pq_error_weights(const double *sumsq_a, const double *sumsq_w, int64_t K, double *lambda,
@@ -207,6 +226,15 @@ pq_status pq_quant_weight(const void *Wt, int64_t N, int64_t K, int64_t ld, cons
  *   the tensor-core layout are written as 0). */
 pq_status pq_quant_act_nvfp4(const void *X, int64_t M, int64_t K, int64_t ld, const float *ts_x,
                              uint8_t *codes, uint8_t *sf, int sf_layout, void *stream);
+
+/* The same quantizer with a channel order applied on the way in (codes and scales of X P): the
+ * calibration-time form, used to evaluate a candidate order on the layer output (pq_output_error)
+ * before any producer has been rewritten to emit permuted activations.  One block per row stages
+ * the row in shared memory and gathers from there; perm == NULL is pq_quant_act_nvfp4.
+ *   perm : device int32 [K].  K <= 16384.  Other arguments as for pq_quant_act_nvfp4. */
+pq_status pq_quant_act_nvfp4_perm(const void *X, int64_t M, int64_t K, int64_t ld, const int32_t *perm,
+                                  const float *ts_x, uint8_t *codes, uint8_t *sf, int sf_layout,
+                                  void *stream);
 
 /* W4A4 block-scaled GEMM, right-hand side of Eq. 8:
  *     Y[m,n] = bf16( ts_x*ts_w * sum_kb sfx[m,kb]*sfw[n,kb] * sum_{j<16} qx[m,16kb+j]*qw[n,16kb+j] )

@@ -15,7 +15,7 @@ LIB_PATH = os.path.join(_HERE, "libpq.so")
 
 PQ_OK = 0
 PQ_SF_LINEAR, PQ_SF_TCGEN05 = 0, 1
-OP_CALIB_STATS, OP_SELECT_PERM, OP_GROUP_ERROR, OP_QUANT_WEIGHT, OP_GEMM = 1, 2, 3, 4, 5
+OP_CALIB_STATS, OP_SELECT_PERM, OP_GROUP_ERROR, OP_QUANT_WEIGHT, OP_GEMM, OP_OUTPUT_ERROR = 1, 2, 3, 4, 5, 6
 CHUNK_ROWS = 16
 KIND_NVFP4, KIND_INT = 0, 1
 
@@ -39,6 +39,8 @@ _SIGNATURES = {
     "pq_workspace_bytes": (_sz, [_int, _i64, _i64, _i64, _int]),
     "pq_sf_bytes": (_sz, [_i64, _i64, _int]),
     "pq_calib_stats": (_int, [_vp, _i64, _i64, _i64, _vp, _vp, _vp, _sz, _vp]),
+    "pq_quant_act_nvfp4_perm": (_int, [_vp, _i64, _i64, _i64, _vp, _vp, _vp, _vp, _int, _vp]),
+    "pq_output_error": (_int, [_vp, _i64, _vp, _i64, _i64, _i64, _vp, _vp, _sz, _vp]),
     "pq_calib_stats_static": (_int, [_vp, _i64, _i64, _i64, _vp, _vp, _vp]),
     "pq_calib_stats_static_max_bytes": (_sz, []),
     "pq_tensor_scale": (_int, [_vp, _i64, _vp, _vp]),
@@ -142,6 +144,16 @@ def pq_calib_stats(T, sumsq, amax, ws):
                                                   _p(amax), w, wb, _stream()))
 
 
+def pq_output_error(Yref, Yq, err, ws):
+    """err[n] += sum over rows of (Yref - Yq)^2: Yref fp32 [rows, N], Yq bf16 [rows, N], err fp64 [N]."""
+    _bf16(Yq)
+    assert Yref.dtype == torch.float32 and Yref.dim() == 2 and Yref.stride(1) == 1 and Yref.shape == Yq.shape
+    assert err.dtype == torch.float64 and err.numel() == Yq.shape[1]
+    w, wb = _ws(ws)
+    _check("pq_output_error", lib().pq_output_error(_p(Yref), Yref.stride(0), _p(Yq), Yq.stride(0), Yq.shape[0],
+                                                    Yq.shape[1], _p(err), w, wb, _stream()))
+
+
 def pq_calib_stats_static(T, sumsq, amax):
     """pq_calib_stats without a workspace argument: for callers that may not allocate device
     memory, the partial sums live in a fixed 8 MiB array inside the library (one per GPU).  Raises
@@ -208,6 +220,16 @@ def pq_quant_act_nvfp4(X, ts_x, codes, sf, sf_layout):
     assert codes.dtype == torch.uint8 and sf.dtype == torch.uint8 and ts_x.dtype == torch.float32
     _check("pq_quant_act_nvfp4", lib().pq_quant_act_nvfp4(_p(X), X.shape[0], X.shape[1], X.stride(0), _p(ts_x),
                                                           _p(codes), _p(sf), sf_layout, _stream()))
+
+
+def pq_quant_act_nvfp4_perm(X, perm, ts_x, codes, sf, sf_layout):
+    """Codes and scales of X with its channels taken in the order `perm` (int32 [K], or None)."""
+    _bf16(X)
+    assert codes.dtype == torch.uint8 and sf.dtype == torch.uint8 and ts_x.dtype == torch.float32
+    assert perm is None or (perm.dtype == torch.int32 and perm.numel() == X.shape[1] and perm.is_contiguous())
+    _check("pq_quant_act_nvfp4_perm", lib().pq_quant_act_nvfp4_perm(_p(X), X.shape[0], X.shape[1], X.stride(0),
+                                                                    _p(perm), _p(ts_x), _p(codes), _p(sf),
+                                                                    sf_layout, _stream()))
 
 
 def pq_gemm_w4a4(xq, sfx, ts_x, wq, sfw, ts_w, Y, ws):

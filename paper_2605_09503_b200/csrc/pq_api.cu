@@ -46,6 +46,7 @@ extern "C" size_t pq_workspace_bytes(int op, int64_t rows, int64_t K, int64_t N,
         }
         case PQ_OP_QUANT_WEIGHT: return 256;
         case PQ_OP_GEMM: return 256;
+        case PQ_OP_OUTPUT_ERROR: return round256(static_cast<size_t>(slabs) * K * sizeof(double));
         default: return 0;
     }
 }

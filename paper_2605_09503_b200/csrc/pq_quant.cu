@@ -342,6 +342,40 @@ extern "C" pq_status pq_quant_act_nvfp4(const void *X, int64_t M, int64_t K, int
     return pq_quant_act_nvfp4_shaped(X, M, K, ld, ts_x, codes, sf, sf_layout, 0, stream);
 }
 
+// Gather by an order (a row of the candidate table, or the one `select` names) and quantize with
+// the tensor scale at ts.
+static pq_status launch_gather(const uint16_t *w, int64_t N, int64_t K, int64_t ld, const int32_t *perm,
+                               const int32_t *perm_select, const float *ts, uint8_t *codes, uint8_t *sf,
+                               int sf_layout, cudaStream_t st) {
+    const size_t smem = static_cast<size_t>(K) * 2;
+    const int grid = static_cast<int>(N < 148 * 8 ? N : 148 * 8);
+    if (sf_layout == PQ_SF_TCGEN05) {
+        const int64_t rows_pad = pq_ceil_div(N, 128) * 128;
+        if (rows_pad > N) sf_zero_pad_kernel<<<64, 256, 0, st>>>(sf, N, rows_pad, K);
+        if (allow_smem(quant_nvfp4_gather_kernel<PQ_SF_TCGEN05>, smem) != PQ_OK) return PQ_ERR_CUDA;
+        quant_nvfp4_gather_kernel<PQ_SF_TCGEN05><<<grid, kQuantThreads, smem, st>>>(
+            w, N, K, ld, perm, perm_select, ts, codes, sf);
+    } else {
+        if (allow_smem(quant_nvfp4_gather_kernel<PQ_SF_LINEAR>, smem) != PQ_OK) return PQ_ERR_CUDA;
+        quant_nvfp4_gather_kernel<PQ_SF_LINEAR><<<grid, kQuantThreads, smem, st>>>(
+            w, N, K, ld, perm, perm_select, ts, codes, sf);
+    }
+    return pq_launch_status();
+}
+
+extern "C" pq_status pq_quant_act_nvfp4_perm(const void *X, int64_t M, int64_t K, int64_t ld, const int32_t *perm,
+                                             const float *ts_x, uint8_t *codes, uint8_t *sf, int sf_layout,
+                                             void *stream) {
+    if (!perm) return pq_quant_act_nvfp4(X, M, K, ld, ts_x, codes, sf, sf_layout, stream);
+    PQ_REQUIRE(X && ts_x && codes && sf, PQ_ERR_NULL);
+    PQ_REQUIRE(sf_layout == PQ_SF_LINEAR || sf_layout == PQ_SF_TCGEN05, PQ_ERR_FORMAT);
+    PQ_REQUIRE(M > 0 && K > 0 && K % 16 == 0 && K <= 16384 && ld >= K, PQ_ERR_SHAPE);
+    PQ_REQUIRE(sf_layout == PQ_SF_LINEAR || K % 64 == 0, PQ_ERR_SHAPE);
+    PQ_REQUIRE(pq_aligned16(X) && ld % 8 == 0 && pq_aligned16(codes) && pq_aligned16(sf), PQ_ERR_ALIGN);
+    return launch_gather(static_cast<const uint16_t *>(X), M, K, ld, perm, nullptr, ts_x, codes, sf, sf_layout,
+                         static_cast<cudaStream_t>(stream));
+}
+
 extern "C" pq_status pq_quant_weight(const void *Wt, int64_t N, int64_t K, int64_t ld,
                                      const int32_t *perm, const int32_t *perm_select, uint8_t *codes,
                                      uint8_t *sf, int sf_layout, float *ts_w, void *ws, size_t ws_bytes,
@@ -370,20 +404,7 @@ extern "C" pq_status pq_quant_weight(const void *Wt, int64_t N, int64_t K, int64
     weight_scale_kernel<<<1, 1, 0, st>>>(amax_bits, ts_w);
     if (!perm) return pq_quant_act_nvfp4(Wt, N, K, ld, ts_w, codes, sf, sf_layout, stream);
 
-    const size_t smem = static_cast<size_t>(K) * 2;
-    const int grid = static_cast<int>(N < 148 * 8 ? N : 148 * 8);
-    if (sf_layout == PQ_SF_TCGEN05) {
-        const int64_t rows_pad = pq_ceil_div(N, 128) * 128;
-        if (rows_pad > N) sf_zero_pad_kernel<<<64, 256, 0, st>>>(sf, N, rows_pad, K);
-        if (allow_smem(quant_nvfp4_gather_kernel<PQ_SF_TCGEN05>, smem) != PQ_OK) return PQ_ERR_CUDA;
-        quant_nvfp4_gather_kernel<PQ_SF_TCGEN05><<<grid, kQuantThreads, smem, st>>>(
-            w, N, K, ld, perm, perm_select, ts_w, codes, sf);
-    } else {
-        if (allow_smem(quant_nvfp4_gather_kernel<PQ_SF_LINEAR>, smem) != PQ_OK) return PQ_ERR_CUDA;
-        quant_nvfp4_gather_kernel<PQ_SF_LINEAR><<<grid, kQuantThreads, smem, st>>>(
-            w, N, K, ld, perm, perm_select, ts_w, codes, sf);
-    }
-    return pq_launch_status();
+    return launch_gather(w, N, K, ld, perm, perm_select, ts_w, codes, sf, sf_layout, st);
 }
 
 extern "C" pq_status pq_fakequant_int(const void *T, int64_t rows, int64_t K, int64_t ld, pq_format fmt,

@@ -81,6 +81,72 @@ calib_stats_slab(const uint16_t *__restrict__ T, int64_t rows, int64_t K, int64_
     }
 }
 
+// Output-side calibration error: the same slab / chunk walk over the fp32 difference of two
+// tensors (fp32 reference, bf16 quantized-layer output): 6 bytes per element, streaming.  A lane
+// owns 8 adjacent columns; eight rows (two 16-byte loads of the reference and one of the output per
+// row) are in flight at a time, the rows of a chunk are added in order.
+constexpr int kDiffRows = 8;
+
+__device__ __forceinline__ void diff_row(const float4 &r0, const float4 &r1, const uint4 &q, float (&s)[8]) {
+    float y[8];
+    pq::unpack8(q, y);
+    const float ref[8] = {r0.x, r0.y, r0.z, r0.w, r1.x, r1.y, r1.z, r1.w};
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        const float d = __fsub_rn(ref[i], y[i]);
+        s[i] = __fmaf_rn(d, d, s[i]);
+    }
+}
+
+__global__ void __launch_bounds__(kStatsThreads)
+output_error_slab(const float *__restrict__ Yref, int64_t ld_ref, const uint16_t *__restrict__ Yq, int64_t ld_q,
+                  int64_t rows, int64_t N, double *__restrict__ slab_sum /*[slabs, N]*/) {
+    __shared__ __align__(16) float sum_s[kSlabChunks][kStatsCols];
+    pq::dependents_may_launch();
+    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+    const int64_t col0 = static_cast<int64_t>(blockIdx.y) * kStatsCols;
+    const int64_t col = col0 + lane * 8;
+    const int64_t slab = blockIdx.x;
+    const int64_t r0 = slab * PQ_SLAB_ROWS + w * PQ_CHUNK_ROWS;
+    const int64_t left = rows - r0;
+    const int n = left >= PQ_CHUNK_ROWS ? PQ_CHUNK_ROWS : (left > 0 ? static_cast<int>(left) : 0);
+
+    float s[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) s[i] = 0.0f;
+    if (col < N) {
+        const float *pr = Yref + r0 * ld_ref + col;
+        const uint16_t *yq_row = Yq + r0 * ld_q + col;
+        for (int t0 = 0; t0 < n; t0 += kDiffRows) {
+            float4 a[kDiffRows], b[kDiffRows];
+            uint4 q[kDiffRows];
+#pragma unroll
+            for (int u = 0; u < kDiffRows; ++u) {
+                if (t0 + u < n) {
+                    const float4 *src = reinterpret_cast<const float4 *>(pr + static_cast<int64_t>(t0 + u) * ld_ref);
+                    a[u] = __ldcs(src), b[u] = __ldcs(src + 1);
+                    q[u] = __ldcs(reinterpret_cast<const uint4 *>(yq_row + static_cast<int64_t>(t0 + u) * ld_q));
+                }
+            }
+#pragma unroll
+            for (int u = 0; u < kDiffRows; ++u)
+                if (t0 + u < n) diff_row(a[u], b[u], q[u], s);
+        }
+    }
+    float4 *ds = reinterpret_cast<float4 *>(&sum_s[w][lane * 8]);
+    ds[0] = make_float4(s[0], s[1], s[2], s[3]);
+    ds[1] = make_float4(s[4], s[5], s[6], s[7]);
+    __syncthreads();
+    // one thread per column: the slab's chunk partials in chunk order, from zero
+    const int c = threadIdx.x;
+    if (col0 + c < N) {
+        double acc = 0.0;
+#pragma unroll
+        for (int k = 0; k < kSlabChunks; ++k) acc = __dadd_rn(acc, static_cast<double>(sum_s[k][c]));
+        slab_sum[slab * N + col0 + c] = acc;
+    }
+}
+
 __global__ void tensor_scale_kernel(const float *__restrict__ amax, int64_t K, float *ts) {
     __shared__ float red[32];
     float a = 0.0f;
@@ -122,6 +188,25 @@ extern "C" pq_status pq_calib_stats(const void *T, int64_t rows, int64_t K, int6
     float *slab_max = reinterpret_cast<float *>(slab_sum + slabs * K);
     calib_stats_slab<<<grid, kStatsThreads, 0, st>>>(static_cast<const uint16_t *>(T), rows, K, ld, slab_sum, slab_max);
     PQ_CUDA_OK((pq::launch_fold<double, 1, true>(slab_sum, slab_max, slabs, K, sumsq, amax, st)));
+    return pq_launch_status();
+}
+
+extern "C" pq_status pq_output_error(const float *Yref, int64_t ld_ref, const void *Yq, int64_t ld_q, int64_t rows,
+                                     int64_t N, double *err, void *ws, size_t ws_bytes, void *stream) {
+    PQ_REQUIRE(Yref && Yq && err, PQ_ERR_NULL);
+    PQ_REQUIRE(rows > 0 && N > 0 && N % 8 == 0 && ld_ref >= N && ld_q >= N, PQ_ERR_SHAPE);
+    PQ_REQUIRE(pq_aligned16(Yref) && ld_ref % 4 == 0 && pq_aligned16(Yq) && ld_q % 8 == 0, PQ_ERR_ALIGN);
+    const size_t need = pq_workspace_bytes(PQ_OP_OUTPUT_ERROR, rows, N, 0, 0);
+    PQ_REQUIRE(ws && ws_bytes >= need, PQ_ERR_WORKSPACE);
+    PQ_REQUIRE(pq_aligned256(ws), PQ_ERR_ALIGN);
+    const int64_t slabs = pq_ceil_div(rows, PQ_SLAB_ROWS);
+    PQ_REQUIRE(slabs < (1ll << 31) && N <= 65535ll * kStatsCols, PQ_ERR_SHAPE);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    dim3 grid(static_cast<unsigned>(slabs), static_cast<unsigned>(pq_ceil_div(N, kStatsCols)));
+    double *slab_sum = static_cast<double *>(ws);
+    output_error_slab<<<grid, kStatsThreads, 0, st>>>(Yref, ld_ref, static_cast<const uint16_t *>(Yq), ld_q, rows, N,
+                                                      slab_sum);
+    PQ_CUDA_OK((pq::launch_fold<double, 1, false>(slab_sum, nullptr, slabs, N, err, nullptr, st)));
     return pq_launch_status();
 }
 

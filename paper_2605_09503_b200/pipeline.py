@@ -89,6 +89,40 @@ def calibrate(batches, Wt, fmt=NVFP4, J=5, tau=0.0, sf_layout=B.PQ_SF_TCGEN05) -
     return Calibration(sumsq_a, sumsq_w, amax_a, ts_x, ts_w, perms, err_x, err_w, lam, E, select, wq, sfw, rows_a)
 
 
+def select_by_output_error(batches, refs, Wt, perms, ts_x, tau=0.0):
+    """The acceptance rule of Eq. 10 with E read on the layer's output (Sec. 3.3): for the original
+    order and every candidate row of `perms` (int32 [P, K]) quantize W and the calibration batches in
+    that order, run the W4A4 GEMM and accumulate the squared distance to the unquantized outputs
+    `refs` (fp32 [T, N] per batch, from any GEMM the caller trusts).  Returns (E fp64 [P+1], select
+    int32 [2] = {best, accept}), both on the device; `select` is what pq_quant_weight consumes."""
+    dev = Wt.device
+    N, K = Wt.shape
+    P = perms.shape[0]
+    max_rows = max(b.shape[0] for b in batches)
+    err = torch.zeros(P + 1, N, dtype=torch.float64, device=dev)
+    wq = torch.empty(N, K // 2, dtype=torch.uint8, device=dev)
+    sfw = torch.empty(B.sf_bytes(N, K, B.PQ_SF_TCGEN05), dtype=torch.uint8, device=dev)
+    ts_w = torch.empty(1, dtype=torch.float32, device=dev)
+    xq = torch.empty(max_rows, K // 2, dtype=torch.uint8, device=dev)
+    sfx = torch.empty(B.sf_bytes(max_rows, K, B.PQ_SF_TCGEN05), dtype=torch.uint8, device=dev)
+    Y = torch.empty(max_rows, N, dtype=torch.bfloat16, device=dev)
+    ws_w = B.workspace(B.OP_QUANT_WEIGHT, N, K)
+    ws_g = B.workspace(B.OP_GEMM, max_rows, K, N)
+    ws_e = B.workspace(B.OP_OUTPUT_ERROR, max_rows, N)
+    for p in range(P + 1):
+        order = None if p == 0 else perms[p - 1]
+        B.pq_quant_weight(Wt, order, None, wq, sfw, B.PQ_SF_TCGEN05, ts_w, ws_w)
+        for x, ref in zip(batches, refs):
+            T = x.shape[0]
+            B.pq_quant_act_nvfp4_perm(x, order, ts_x, xq[:T], sfx, B.PQ_SF_TCGEN05)
+            B.pq_gemm_w4a4(xq[:T], sfx, ts_x, wq, sfw, ts_w, Y[:T], ws_g)
+            B.pq_output_error(ref, Y[:T], err[p], ws_e)
+    select = torch.zeros(2, dtype=torch.int32, device=dev)
+    E = torch.empty(P + 1, dtype=torch.float64, device=dev)
+    B.pq_accept(err, torch.zeros_like(err), None, tau, select[0:1], select[1:2], E)
+    return E, select
+
+
 class QuantLinear:
     """Runtime half: holds the quantized weight and the intermediates of one layer."""
 
