@@ -473,6 +473,19 @@ def run_ours(args):
                                                                             ws_qw), max(5, it // 4)),
               2 * N * K * 2 + N * K // 2 + N * K // 16, note="two reads of W (absmax, then gather + quantize)")
 
+        # output-side calibration error: fp32 reference and bf16 layer output of one batch (6 B per element)
+        yrefs = [torch.randn(M, N, device=dev) for _ in range(2)]
+        yqs = [(r * 1.01).to(torch.bfloat16) for r in yrefs]
+        eo = torch.zeros(N, dtype=torch.float64, device=dev)
+        ws_oe = B.workspace(B.OP_OUTPUT_ERROR, M, N)
+        stage("output_error", graph_loop(torch, lambda i: B.pq_output_error(yrefs[i % 2], yqs[i % 2], eo, ws_oe), it),
+              M * N * 6)
+        stage("quant_act_nvfp4_candidate_order",
+              graph_loop(torch, lambda i: B.pq_quant_act_nvfp4_perm(xs[i % XROT], order, cal.ts_x, xq_rot[i % XROT],
+                                                                    sfx_rot[i % XROT], B.PQ_SF_TCGEN05), it),
+              quant_bytes, note="calibration-time gather quantizer, one block per row")
+        del yrefs, yqs
+
     # ---- end to end: host tensors in, host tensor out, through the C ABI
     xh = [x.pin_memory() for x in xs_host[:2]]
     yh = [torch.empty(M, N, dtype=torch.bfloat16).pin_memory() for _ in range(2)]

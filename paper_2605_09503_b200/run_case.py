@@ -14,7 +14,7 @@ import torch
 
 from . import binding as B
 
-CASES = ["probe", "norm_quant", "gemm", "quant", "linear", "batched", "stats", "error", "error_perm", "fakequant", "fakequant_perm", "quant_weight",
+CASES = ["probe", "output_error", "norm_quant", "gemm", "quant", "linear", "batched", "stats", "error", "error_perm", "fakequant", "fakequant_perm", "quant_weight",
          "quant_weight_perm", "select_perm"]
 
 
@@ -135,6 +135,13 @@ def main():
         sfx = [torch.empty(B.sf_bytes(M, K, 1), dtype=torch.uint8, device=dev) for _ in range(R)]
         bytes_moved = M * K * 2 + M * K // 2 + M * K // 16
         fn = lambda i: B.pq_quant_act_nvfp4(X[i % R], ts, xq[i % R], sfx[i % R], B.PQ_SF_TCGEN05)
+    elif args.case == "output_error":
+        yref = [torch.randn(M, N, device=dev, generator=g) for _ in range(2)]
+        yq = [(r * 1.01).to(torch.bfloat16) for r in yref]
+        eo = torch.zeros(N, dtype=torch.float64, device=dev)
+        ws = B.workspace(B.OP_OUTPUT_ERROR, M, N)
+        bytes_moved = M * N * 6
+        fn = lambda i: B.pq_output_error(yref[i % 2], yq[i % 2], eo, ws)
     elif args.case == "stats":
         X = [acts(M) for _ in range(R)]
         S = torch.zeros(K, dtype=torch.float64, device=dev)
