@@ -181,11 +181,16 @@ __device__ __forceinline__ float run_sse(const float (&x)[8], const float (&q)[8
 // {0x0000, 0x3F00, 0x3F80, 0x3FC0, 0x4000, 0x4040, 0x4080, 0x40C0}; prmt picks the high and low
 // bytes with the four codes of a 16-bit half as selectors, a second prmt interleaves them into
 // bf16 pairs, and a bf16 widens to fp32 by a shift.
+__device__ __forceinline__ void e2m1_levels(uint32_t codes, float (&q)[8]);
 __device__ __forceinline__ void nvfp4_levels_abs(const float (&x)[8], float r, float (&q)[8]) {
     float y[8];
 #pragma unroll
     for (int i = 0; i < 8; ++i) y[i] = __fmul_rn(fabsf(x[i]), r);
-    const uint32_t codes = f32x8_to_e2m1(y);
+    e2m1_levels(f32x8_to_e2m1(y), q);
+}
+
+// Eight E2M1 codes of non-negative values -> their fp32 magnitudes (the byte tables above).
+__device__ __forceinline__ void e2m1_levels(uint32_t codes, float (&q)[8]) {
 #pragma unroll
     for (int h = 0; h < 2; ++h) {
         const uint32_t sel = h ? codes >> 16 : codes & 0xFFFFu;

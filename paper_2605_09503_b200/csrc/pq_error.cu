@@ -52,27 +52,92 @@ __device__ __forceinline__ void build_scale_table(float2 *table, float ts) {
     }
 }
 
+// Two fp32 lanes in one 64-bit register and the packed IEEE operations on them: one issue slot
+// for two results, each rounded exactly like the scalar instruction.
+__device__ __forceinline__ uint64_t pack2(float lo, float hi) {
+    uint64_t r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+    return r;
+}
+__device__ __forceinline__ void unpack2(uint64_t v, float &lo, float &hi) {
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ uint64_t mul2(uint64_t a, uint64_t b) {
+    uint64_t r;
+    asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+    return r;
+}
+__device__ __forceinline__ uint64_t fma2(uint64_t a, uint64_t b, uint64_t c) {
+    uint64_t r;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r) : "l"(a), "l"(b), "l"(c));
+    return r;
+}
+
+__device__ __forceinline__ uint64_t add2(uint64_t a, uint64_t b) {
+    uint64_t r;
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+    return r;
+}
+
 // Error of one row's 16 channels held by this lane; TEAM16 = group / 16 adjacent lanes share a group.
-// c6 = 6 * ts (NVFP4 only).
+// c6 = 6 * ts (NVFP4 only).  The lane's two 8-channel runs are carried side by side in packed
+// registers: per run the operations and their order are those of the scalar definition (scale the
+// magnitude by the reciprocal, round to a level, residual by one fused multiply-add, squares added in
+// channel order), two results per instruction.  Magnitudes are taken on the bf16 pairs, which is exact.
 template <int KIND, int TEAM16>
 __device__ __forceinline__ float row_sse16(const uint4 &lo, const uint4 &hi, float c6, const float2 *table, float Qf) {
+    const uint32_t m = 0x7FFF7FFFu;
     float xa[8], xb[8];
-    pq::unpack8(lo, xa);
-    pq::unpack8(hi, xb);
-    const float amax = pq::team_max<TEAM16>(fmaxf(pq::absmax8(xa), pq::absmax8(xb)));
-    float qa[8], qb[8], d, r;
+    pq::unpack8(make_uint4(lo.x & m, lo.y & m, lo.z & m, lo.w & m), xa);
+    pq::unpack8(make_uint4(hi.x & m, hi.y & m, hi.z & m, hi.w & m), xb);
+    float amax = 0.0f;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) amax = fmaxf(amax, fmaxf(xa[i], xb[i]));
+    amax = pq::team_max<TEAM16>(amax);
+    float d, r;
     if (KIND == 0) {
         const float2 dr = table[pq::f32_to_e4m3(__fdiv_rn(amax, c6))];
         d = dr.x, r = dr.y;
-        pq::nvfp4_levels_abs(xa, r, qa);
-        pq::nvfp4_levels_abs(xb, r, qb);
     } else {
         pq::int_scale(amax, Qf, d, r);
-        pq::int_levels_abs(xa, r, Qf, qa);
-        pq::int_levels_abs(xb, r, Qf, qb);
     }
+    const uint64_t r2 = pack2(r, r), nd2 = pack2(-d, -d);
+    uint64_t x2[8], q2[8];
+    if (KIND == 0) {
+        float ya[8], yb[8], qa[8], qb[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            x2[i] = pack2(xa[i], xb[i]);
+            unpack2(mul2(x2[i], r2), ya[i], yb[i]);
+        }
+        pq::e2m1_levels(pq::f32x8_to_e2m1(ya), qa);
+        pq::e2m1_levels(pq::f32x8_to_e2m1(yb), qb);
+#pragma unroll
+        for (int i = 0; i < 8; ++i) q2[i] = pack2(qa[i], qb[i]);
+    } else {
+        // min(rint(y), Q): adding and subtracting 1.5 * 2^23 rounds like rint for y < 2^22, beyond that the clamp decides
+        // (the first addition is written as y * 1 + magic: a packed multiply directly followed by a packed
+        // add was seen to come out as one fused operation, which rounds once instead of twice)
+        const uint64_t magic = pack2(12582912.0f, 12582912.0f), unmagic = pack2(-12582912.0f, -12582912.0f);
+        const uint64_t one2 = pack2(1.0f, 1.0f);
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            x2[i] = pack2(xa[i], xb[i]);
+            float za, zb;
+            unpack2(add2(fma2(mul2(x2[i], r2), one2, magic), unmagic), za, zb);
+            q2[i] = pack2(fminf(za, Qf), fminf(zb, Qf));
+        }
+    }
+    uint64_t acc2 = pack2(0.0f, 0.0f);
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        const uint64_t delta = fma2(q2[i], nd2, x2[i]);
+        acc2 = fma2(delta, delta, acc2);
+    }
+    float sa, sb;
+    unpack2(acc2, sa, sb);
     // runs of 8 channels, then the balanced adjacent-pair tree: its first level is this lane's two runs
-    return pq::team_sum<TEAM16>(__fadd_rn(pq::run_sse_abs(xa, qa, d), pq::run_sse_abs(xb, qb, d)));
+    return pq::team_sum<TEAM16>(__fadd_rn(sa, sb));
 }
 
 constexpr int kSlabChunks = PQ_SLAB_ROWS / PQ_CHUNK_ROWS;  // 8

@@ -21,10 +21,10 @@
 //                boxes in swizzled shared memory and write them with TMA stores (full 128-byte
 //                lines) while the next tile's main loop runs.
 //   warps 10..17 scale-factor stagers: read the stage's scale blocks from shared memory and write
-//                them into one of four scale slots in tensor memory with tcgen05.st (one warp per
+//                them into one of two scale slots in tensor memory with tcgen05.st (one warp per
 //                lane quadrant; two sets of four warps take alternate K iterations).
 // 256 divides every FLUX output width (3072, 9216, 12288).  The 512 tensor-memory columns hold one
-// 256-column accumulator plus four scale slots (4 x 48); the epilogue warps pull the accumulator
+// 256-column accumulator plus two scale slots (2 x 48); the epilogue warps pull the accumulator
 // into registers as packed bf16 within a few hundred cycles and store it from there.
 //
 // Measurements on B200 behind these choices:
@@ -72,9 +72,14 @@ constexpr int kEpiBytes = kEpiWarps * kEpiBox;      // one staging box per epilo
 constexpr int kFirstStager = 2 + kEpiWarps;
 constexpr int kThreads = 32 * (kFirstStager + 8);   // producer, MMA issuer, 8 epilogue and 8 stager warps
 constexpr int kTmemCols = 512;
-// One 256-column accumulator, then four scale slots.  A slot holds the scales of one stage: per
+// One 256-column accumulator, then two scale slots, one per stager set (a set always writes the same
+// slot, and only after the MMAs that read it two iterations earlier have completed).  With four slots,
+// i.e. stagers running up to four stages ahead of the tensor pipe with both sets writing at once, about
+// one launch in 450 of the 4608 x 3072 x 9216 product came out with the rows of a lane quadrant of some
+// tiles wrong (off as if part of K had met other scale factors); two slots cost nothing (the stage time is bounded by operand
+// delivery) and 18000 launches were clean.  A slot holds the scales of one stage: per
 // 64-channel K block 4 columns of A scales (128 rows) and 8 columns of B scales (256 rows).
-constexpr int kSfSlots = 4;
+constexpr int kSfSlots = 2;
 constexpr uint32_t kSfSlotCol0 = BN, kSfSlotCols = 4 * (4 + 8), kSfbOfs = 16;
 static_assert(kSfSlotCol0 + kSfSlots * kSfSlotCols <= 512, "tensor memory columns");
 constexpr long long kWaitCycles = 4000000000ll;  // about two seconds of SM clock per wait
@@ -256,7 +261,17 @@ __device__ __forceinline__ void tc_ld16(uint32_t taddr, uint32_t (&v)[16]) {
         : "r"(taddr)
         : "memory");
 }
-__device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+// The registers of a tcgen05.ld hold its result only after tcgen05.wait::ld.  The wait names them as
+// in/out operands: whatever reads them afterwards then depends on the wait and cannot be scheduled in
+// front of it (arithmetic on the loaded values has no other tie to the wait instruction; without it a
+// tile was occasionally packed from registers the load had not written yet).
+__device__ __forceinline__ void tc_wait_ld(uint32_t (&v)[16]) {
+    asm volatile("tcgen05.wait::ld.sync.aligned;"
+                 : "+r"(v[0]), "+r"(v[1]), "+r"(v[2]), "+r"(v[3]), "+r"(v[4]), "+r"(v[5]), "+r"(v[6]), "+r"(v[7]),
+                   "+r"(v[8]), "+r"(v[9]), "+r"(v[10]), "+r"(v[11]), "+r"(v[12]), "+r"(v[13]), "+r"(v[14]), "+r"(v[15])
+                 :
+                 : "memory");
+}
 __device__ __forceinline__ void tc_st4(uint32_t taddr, const uint4 &v) {
     asm volatile("tcgen05.st.sync.aligned.32x32b.x4.b32 [%0], {%1, %2, %3, %4};" ::"r"(taddr), "r"(v.x), "r"(v.y),
                  "r"(v.z), "r"(v.w)
@@ -471,7 +486,7 @@ gemm_w4a4_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
                 if ((it & 1u) != set) continue;
                 const int s = it % kStages;
                 const uint32_t t = it % kSfSlots;
-                // the stage's scale blocks have landed, and the MMAs that read this slot three
+                // the stage's scale blocks have landed, and the MMAs that read this slot kSfSlots
                 // iterations ago have completed (their commit released that iteration's stage)
                 if (!mbar_wait(sf_ready_bar(s), (it / kStages) & 1u, abort_flag, p.status)) {
                     ok = false;
@@ -544,11 +559,11 @@ gemm_w4a4_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
             tc_ld16(acc, va);
 #pragma unroll
             for (int c = 0; c < 8; c += 2) {
-                tc_wait_ld();
+                tc_wait_ld(va);
                 tc_ld16(acc + (c + 1) * 16, vb);
 #pragma unroll
                 for (int i = 0; i < 8; ++i) pk[8 * c + i] = pack_bf16(va[2 * i], va[2 * i + 1], alpha);
-                tc_wait_ld();
+                tc_wait_ld(vb);
                 if (c + 2 < 8) tc_ld16(acc + (c + 2) * 16, va);
 #pragma unroll
                 for (int i = 0; i < 8; ++i) pk[8 * (c + 1) + i] = pack_bf16(vb[2 * i], vb[2 * i + 1], alpha);

@@ -132,3 +132,24 @@ def test_full_size_batched_equals_serial():
     layer.check()
     for y, r in zip(ys, ref):
         assert torch.equal(y.view(torch.int16), r.view(torch.int16))
+
+
+def test_repeated_launches_give_the_same_bits():
+    """The same product 1200 times, serial and batched: every launch must reproduce the first one
+    bit for bit (a rare ordering fault inside the kernel shows up as a few wrong 32-row blocks in one
+    launch out of several hundred, which a single comparison against the oracle does not catch)."""
+    cfg = inputs.CONFIGS["qkv"]
+    w, wq, sfw, ts_w = _weights(cfg)
+    xs = [inputs.activations(cfg, 0, 2000 + i).to(DEV) for i in range(4)]
+    ts_x = torch.tensor([0.3], dtype=torch.float32, device=DEV)
+    layer = pipeline.QuantLinear(wq, sfw, ts_w, ts_x, cfg.M)
+    ref = [layer(x).clone() for x in xs]
+    ys = [torch.zeros(cfg.M, cfg.N, dtype=torch.bfloat16, device=DEV) for _ in xs]
+    wrong = 0
+    for rep in range(150):
+        layer.forward_batches(xs, ys, n_sets=4)
+        wrong += sum(int(not torch.equal(y.view(torch.int16), r.view(torch.int16))) for y, r in zip(ys, ref))
+        for x, r in zip(xs, ref):
+            wrong += int(not torch.equal(layer(x).view(torch.int16), r.view(torch.int16)))
+    layer.check()
+    assert wrong == 0
