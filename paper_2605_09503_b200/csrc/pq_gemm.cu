@@ -77,7 +77,7 @@ constexpr int kTmemCols = 512;
 // i.e. stagers running up to four stages ahead of the tensor pipe with both sets writing at once, about
 // one launch in 450 of the 4608 x 3072 x 9216 product came out with the rows of a lane quadrant of some
 // tiles wrong (off as if part of K had met other scale factors); two slots cost nothing (the stage time is bounded by operand
-// delivery) and 18000 launches were clean.  A slot holds the scales of one stage: per
+// delivery) and 36000 launches were clean (so were three slots, in either column range).  A slot holds the scales of one stage: per
 // 64-channel K block 4 columns of A scales (128 rows) and 8 columns of B scales (256 rows).
 constexpr int kSfSlots = 2;
 constexpr uint32_t kSfSlotCol0 = BN, kSfSlotCols = 4 * (4 + 8), kSfbOfs = 16;
