@@ -1,0 +1,89 @@
+"""Every entry point launched many times on the same inputs must reproduce its first result bit for
+bit: a timing-dependent ordering fault between the warps of a kernel, or between a kernel and its
+programmatic dependent, shows up as an occasional deviating launch that a single comparison against
+the oracle does not catch."""
+import pytest
+import torch
+
+from paper_2605_09503_b200 import binding as B, inputs, pipeline
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda"
+REPS = 100
+
+
+def _same(a, b):
+    va = a.view(torch.int64) if a.dtype == torch.float64 else a.contiguous().view(torch.uint8)
+    vb = b.view(torch.int64) if b.dtype == torch.float64 else b.contiguous().view(torch.uint8)
+    return torch.equal(va, vb)
+
+
+def _repeat(fn, outs, reps=REPS):
+    fn()
+    ref = [o.clone() for o in outs]
+    deviating = 0
+    for _ in range(reps):
+        for o in outs:
+            o.fill_(0xEE) if o.dtype == torch.uint8 else o.zero_()
+        fn()
+        deviating += int(not all(_same(o, r) for o, r in zip(outs, ref)))
+    torch.cuda.synchronize()
+    return deviating
+
+
+def test_streaming_entry_points_repeat_bit_for_bit():
+    cfg = inputs.CONFIGS["qkv"]
+    M, K = 2048 + 40, cfg.K
+    x = inputs.activations(cfg, 0, 77, rows=M).to(DEV)
+    g = torch.Generator(device=DEV)
+    g.manual_seed(3)
+    perms = torch.stack([torch.randperm(K, device=DEV, generator=g) for _ in range(3)]).to(torch.int32)
+    ts = torch.tensor([0.3], dtype=torch.float32, device=DEV)
+
+    S = torch.zeros(K, dtype=torch.float64, device=DEV)
+    A = torch.zeros(K, dtype=torch.float32, device=DEV)
+    ws = B.workspace(B.OP_CALIB_STATS, M, K)
+    assert _repeat(lambda: B.pq_calib_stats(x, S, A, ws), [S, A]) == 0
+
+    wse = B.workspace(B.OP_GROUP_ERROR, M, K, 0, 3)
+    e1 = torch.zeros(1, K // 16, dtype=torch.float64, device=DEV)
+    assert _repeat(lambda: B.pq_group_error(x, pipeline.NVFP4, ts, None, e1, wse), [e1]) == 0
+    e2 = torch.zeros(1, K // 64, dtype=torch.float64, device=DEV)
+    assert _repeat(lambda: B.pq_group_error(x, (B.KIND_INT, 8, 64), None, None, e2, wse), [e2]) == 0
+    e3 = torch.zeros(3, K // 16, dtype=torch.float64, device=DEV)
+    assert _repeat(lambda: B.pq_group_error(x, pipeline.NVFP4, ts, perms, e3, wse), [e3], reps=20) == 0
+
+    xq = torch.empty(M, K // 2, dtype=torch.uint8, device=DEV)
+    sfx = torch.empty(B.sf_bytes(M, K, B.PQ_SF_TCGEN05), dtype=torch.uint8, device=DEV)
+    assert _repeat(lambda: B.pq_quant_act_nvfp4(x, ts, xq, sfx, B.PQ_SF_TCGEN05), [xq, sfx]) == 0
+    assert _repeat(lambda: B.pq_quant_act_nvfp4_perm(x, perms[0], ts, xq, sfx, B.PQ_SF_TCGEN05), [xq, sfx]) == 0
+    a = 0.2 * torch.randn(K, device=DEV, generator=g)
+    b = torch.randn(K, device=DEV, generator=g)
+    for kind in (B.NORM_RMS, B.NORM_ADALN):
+        assert _repeat(lambda: B.pq_norm_quant_nvfp4(x, kind, a, b, 1e-6, perms[1], ts, xq, sfx, B.PQ_SF_TCGEN05),
+                       [xq, sfx]) == 0
+    fq = torch.empty(M, K, dtype=torch.bfloat16, device=DEV)
+    assert _repeat(lambda: B.pq_fakequant_int(x, (B.KIND_INT, 4, 64), None, fq), [fq]) == 0
+
+    N = 1024
+    yref = torch.randn(M, N, device=DEV, generator=g)
+    yq = (yref * 1.01).to(torch.bfloat16)
+    eo = torch.zeros(N, dtype=torch.float64, device=DEV)
+    wso = B.workspace(B.OP_OUTPUT_ERROR, M, N)
+    assert _repeat(lambda: B.pq_output_error(yref, yq, eo, wso), [eo]) == 0
+
+
+@pytest.mark.parametrize("m,k,n", [(4608, 12288, 3072), (1000, 3072, 3080)])
+def test_linear_repeats_bit_for_bit_on_long_and_ragged_shapes(m, k, n):
+    g = torch.Generator(device=DEV)
+    g.manual_seed(m + n)
+    X = torch.randn(m, k, device=DEV, generator=g).to(torch.bfloat16)
+    W = (torch.randn(n, k, device=DEV, generator=g) * 0.05).to(torch.bfloat16)
+    wq = torch.empty(n, k // 2, dtype=torch.uint8, device=DEV)
+    sfw = torch.empty(B.sf_bytes(n, k, B.PQ_SF_TCGEN05), dtype=torch.uint8, device=DEV)
+    ts_w = torch.empty(1, dtype=torch.float32, device=DEV)
+    B.pq_quant_weight(W, None, None, wq, sfw, B.PQ_SF_TCGEN05, ts_w, B.workspace(B.OP_QUANT_WEIGHT, n, k))
+    layer = pipeline.QuantLinear(wq, sfw, ts_w, torch.tensor([0.002], dtype=torch.float32, device=DEV), m)
+    out = torch.empty(m, n, dtype=torch.bfloat16, device=DEV)
+    assert _repeat(lambda: layer(X, out), [out], reps=300) == 0
+    layer.check()
