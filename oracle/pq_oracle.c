@@ -282,6 +282,22 @@ int pqo_select_perm(const double *sumsq_a, int64_t rows_a, const double *sumsq_w
     return 0;
 }
 
+/* The absmax criterion of the reordering ablation (Tab. 2(a)): channels by descending absmax,
+ * equal values by ascending channel.  perm[pos] = channel read at position pos. */
+int pqo_order_by_absmax(const float *amax, int64_t K, int32_t *perm) {
+    if (!amax || !perm || K <= 0) return 1;
+    keyed *buf = (keyed *)malloc(sizeof(keyed) * (size_t)K);
+    if (!buf) return 2;
+    for (int64_t i = 0; i < K; ++i) {
+        buf[i].key = (double)amax[i];
+        buf[i].idx = (int32_t)i;
+    }
+    qsort(buf, (size_t)K, sizeof(keyed), keyed_desc);
+    for (int64_t i = 0; i < K; ++i) perm[i] = buf[i].idx;
+    free(buf);
+    return 0;
+}
+
 /* ------------------------------------------------------------------ calibration error */
 
 /* Eq. 3 on one batch: for every candidate order p and group column k,

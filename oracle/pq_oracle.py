@@ -43,6 +43,7 @@ def _declare(L):
     L.pqo_calib_stats.argtypes = [_P, _i64, _i64, _i64, _P, _P]
     L.pqo_select_perm.argtypes = [_P, _i64, _P, _i64, _i64, C.c_int, _P]
     L.pqo_output_error.argtypes = [_P, _i64, _P, _i64, _i64, _i64, _P]
+    L.pqo_order_by_absmax.argtypes = [_P, _i64, _P]
     L.pqo_group_error.argtypes = [_P, _i64, _i64, _i64, C.c_int, C.c_int, C.c_int, C.c_float, _P,
                                   C.c_int, _P]
     L.pqo_accept.argtypes = [_P, C.c_double, _P, C.c_double, C.c_int, _i64, C.c_double, _P, _P, _P]
@@ -158,6 +159,14 @@ def select_perm(sumsq_a, rows_a, sumsq_w, rows_w, J=5):
     _check(lib().pqo_select_perm(_ptr(sumsq_a), rows_a, _ptr(sumsq_w), rows_w, K, J, _ptr(perms)),
            "select_perm")
     return perms
+
+
+def order_by_absmax(amax):
+    """Tab. 2(a) absmax criterion: channels by descending absmax, ties by ascending channel (int32 [K])."""
+    amax = np.ascontiguousarray(amax, dtype=np.float32)
+    perm = np.empty(amax.size, dtype=np.int32)
+    _check(lib().pqo_order_by_absmax(_ptr(amax), amax.size, _ptr(perm)), "order_by_absmax")
+    return perm
 
 
 def group_error(T, kind, bits, group, ts=1.0, perms=None, err=None):

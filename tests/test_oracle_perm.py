@@ -253,3 +253,29 @@ def test_tau_monotone_and_zero_error_rejects():
 
 def test_error_weight():
     assert O.error_weight(np.array([1.0, 3.0])) == 0.25
+
+
+# ---------------------------------------------------------------- absmax criterion (Tab. 2(a))
+def test_absmax_order_against_a_stable_library_sort_and_by_hand():
+    a = np.array([3.0, 0.5, 3.0, 7.25, 0.0, 0.5, 1e-30, 7.25], dtype=np.float32)
+    # by hand: 7.25 (ch 3), 7.25 (ch 7), 3 (ch 0), 3 (ch 2), .5 (ch 1), .5 (ch 5), 1e-30 (ch 6), 0 (ch 4)
+    assert O.order_by_absmax(a).tolist() == [3, 7, 0, 2, 1, 5, 6, 4]
+    g = np.random.default_rng(3)
+    big = np.round(np.abs(g.standard_normal(5000)) * 8).astype(np.float32) / 8      # many ties
+    got = O.order_by_absmax(big)
+    assert np.array_equal(got, np.argsort(-big.astype(np.float64), kind="stable"))
+    assert sorted(got.tolist()) == list(range(5000))
+
+
+def test_absmax_order_of_real_statistics_differs_from_the_second_moment_order():
+    """Heavy-tailed columns: a rare spike raises a channel's absmax but hardly its second moment, so
+    the two criteria of Tab. 2(a) are different orders (and each is sorted by its own key)."""
+    g = np.random.default_rng(9)
+    x = g.standard_normal((512, 64)).astype(np.float32) * np.linspace(0.5, 2.0, 64, dtype=np.float32)
+    x[7, 5] = 12.0
+    xb = bf(x)
+    S, A = O.calib_stats(xb)
+    by_max = O.order_by_absmax(A)
+    by_moment = O.select_perm(S, 512, np.ones(64), 1, J=1)[1]
+    assert by_max[0] == 5 and by_moment[0] != 5
+    assert np.all(np.diff(A[by_max]) <= 0) and np.all(np.diff(S[by_moment]) <= 0)
