@@ -189,6 +189,14 @@ pq_status pq_output_error(const float *Yref, int64_t ld_ref, const void *Yq, int
                           int64_t rows, int64_t N, double *err, void *ws, size_t ws_bytes,
                           void *stream);
 
+/* The absmax criterion of the reordering ablation (Tab. 2(a)) as one more candidate order:
+ * perm[pos] = channel with the pos-th largest absmax, equal values in ascending channel order.
+ * The row can be appended to the candidate table that pq_group_error / pq_accept evaluate.
+ *   amax : device fp32 [K] (as accumulated by pq_calib_stats).  K <= 16384.
+ *   perm : device int32 [K] out.  ws : pq_workspace_bytes(PQ_OP_SELECT_PERM, 0, K, 0, 1). */
+pq_status pq_order_by_absmax(const float *amax, int64_t K, int32_t *perm, void *ws, size_t ws_bytes,
+                             void *stream);
+
 /* Relative-error weights for pq_accept: lambda[0] = 1 / sum_i sumsq_a[i], lambda[1] =
  * 1 / sum_i sumsq_w[i] (sequential fp64 sums in channel order).  lambda: device fp64 [2]. */
 pq_status pq_error_weights(const double *sumsq_a, const double *sumsq_w, int64_t K, double *lambda,

@@ -40,6 +40,7 @@ _SIGNATURES = {
     "pq_sf_bytes": (_sz, [_i64, _i64, _int]),
     "pq_calib_stats": (_int, [_vp, _i64, _i64, _i64, _vp, _vp, _vp, _sz, _vp]),
     "pq_quant_act_nvfp4_perm": (_int, [_vp, _i64, _i64, _i64, _vp, _vp, _vp, _vp, _int, _vp]),
+    "pq_order_by_absmax": (_int, [_vp, _i64, _vp, _vp, _sz, _vp]),
     "pq_output_error": (_int, [_vp, _i64, _vp, _i64, _i64, _i64, _vp, _vp, _sz, _vp]),
     "pq_calib_stats_static": (_int, [_vp, _i64, _i64, _i64, _vp, _vp, _vp]),
     "pq_calib_stats_static_max_bytes": (_sz, []),
@@ -142,6 +143,13 @@ def pq_calib_stats(T, sumsq, amax, ws):
     w, wb = _ws(ws)
     _check("pq_calib_stats", lib().pq_calib_stats(_p(T), T.shape[0], T.shape[1], T.stride(0), _p(sumsq),
                                                   _p(amax), w, wb, _stream()))
+
+
+def pq_order_by_absmax(amax, perm, ws):
+    """perm[pos] = channel with the pos-th largest absmax (ties by ascending channel); int32 [K]."""
+    assert amax.dtype == torch.float32 and perm.dtype == torch.int32 and perm.numel() == amax.numel()
+    w, wb = _ws(ws)
+    _check("pq_order_by_absmax", lib().pq_order_by_absmax(_p(amax), amax.numel(), _p(perm), w, wb, _stream()))
 
 
 def pq_output_error(Yref, Yq, err, ws):

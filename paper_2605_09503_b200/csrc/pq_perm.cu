@@ -26,6 +26,12 @@ __global__ void perm_keys(const double *__restrict__ sa, double rows_a, const do
     }
 }
 
+// keys[i] = bit pattern of the channel's absmax widened to fp64 (exact; non-negative).
+__global__ void absmax_keys(const float *__restrict__ amax, int64_t K, unsigned long long *__restrict__ keys) {
+    const int64_t i = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
+    if (i < K) keys[i] = static_cast<unsigned long long>(__double_as_longlong(static_cast<double>(fabsf(amax[i]))));
+}
+
 constexpr int kRankThreads = 256;
 
 __global__ void __launch_bounds__(kRankThreads)
@@ -93,6 +99,19 @@ extern "C" pq_status pq_select_perm(const double *sumsq_a, int64_t rows_a, const
         sumsq_a, static_cast<double>(rows_a), sumsq_w, static_cast<double>(rows_w), K, J, keys);
     dim3 grid(static_cast<unsigned>(pq_ceil_div(K, kRankThreads)), static_cast<unsigned>(J + 1));
     perm_rank<<<grid, kRankThreads, 0, st>>>(keys, K, perms);
+    return pq_launch_status();
+}
+
+extern "C" pq_status pq_order_by_absmax(const float *amax, int64_t K, int32_t *perm, void *ws, size_t ws_bytes,
+                                        void *stream) {
+    PQ_REQUIRE(amax && perm, PQ_ERR_NULL);
+    PQ_REQUIRE(K > 0 && K <= 16384, PQ_ERR_SHAPE);
+    PQ_REQUIRE(ws && ws_bytes >= pq_workspace_bytes(PQ_OP_SELECT_PERM, 0, K, 0, 1), PQ_ERR_WORKSPACE);
+    PQ_REQUIRE(pq_aligned256(ws), PQ_ERR_ALIGN);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    unsigned long long *keys = static_cast<unsigned long long *>(ws);
+    absmax_keys<<<static_cast<unsigned>(pq_ceil_div(K, 128)), 128, 0, st>>>(amax, K, keys);
+    perm_rank<<<dim3(static_cast<unsigned>(pq_ceil_div(K, kRankThreads)), 1), kRankThreads, 0, st>>>(keys, K, perm);
     return pq_launch_status();
 }
 

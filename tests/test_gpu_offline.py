@@ -232,3 +232,31 @@ def test_workspaces_are_not_overrun(rows, K):
             err = torch.zeros(P, K // fmt[2], dtype=torch.float64, device=DEV)
             B.pq_group_error(x, fmt, ts, pm, err, ws)
             assert bool((buf[need:] == 0xA5).all())
+
+
+@pytest.mark.parametrize("K", [16, 3072, 16384])
+def test_absmax_order_bit_exact_with_ties(K):
+    """Tab. 2(a) absmax criterion: same permutation as the oracle, ties included."""
+    g = torch.Generator().manual_seed(K)
+    amax = (torch.randn(K, generator=g).abs() * 8).round() / 8          # many equal values
+    perm = torch.empty(K, dtype=torch.int32, device=DEV)
+    B.pq_order_by_absmax(dev(amax.float()), perm, B.workspace(B.OP_SELECT_PERM, 0, K, 0, 1))
+    assert np.array_equal(perm.cpu().numpy(), O.order_by_absmax(amax.numpy()))
+
+
+def test_absmax_order_as_an_extra_candidate_of_the_error_pass():
+    rows, K = 200, 512
+    x = inputs.activations(small_cfg(rows, K), 3, 0)
+    S = torch.zeros(K, dtype=torch.float64, device=DEV)
+    A = torch.zeros(K, dtype=torch.float32, device=DEV)
+    B.pq_calib_stats(dev(x), S, A, B.workspace(B.OP_CALIB_STATS, rows, K))
+    perm = torch.empty(1, K, dtype=torch.int32, device=DEV)
+    B.pq_order_by_absmax(A, perm[0], B.workspace(B.OP_SELECT_PERM, 0, K, 0, 1))
+    _, A_o = O.calib_stats(inputs.bits(x))
+    perm_o = O.order_by_absmax(A_o)
+    assert np.array_equal(perm.cpu().numpy()[0], perm_o)
+    ts = torch.tensor([0.02], dtype=torch.float32)
+    err = torch.zeros(1, K // 16, dtype=torch.float64, device=DEV)
+    B.pq_group_error(dev(x), (0, 4, 16), dev(ts), perm, err, B.workspace(B.OP_GROUP_ERROR, rows, K, 0, 1))
+    want = O.group_error(inputs.bits(x), 0, 4, 16, ts=ts.item(), perms=perm_o[None, :])
+    assert np.array_equal(err.cpu().numpy(), want)
