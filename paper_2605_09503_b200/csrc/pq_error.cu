@@ -73,6 +73,11 @@ __device__ __forceinline__ uint64_t fma2(uint64_t a, uint64_t b, uint64_t c) {
     return r;
 }
 
+__device__ __forceinline__ uint32_t max_bf16x2(uint32_t a, uint32_t b) {
+    uint32_t r;
+    asm("max.bf16x2 %0, %1, %2;" : "=r"(r) : "r"(a), "r"(b));
+    return r;
+}
 __device__ __forceinline__ uint64_t add2(uint64_t a, uint64_t b) {
     uint64_t r;
     asm("add.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
@@ -87,12 +92,15 @@ __device__ __forceinline__ uint64_t add2(uint64_t a, uint64_t b) {
 template <int KIND, int TEAM16>
 __device__ __forceinline__ float row_sse16(const uint4 &lo, const uint4 &hi, float c6, const float2 *table, float Qf) {
     const uint32_t m = 0x7FFF7FFFu;
+    const uint4 la = make_uint4(lo.x & m, lo.y & m, lo.z & m, lo.w & m);
+    const uint4 ha = make_uint4(hi.x & m, hi.y & m, hi.z & m, hi.w & m);
     float xa[8], xb[8];
-    pq::unpack8(make_uint4(lo.x & m, lo.y & m, lo.z & m, lo.w & m), xa);
-    pq::unpack8(make_uint4(hi.x & m, hi.y & m, hi.z & m, hi.w & m), xb);
-    float amax = 0.0f;
-#pragma unroll
-    for (int i = 0; i < 8; ++i) amax = fmaxf(amax, fmaxf(xa[i], xb[i]));
+    pq::unpack8(la, xa);
+    pq::unpack8(ha, xb);
+    // absmax of the 16 magnitudes on the bf16 pairs (exact: a maximum selects one of its inputs)
+    const uint32_t mx = max_bf16x2(max_bf16x2(max_bf16x2(la.x, la.y), max_bf16x2(la.z, la.w)),
+                                   max_bf16x2(max_bf16x2(ha.x, ha.y), max_bf16x2(ha.z, ha.w)));
+    float amax = fmaxf(__uint_as_float(mx << 16), __uint_as_float(mx & 0xFFFF0000u));
     amax = pq::team_max<TEAM16>(amax);
     float d, r;
     if (KIND == 0) {
