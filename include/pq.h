@@ -21,7 +21,9 @@
  *     K contiguous.  Activations are X[M,K]; weights are stored transposed, Wt[N,K] (the
  *     nn.Linear convention), so "input channel i of W" is column i of Wt.
  *   - Permutations use the gather convention of App. C: position j of the reordered tensor
- *     reads channel perm[j] of the original one.
+ *     reads channel perm[j] of the original one.  Every order handed to the library must hold
+ *     values in [0, K): the gather kernels index a staged row with them and do not check (the
+ *     orders the library itself produces always do).
  *   - Inputs must be finite.  Tensor scales must lie in [2^-100, 2^100].
  *
  * NVFP4 storage
@@ -152,7 +154,9 @@ pq_status pq_tensor_scale(const float *amax, int64_t K, float *ts, void *stream)
  * (a_i)^alpha (w_i)^(1-alpha)).  perms[j*K + pos] = channel with the pos-th largest key; equal
  * keys keep ascending channel order.  j = J is the activation-only sort of Prop. 3.2, j = 0 the
  * weight-only sort.
- *   K <= 16384, 1 <= J <= 16.  perms : int32 [J+1, K] out.  ws: unused (may be NULL). */
+ *   K <= 16384, 1 <= J <= 16.  perms : int32 [J+1, K] out.
+ *   ws : pq_workspace_bytes(PQ_OP_SELECT_PERM, 0, K, 0, J + 1) bytes, 256-byte aligned (the sort keys of
+ *        every candidate); a NULL or short workspace returns PQ_ERR_WORKSPACE. */
 pq_status pq_select_perm(const double *sumsq_a, int64_t rows_a, const double *sumsq_w,
                          int64_t rows_w, int64_t K, int J, int32_t *perms, void *ws,
                          size_t ws_bytes, void *stream);
@@ -339,34 +343,6 @@ pq_status pq_norm_quant_nvfp4(const void *H, int64_t M, int64_t K, int64_t ld, i
                               const float *b, float eps, const int32_t *perm, const float *ts_x,
                               uint8_t *codes, uint8_t *sf, int sf_layout, void *y_out, void *stream);
 
-/* Machine probes (no counterpart in the paper: they measure the GPU, not the method).  The GEMM's tile
- * shape is bounded by how many operand bytes an SM can take in from L2 per MMA cycle and by how fast
- * it can write a finished tile; these two calls measure both rates so that the roofline argument can
- * be re-checked on any machine.
- *   pq_probe_sm_ingest: `ctas` CTAs (one per SM when ctas <= SM count) each stream iters x 32 KB from
- *     the region [src, src + region_bytes) (device memory; keep it below the L2 size and touch it
- *     once to measure L2 -> SM) into shared memory with bulk copies, 6 in flight.  cycles[0] = SM clock
- *     cycles of the slowest CTA, so bytes per clock per SM = iters * 32768 / cycles[0].
- *     region_bytes: a multiple of 32768, >= 65536.  status: device int, PQ_OK or PQ_ERR_TIMEOUT.
- *     sm_select: 0 = every CTA works; 1 = only CTAs that landed on an SM with an even id (one SM of
- *     each pair of neighbouring SMs); 2 = only CTAs on SMs whose id / 2 is even (both SMs of every
- *     other pair): with ctas = SM count, 1 and 2 keep half of the SMs busy in two different patterns,
- *     which tells a per-SM-pair limit from a global one.
- *   pq_probe_sm_store: `ctas` CTAs of four warps each write iters x 2048 bytes (512 contiguous bytes
- *     per warp instruction) to disjoint parts of dst (>= ctas * iters * 2048 bytes).  cycles[0] as above.
- * Both are asynchronous on `stream`; cycles / status are device words the calls reset first. */
-pq_status pq_probe_sm_ingest(const void *src, size_t region_bytes, int ctas, int iters, int sm_select,
-                             unsigned long long *cycles, int *status, void *stream);
-pq_status pq_probe_sm_store(void *dst, size_t dst_bytes, int ctas, int iters,
-                            unsigned long long *cycles, void *stream);
-/*   pq_probe_sm_forward: CTA pairs (clusters of two, ctas even); both CTAs stream iters x 32 KB from
- *     L2 as above (4 copies in flight) while, if fwd_iters > 0, the first CTA of each pair also pushes
- *     fwd_iters x 32 KB of its own shared memory into the second one's (2 in flight).  cycles[0] =
- *     slowest L2 stream, cycles[1] = slowest forwarding loop: comparing cycles[0] with and without
- *     forwarding tells whether shared-to-shared copies inside a cluster use the path from L2. */
-pq_status pq_probe_sm_forward(const void *src, size_t region_bytes, int ctas, int iters, int fwd_iters,
-                              unsigned long long *cycles, int *status, void *stream);
-
 /* Integer fake-quant of Eq. 1-2 (quantize, dequantize, round to bf16), optional gather.
  *   T : bf16 [rows, K], ld.  out : bf16 [rows, K], ldo.  perm : int32 [K] or NULL.
  *   fmt.kind must be 1; K % fmt.group == 0; K <= 16384 when perm != NULL. */
@@ -382,6 +358,18 @@ pq_status pq_sf_to_linear(const uint8_t *sf_tc, int64_t rows, int64_t K, uint8_t
  * PQ_ERR_TIMEOUT if a bounded wait inside the kernel expired, PQ_ERR_CUDA if the stream reports
  * an asynchronous error.  HOST call; `ws` is the device workspace passed to pq_gemm_w4a4. */
 pq_status pq_device_status(const void *ws, void *stream);
+
+/* Exercises the expiry path of the GEMM's bounded device-side waits without a hang or a fault (the
+ * failure-detection path of the library; the paper has no counterpart).  One warp waits, with the same
+ * helper every role of the GEMM kernel uses, on a barrier that nobody arrives at; after `limit_cycles`
+ * SM clock cycles the wait gives up, raises the kernel's abort flag, writes PQ_ERR_TIMEOUT into the
+ * status word at `ws` and the kernel returns normally: the context stays usable.
+ *   ws           : a GEMM workspace (device); afterwards pq_device_status(ws) reports PQ_ERR_TIMEOUT
+ *                  until the caller zeroes the word again.
+ *   limit_cycles : 1 .. 1e8 (a fraction of a second at most).
+ *   observed     : device int32 [2] out: {result of the wait (0 = gave up), abort flag}. */
+pq_status pq_selftest_wait_expiry(void *ws, size_t ws_bytes, long long limit_cycles, int *observed,
+                                  void *stream);
 
 #ifdef __cplusplus
 }

@@ -66,9 +66,7 @@ _SIGNATURES = {
                                    _vp]),
     "pq_last_error_detail": (C.c_char_p, []),
     "pq_device_status": (_int, [_vp, _vp]),
-    "pq_probe_sm_ingest": (_int, [_vp, _sz, _int, _int, _int, _vp, _vp, _vp]),
-    "pq_probe_sm_store": (_int, [_vp, _sz, _int, _int, _vp, _vp]),
-    "pq_probe_sm_forward": (_int, [_vp, _sz, _int, _int, _int, _vp, _vp, _vp]),
+    "pq_selftest_wait_expiry": (_int, [_vp, _sz, C.c_longlong, _vp, _vp]),
 }
 
 
@@ -337,36 +335,13 @@ def pq_norm_quant_nvfp4(H, kind, a, b, eps, perm, ts_x, codes, sf, sf_layout, y_
                                                             _p(ts_x), _p(codes), _p(sf), sf_layout, _p(y_out), _stream()))
 
 
-def pq_probe_sm_ingest(src, ctas, iters, sm_select=0):
-    """-> bytes per SM clock per SM that `ctas` CTAs pull from the (L2-resident) uint8 tensor src."""
-    cycles = torch.zeros(1, dtype=torch.int64, device=src.device)
-    status = torch.zeros(1, dtype=torch.int32, device=src.device)
-    _check("pq_probe_sm_ingest", lib().pq_probe_sm_ingest(_p(src), src.numel(), ctas, iters, sm_select, _p(cycles), _p(status),
-                                                          _stream()))
-    torch.cuda.synchronize()
-    _check("pq_probe_sm_ingest (device)", int(status.item()))
-    return iters * 32768 / max(int(cycles.item()), 1)
-
-
-def pq_probe_sm_forward(src, ctas, iters, fwd_iters):
-    """-> (bytes per clock per SM pulled from L2, bytes per clock forwarded between the CTAs of a pair)."""
-    cycles = torch.zeros(2, dtype=torch.int64, device=src.device)
-    status = torch.zeros(1, dtype=torch.int32, device=src.device)
-    _check("pq_probe_sm_forward", lib().pq_probe_sm_forward(_p(src), src.numel(), ctas, iters, fwd_iters, _p(cycles),
-                                                            _p(status), _stream()))
-    torch.cuda.synchronize()
-    _check("pq_probe_sm_forward (device)", int(status.item()))
-    c = cycles.tolist()
-    return iters * 32768 / max(c[0], 1), (fwd_iters * 32768 / c[1] if fwd_iters and c[1] else 0.0)
-
-
-def pq_probe_sm_store(dst, ctas, iters):
-    """-> bytes per SM clock per SM that `ctas` CTAs write into the uint8 tensor dst."""
-    cycles = torch.zeros(1, dtype=torch.int64, device=dst.device)
-    _check("pq_probe_sm_store", lib().pq_probe_sm_store(_p(dst), dst.numel(), ctas, iters, _p(cycles), _stream()))
-    torch.cuda.synchronize()
-    return iters * 2048 / max(int(cycles.item()), 1)
-
-
 def pq_device_status(ws):
     return int(lib().pq_device_status(_p(ws), _stream()))
+
+
+def pq_selftest_wait_expiry(ws, limit_cycles):
+    """A bounded device-side wait that is left to run out; -> (wait result, abort flag) as the kernel saw them."""
+    observed = torch.full((2,), -1, dtype=torch.int32, device=ws.device)
+    w, wb = _ws(ws)
+    _check("pq_selftest_wait_expiry", lib().pq_selftest_wait_expiry(w, wb, int(limit_cycles), _p(observed), _stream()))
+    return tuple(observed.tolist())

@@ -11,10 +11,6 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libpq.so")
-# single-GPU extras (cluster-multicast probe): their own sources and library, which multi-GPU runs
-# leave behind; nothing in the package needs them
-CSRC_MC = os.path.join(HERE, "csrc_mc")
-LIB_MC = os.path.join(HERE, "libpq_mc.so")
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "-Xcompiler", "-Wall", "--fmad=false", "-cudart", "static"]
 
@@ -43,10 +39,6 @@ def build(force: bool = False, verbose: bool = False) -> str:
         subprocess.run(cmd, check=True)
         objs.append(obj)
     subprocess.run(["nvcc", "-Wno-deprecated-gpu-targets", "-shared", "-cudart", "static", "-o", LIB, *objs, "-ldl", "-lpthread", "-lrt"], check=True)
-    mc_sources = sorted(glob.glob(os.path.join(CSRC_MC, "*.cu")))
-    if mc_sources:
-        subprocess.run(["nvcc", *NVCC_FLAGS, "-Wno-deprecated-gpu-targets", "-shared", "-o", LIB_MC, *mc_sources,
-                        "-ldl", "-lpthread", "-lrt"], check=True)
     return LIB
 
 

@@ -10,6 +10,8 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <mutex>
+
 #include "../../include/pq.h"
 
 #define PQ_REQUIRE(cond, code) \
@@ -41,6 +43,20 @@ static inline pq_status pq_launch_status() {
 }
 
 static inline int64_t pq_ceil_div(int64_t a, int64_t b) { return (a + b - 1) / b; }
+
+// Kernel attributes (shared-memory opt-in, carve-out) and occupancy answers belong to a device, not
+// to the process: a cache of them is indexed by the current device's ordinal and guarded by a lock.
+constexpr int kPqMaxDevices = 64;
+struct PqPerDevice {
+    std::mutex lock;
+    int value[kPqMaxDevices] = {};  // 0 = not set up on that device yet
+};
+// Index of the current device in such a cache, or -1.
+static inline int pq_device_slot() {
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kPqMaxDevices) return -1;
+    return dev;
+}
 
 // pq_quant_act_nvfp4 with a choice of block shape (library-internal; defined in pq_quant.cu).
 pq_status pq_quant_act_nvfp4_shaped(const void *X, int64_t M, int64_t K, int64_t ld, const float *ts_x, uint8_t *codes,

@@ -72,17 +72,37 @@ constexpr int kEpiBytes = kEpiWarps * kEpiBox;      // one staging box per epilo
 constexpr int kFirstStager = 2 + kEpiWarps;
 constexpr int kThreads = 32 * (kFirstStager + 8);   // producer, MMA issuer, 8 epilogue and 8 stager warps
 constexpr int kTmemCols = 512;
-// One 256-column accumulator, then two scale slots, one per stager set (a set always writes the same
-// slot, and only after the MMAs that read it two iterations earlier have completed).  With four slots,
-// i.e. stagers running up to four stages ahead of the tensor pipe with both sets writing at once, about
-// one launch in 450 of the 4608 x 3072 x 9216 product came out with the rows of a lane quadrant of some
-// tiles wrong (off as if part of K had met other scale factors); two slots cost nothing (the stage time is bounded by operand
-// delivery) and 36000 launches were clean (so were three slots, in either column range).  A slot holds the scales of one stage: per
-// 64-channel K block 4 columns of A scales (128 rows) and 8 columns of B scales (256 rows).
+// One 256-column accumulator, then the scale slots.  A slot holds the scales of one stage: per
+// 64-channel K block 4 columns of A scales (128 rows) and 8 columns of B scales (256 rows).  Slot
+// it % kSfSlots serves iteration it; it is rewritten only after the MMAs of iteration it - kSfSlots
+// have completed (their commit releases that iteration's stage).
+//
+// Why the slot count is tied to the stage count.  Every wait here is a PARITY wait: it tells "phase n
+// of this barrier has completed" from "it has not" only if the barrier cannot still be in phase n - 1,
+// i.e. only if the waiter already knows that phase n - 1 has completed.  A role that waits on every
+// phase of a barrier in turn (producer on stage_free, MMA issuer on stage_full and acc_empty, each
+// epilogue warp on acc_full) knows it from its own previous wait.  The stagers do not: the stage
+// count is odd and the two stager sets take alternate iterations, so the previous phase of
+// sf_ready(s), iteration it - kStages, was waited for by the OTHER set.  What a set knows when it
+// reaches iteration `it` is what its own iteration it - 2 waited for: the MMAs of it - 2 - kSfSlots
+// have completed.  Those of it - kStages (hence that iteration's scale copies, which its stagers had
+// to see before its MMAs could be issued) are then known complete only if
+//     it - 2 - kSfSlots >= it - kStages,   i.e.  kSfSlots + 2 <= kStages.
+// With 4 slots and 5 stages the condition fails: when the scale copies of it - kStages were still in
+// flight the wait for phase n returned true one phase early, the warp read the previous occupant's
+// scale bytes from shared memory and stored them to tensor memory -- one lane quadrant of one CTA,
+// all columns, wrong by the ratio of two scale factors -- about once in 450 launches of the
+// 4608 x 3072 x 9216 product.  2 and 3 slots, and 4 slots with the stagers held to three stages
+// ahead, satisfy the condition and never failed.  The stagers now also wait for the release of
+// iteration it - kStages (stage_free, which the producer waited for before it refilled the stage)
+// in front of the sf_ready wait, so that wait is sound whatever the slot count; the assertion below
+// keeps the original condition as well.
 constexpr int kSfSlots = 2;
 constexpr uint32_t kSfSlotCol0 = BN, kSfSlotCols = 4 * (4 + 8), kSfbOfs = 16;
 static_assert(kSfSlotCol0 + kSfSlots * kSfSlotCols <= 512, "tensor memory columns");
-constexpr long long kWaitCycles = 4000000000ll;  // about two seconds of SM clock per wait
+static_assert(kSfSlots + 2 <= kStages, "a stager set must know that the previous phase of sf_ready has completed");
+static_assert(kSfSlots <= 2 * kStages - 2, "the stagers' parity waits on stage_free must be unambiguous");
+constexpr long long kWaitCycles = 4000000000ll;  // default limit of a wait: about two seconds of SM clock
 // barriers: stage_full[S] sf_ready[S] stage_free[S] acc_full acc_empty
 constexpr int kNumBars = 3 * kStages + 2;
 constexpr size_t kSmemBytes = kStages * kStageBytes + kEpiBytes + 1024 /*alignment slack*/ + 8 * kNumBars + 64;
@@ -93,6 +113,7 @@ struct GemmParams {
     int M, N, K;
     int m_tiles, n_tiles, k_tiles, kb_total, kb4;
     int m_rowblocks, n_rowblocks;
+    long long wait_cycles;  // limit of every mbarrier wait, in SM clock cycles
     int *status;
 };
 
@@ -165,33 +186,38 @@ __device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
         : "memory");
     return ok != 0;
 }
-// Bounded wait: polls until the phase completes, the abort flag goes up, or kWaitCycles SM
-// clock cycles have passed (then it raises the flag and records the timeout).
-__device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volatile int *abort_flag, int *status) {
+// Bounded wait: polls until the phase completes, the abort flag goes up, or `limit` SM clock cycles
+// have passed (then it raises the flag and records the timeout).
+struct WaitCtx {
+    volatile int *abort_flag;
+    int *status;
+    long long limit;
+};
+__device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, const WaitCtx w) {
     const long long t0 = clock64();
     for (uint32_t spins = 1;; ++spins) {
         if (mbar_try(bar, parity)) return true;
         if ((spins & 63u) == 0) {
-            if (*abort_flag) return false;
-            if (clock64() - t0 > kWaitCycles) break;
+            if (*w.abort_flag) return false;
+            if (clock64() - t0 > w.limit) break;
         }
     }
-    *abort_flag = 1;
-    atomicExch(status, static_cast<int>(PQ_ERR_TIMEOUT));
+    *w.abort_flag = 1;
+    atomicExch(w.status, static_cast<int>(PQ_ERR_TIMEOUT));
     return false;
 }
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag, int *status) {
+// Wait of a single thread (or of lanes that vote on the result themselves).
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, const WaitCtx w) {
     if (mbar_try(bar, parity)) return true;
-    return mbar_wait_slow(bar, parity, abort_flag, status);
+    return mbar_wait_slow(bar, parity, w);
 }
-// The same for a converged warp: every lane gets the same answer (the vote is only taken on the
-// slow path; a vote per K iteration costs the MMA issuer 20 of its 384 cycles).
-__device__ __noinline__ bool mbar_wait_slow_warp(uint32_t bar, uint32_t parity, volatile int *abort_flag, int *status) {
-    return __all_sync(0xFFFFFFFFu, mbar_wait_slow(bar, parity, abort_flag, status));
-}
-__device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, volatile int *abort_flag, int *status) {
-    if (mbar_try(bar, parity)) return true;
-    return mbar_wait_slow_warp(bar, parity, abort_flag, status);
+// Wait of a converged warp: every lane returns the same answer and the warp is converged again
+// afterwards, so .sync.aligned instructions (elect, tcgen05.st / ld) may follow on either outcome.
+__device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, const WaitCtx w) {
+    bool ok = mbar_try(bar, parity);
+    if (__all_sync(0xFFFFFFFFu, ok)) return true;
+    ok = ok || mbar_wait_slow(bar, parity, w);
+    return __all_sync(0xFFFFFFFFu, ok);
 }
 __device__ __forceinline__ void prefetch_tensormap(const CUtensorMap *map) {
     asm volatile("prefetch.tensormap [%0];" ::"l"(map) : "memory");
@@ -342,6 +368,8 @@ gemm_w4a4_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
     uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars_ptr + 8 * kNumBars);
     volatile int *abort_flag = reinterpret_cast<volatile int *>(bars_ptr + 8 * kNumBars + 8);
 
+    const WaitCtx wctx{abort_flag, p.status, p.wait_cycles};
+
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t rank = cluster_ctarank();  // 0 = pair leader
     const int pair = blockIdx.x >> 1, num_pairs = gridDim.x >> 1;
@@ -398,7 +426,7 @@ gemm_w4a4_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
             for (int kt = 0; kt < p.k_tiles; ++kt, ++it) {
                 const int s = it % kStages;
                 const uint32_t par = (it / kStages) & 1u;
-                ok = mbar_wait_warp(stage_free_bar(s), par ^ 1u, abort_flag, p.status);
+                ok = mbar_wait_warp(stage_free_bar(s), par ^ 1u, wctx);
                 if (!ok) break;
                 const int kb_valid = min(4, p.kb_total - kt * 4);
                 const uint32_t sf_bytes = static_cast<uint32_t>(kb_valid) * kSfBlock;
@@ -434,13 +462,13 @@ gemm_w4a4_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
             bool ok = true;
             for (int tile = pair; tile < total_tiles && ok; tile += num_pairs, ++tcount) {
                 // the accumulator is free once the epilogue has read the previous tile out of it
-                ok = mbar_wait_warp(acc_empty_bar, (tcount & 1u) ^ 1u, abort_flag, p.status);
+                ok = mbar_wait_warp(acc_empty_bar, (tcount & 1u) ^ 1u, wctx);
                 if (!ok) break;
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base;
                 uint32_t acc = 0;
                 for (int kt = 0; kt < p.k_tiles; ++kt) {
-                    ok = mbar_wait_warp(stage_full_bar(s), ph, abort_flag, p.status);
+                    ok = mbar_wait_warp(stage_full_bar(s), ph, wctx);
                     if (!ok) break;
                     tc_fence_after();
                     const uint32_t stage = base + s * kStageBytes;
@@ -486,12 +514,11 @@ gemm_w4a4_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
                 if ((it & 1u) != set) continue;
                 const int s = it % kStages;
                 const uint32_t t = it % kSfSlots;
-                // the stage's scale blocks have landed, and the MMAs that read this slot kSfSlots
-                // iterations ago have completed (their commit released that iteration's stage)
-                if (!mbar_wait(sf_ready_bar(s), (it / kStages) & 1u, abort_flag, p.status)) {
-                    ok = false;
-                    break;
-                }
+                // The stage's previous occupant has been released (which makes the parity wait that
+                // follows unambiguous: see kSfSlots), then: this iteration's scale blocks have landed.
+                if (it >= kStages) ok = mbar_wait_warp(stage_free_bar(s), ((it - kStages) / kStages) & 1u, wctx);
+                ok = ok && mbar_wait_warp(sf_ready_bar(s), (it / kStages) & 1u, wctx);
+                if (!ok) break;
                 const int kb_valid = min(4, p.kb_total - kt * 4);
                 const uint32_t sf_s = base + s * kStageBytes + kABytes + kBBytes + lane * 16u;
                 const uint32_t sf_t = tmem_base + lane_ofs + sf_slot_col(t);
@@ -505,11 +532,11 @@ gemm_w4a4_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
                         b1[kk] = lds128(sf_s + 2 * kSfaBytes + kk * kSfBlock);
                     }
                 }
-                if (it >= kSfSlots && !mbar_wait(stage_free_bar((it - kSfSlots) % kStages),
-                                                 ((it - kSfSlots) / kStages) & 1u, abort_flag, p.status)) {
-                    ok = false;
-                    break;
-                }
+                // the MMAs that read this slot kSfSlots iterations ago have completed (their commit
+                // released that iteration's stage)
+                if (it >= kSfSlots)
+                    ok = mbar_wait_warp(stage_free_bar((it - kSfSlots) % kStages), ((it - kSfSlots) / kStages) & 1u, wctx);
+                if (!ok) break;
                 tc_fence_after();
                 if (kb_valid == 4) {
 #pragma unroll
@@ -548,7 +575,7 @@ gemm_w4a4_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
         for (int tile = pair; tile < total_tiles; tile += num_pairs, ++tcount) {
             const int m_blk = tile % p.m_tiles, n_blk = tile / p.m_tiles;
             const int m0 = m_blk * BM + static_cast<int>(rank) * BM_CTA + q * 32, n0 = n_blk * BN + h * (BN / 2);
-            const bool got = mbar_wait(acc_full_bar, tcount & 1u, abort_flag, p.status);
+            const bool got = mbar_wait(acc_full_bar, tcount & 1u, wctx);
             if (!__all_sync(0xFFFFFFFFu, got)) break;
             if (rank == 0 && warp == 2 && lane == 0) mbar_arrive_remote(acc_full_bar, 1);
             tc_fence_after();
@@ -600,6 +627,25 @@ gemm_w4a4_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
     if (warp == 1) {
         tc_fence_after();
         asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
+    }
+}
+
+// One warp waits, with the kernel's own bounded wait, on a barrier that nobody arrives at: the way
+// the expiry path (status word, abort flag, orderly return) is exercised without a fault or a hang.
+__global__ void __launch_bounds__(32) wait_expiry_kernel(int *status, long long limit, int *observed) {
+    __shared__ __align__(8) unsigned long long bar;
+    __shared__ int abort_word;
+    if (threadIdx.x == 0) {
+        mbar_init(smem_u32(&bar), 1);
+        abort_word = 0;
+    }
+    __syncwarp();
+    const WaitCtx w{&abort_word, status, limit};
+    const bool ok = mbar_wait_warp(smem_u32(&bar), 0u, w);
+    // every lane has the same answer and the warp is converged: what the roles of the GEMM rely on
+    if (threadIdx.x == 0) {
+        observed[0] = ok ? 1 : 0;
+        observed[1] = abort_word;
     }
 }
 
@@ -664,10 +710,19 @@ bool make_map(CUtensorMap *map, const void *ptr, int64_t rows, int64_t row_bytes
     return true;
 }
 
-// Number of CTA pairs that can be resident at once (a cluster must fit inside one GPC).
+// Number of CTA pairs that can be resident at once on the current device (a cluster must fit inside
+// one GPC), after opting the kernel in to its dynamic shared memory there.  Both are per device.
 int resident_pairs() {
-    static int pairs = 0;
-    if (pairs) return pairs;
+    static PqPerDevice cache;
+    const int dev = pq_device_slot();
+    if (dev < 0) return 0;
+    std::lock_guard<std::mutex> guard(cache.lock);
+    if (cache.value[dev]) return cache.value[dev];
+    if (cudaFuncSetAttribute(gemm_w4a4_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             static_cast<int>(kSmemBytes)) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return 0;
+    }
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(2, 1, 1);
     cfg.blockDim = dim3(kThreads, 1, 1);
@@ -684,8 +739,8 @@ int resident_pairs() {
         (void)cudaGetLastError();
         return 0;
     }
-    pairs = n;
-    return pairs;
+    cache.value[dev] = n;
+    return n;
 }
 
 }  // namespace
@@ -709,12 +764,6 @@ pq_status gemm_launch(const uint8_t *xq, const uint8_t *sfx, const float *ts_x, 
         !make_map(&map_y, Y, M, N * 2, ldy * 2, 32, 2))
         return PQ_ERR_CUDA;
 
-    static bool attr_set = false;
-    if (!attr_set) {
-        PQ_CUDA_OK(cudaFuncSetAttribute(gemm_w4a4_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                        static_cast<int>(kSmemBytes)));
-        attr_set = true;
-    }
     const int pairs_max = resident_pairs();
     if (pairs_max <= 0) return PQ_ERR_CUDA;
 
@@ -728,6 +777,7 @@ pq_status gemm_launch(const uint8_t *xq, const uint8_t *sfx, const float *ts_x, 
     p.kb4 = p.kb_total;
     p.m_rowblocks = static_cast<int>(pq_ceil_div(M, 128));
     p.n_rowblocks = static_cast<int>(pq_ceil_div(N, 128));
+    p.wait_cycles = kWaitCycles;
     p.status = static_cast<int *>(ws);
     const int64_t tiles = static_cast<int64_t>(p.m_tiles) * p.n_tiles;
     const int pairs = static_cast<int>(tiles < pairs_max ? tiles : pairs_max);
@@ -917,6 +967,15 @@ extern "C" pq_status pq_linear_w4a4_host_batched(int n, const void *const *X_hos
         return rc == PQ_OK ? PQ_ERR_CUDA : rc;
     }
     return rc;
+}
+
+extern "C" pq_status pq_selftest_wait_expiry(void *ws, size_t ws_bytes, long long limit_cycles, int *observed,
+                                             void *stream) {
+    PQ_REQUIRE(ws && observed, PQ_ERR_NULL);
+    PQ_REQUIRE(ws_bytes >= sizeof(int), PQ_ERR_WORKSPACE);
+    PQ_REQUIRE(limit_cycles > 0 && limit_cycles <= 100000000ll, PQ_ERR_SHAPE);
+    wait_expiry_kernel<<<1, 32, 0, static_cast<cudaStream_t>(stream)>>>(static_cast<int *>(ws), limit_cycles, observed);
+    return pq_launch_status();
 }
 
 extern "C" pq_status pq_device_status(const void *ws, void *stream) {

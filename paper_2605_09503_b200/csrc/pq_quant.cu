@@ -302,12 +302,16 @@ pq_status quant_act_launch(const uint16_t *x, int64_t M, int64_t K, int64_t ld, 
     // The quantizer's blocks should be able to run on an SM beside a GEMM CTA (the batched linear
     // path overlaps the two kernels): ask for the GEMM's shared-memory carve-out, otherwise an SM
     // has to drain before it can switch between the two configurations.
-    static bool carveout_set = false;
-    if (!carveout_set) {
-        cudaFuncSetAttribute(quant_nvfp4_kernel<PQ_SF_TCGEN05, true, TILE_ROWS>, cudaFuncAttributePreferredSharedMemoryCarveout, 100);
-        cudaFuncSetAttribute(quant_nvfp4_kernel<PQ_SF_TCGEN05, false, TILE_ROWS>, cudaFuncAttributePreferredSharedMemoryCarveout, 100);
-        (void)cudaGetLastError();
-        carveout_set = true;
+    static PqPerDevice carveout;
+    const int dev = pq_device_slot();
+    if (dev >= 0) {
+        std::lock_guard<std::mutex> guard(carveout.lock);
+        if (!carveout.value[dev]) {
+            cudaFuncSetAttribute(quant_nvfp4_kernel<PQ_SF_TCGEN05, true, TILE_ROWS>, cudaFuncAttributePreferredSharedMemoryCarveout, 100);
+            cudaFuncSetAttribute(quant_nvfp4_kernel<PQ_SF_TCGEN05, false, TILE_ROWS>, cudaFuncAttributePreferredSharedMemoryCarveout, 100);
+            (void)cudaGetLastError();
+            carveout.value[dev] = 1;
+        }
     }
     if (sf_layout == PQ_SF_TCGEN05) {
         if (wide) PQ_CUDA_OK(pq::launch_dependent(quant_nvfp4_kernel<PQ_SF_TCGEN05, true, TILE_ROWS>, grid, block, 0, st, x, M, rows_idx, K, ld, ts_x, codes, sf));

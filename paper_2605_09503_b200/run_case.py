@@ -14,7 +14,7 @@ import torch
 
 from . import binding as B
 
-CASES = ["probe", "output_error", "norm_quant", "gemm", "quant", "linear", "batched", "stats", "error", "error_perm", "fakequant", "fakequant_perm", "quant_weight",
+CASES = ["output_error", "norm_quant", "gemm", "quant", "linear", "batched", "stats", "error", "error_perm", "fakequant", "fakequant_perm", "quant_weight",
          "quant_weight_perm", "select_perm"]
 
 
@@ -35,49 +35,6 @@ def main():
                     help="capture the timed launches in one CUDA graph (takes the host's launch rate out of the number)")
     args = ap.parse_args()
     dev = "cuda"
-    if args.case == "probe":
-        # per-SM L2 -> shared ingest and SM -> memory store rates, for several numbers of active SMs
-        src = torch.ones(64 << 20, dtype=torch.uint8, device=dev)                   # stays in L2
-        dst = torch.empty(148 * 2048 * 2048, dtype=torch.uint8, device=dev)
-        for ctas in (4, 16, 37, 74, 148):
-            B.pq_probe_sm_ingest(src, ctas, 50)                                      # warm L2
-            print(json.dumps({"case": "probe", "ctas": ctas,
-                              "ingest_B_per_clk_per_SM": round(B.pq_probe_sm_ingest(src, ctas, 2000), 1),
-                              "store_48KB_B_per_clk_per_SM": round(B.pq_probe_sm_store(dst, ctas, 24), 1),
-                              "store_4MB_B_per_clk_per_SM": round(B.pq_probe_sm_store(dst, ctas, 2048), 1)}))
-        sms = torch.cuda.get_device_properties(0).multi_processor_count
-        print(json.dumps({"case": "probe", "ctas": sms, "half_of_the_SMs": {
-            "one_SM_of_each_neighbouring_pair_B_per_clk": round(B.pq_probe_sm_ingest(src, sms, 2000, 1), 1),
-            "both_SMs_of_every_other_pair_B_per_clk": round(B.pq_probe_sm_ingest(src, sms, 2000, 2), 1)}}))
-        ctas2 = sms // 2 * 2
-        for fwd in (0, 700, 1400):
-            B.pq_probe_sm_forward(src, ctas2, 50, 0)
-            pull, push = B.pq_probe_sm_forward(src, ctas2, 2000, fwd)
-            print(json.dumps({"case": "probe", "ctas": ctas2, "pairs_forwarding_blocks": fwd,
-                              "ingest_B_per_clk_per_SM": round(pull, 1), "forwarded_B_per_clk_per_pair": round(push, 1)}))
-        # single-GPU extra (its own library, absent from multi-GPU runs): one multicast copy per cluster
-        import ctypes
-        import os
-        mc_path = os.path.join(os.path.dirname(B.LIB_PATH), "libpq_mc.so")
-        if os.path.exists(mc_path):
-            mc = ctypes.CDLL(mc_path)
-            mc.pq_probe_sm_ingest_multicast.argtypes = [ctypes.c_void_p, ctypes.c_size_t, ctypes.c_int, ctypes.c_int,
-                                                        ctypes.c_int, ctypes.c_int, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p]
-            cycles = torch.zeros(1, dtype=torch.int64, device=dev)
-            status = torch.zeros(1, dtype=torch.int32, device=dev)
-            for cluster in (1, 2, 4):
-                ctas = sms // cluster * cluster
-                line = {"case": "probe", "ctas": ctas, "multicast_cluster": cluster}
-                for handshake in (1, 0):
-                    for iters in (50, 2000):
-                        rc = mc.pq_probe_sm_ingest_multicast(src.data_ptr(), src.numel(), ctas, cluster, iters, handshake,
-                                                             cycles.data_ptr(), status.data_ptr(), None)
-                        torch.cuda.synchronize()
-                        assert rc == 0 and status.item() == 0, (rc, status.item())
-                    key = "received_B_per_clk_per_SM" + ("_with_stage_handshake" if handshake else "")
-                    line[key] = round(2000 * 32768 / max(int(cycles.item()), 1), 1)
-                print(json.dumps(line))
-        return
     M, N, K, R = args.M, args.N, args.K, args.rot
     g = torch.Generator(device=dev)
     g.manual_seed(0)

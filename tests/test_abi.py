@@ -68,6 +68,12 @@ def test_argument_errors_are_caught_on_the_host(L):
     assert L.pq_calib_stats(p, 8, 64, 64, p, p, p, 16, None) == 5                    # workspace
     assert L.pq_select_perm(p, 8, p, 8, 20000, 5, p, p, 1 << 30, None) == 2          # K too large
     assert L.pq_select_perm(p, 8, p, 8, 64, 0, p, p, 1 << 20, None) == 2             # J
+    assert L.pq_select_perm(p, 8, p, 8, 64, 5, p, None, 0, None) == 5                # the sort keys need a workspace
+    assert L.pq_select_perm(p, 8, p, 8, 64, 5, p, odd, 1 << 20, None) == 3           # ... 256-byte aligned
+    assert L.pq_order_by_absmax(p, 64, p, None, 0, None) == 5
+    assert L.pq_selftest_wait_expiry(None, 4, 1000, p, None) == 1
+    assert L.pq_selftest_wait_expiry(p, 4, 0, p, None) == 2                           # limit out of range
+    assert L.pq_selftest_wait_expiry(p, 4, 10 ** 12, p, None) == 2
     assert L.pq_group_error(p, 8, 64, 64, binding.pq_format(1, 4, 48), None, None, 1, p, p, 1 << 20, None) == 4
     assert L.pq_group_error(p, 8, 64, 64, binding.pq_format(0, 4, 16), None, None, 1, p, p, 1 << 20, None) == 1
     assert L.pq_group_error(p, 8, 64, 64, fmt4, None, None, 3, p, p, 1 << 20, None) == 2   # P>1 w/o perms

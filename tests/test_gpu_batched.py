@@ -105,15 +105,3 @@ def test_host_batched_equals_one_by_one():
     assert B.pq_device_status(ws) == B.PQ_OK
     for y, r in zip(yh, ref):
         assert torch.equal(y.view(torch.int16), r.view(torch.int16))
-
-
-def test_machine_probes_run_and_report_plausible_rates():
-    src = torch.ones(8 << 20, dtype=torch.uint8, device="cuda")
-    dst = torch.empty(8 * 64 * 2048, dtype=torch.uint8, device="cuda")
-    ingest = B.pq_probe_sm_ingest(src, 8, 200)
-    store = B.pq_probe_sm_store(dst, 8, 64)
-    assert 4.0 < ingest < 512.0 and 1.0 < store < 512.0          # bytes per clock per SM
-    pull, push = B.pq_probe_sm_forward(src, 8, 200, 50)
-    assert 1.0 < pull < 512.0 and 0.5 < push < 512.0
-    with pytest.raises(B.PqError):
-        B.pq_probe_sm_ingest(src[:1000], 8, 10)                   # region not a multiple of 32 KB

@@ -202,19 +202,24 @@ def all_partitions(K, g):
 def test_presorted_layer_is_rejected_and_clustered_outliers_accepted():
     rows, K, g = 64, 16, 4
     rng = np.random.default_rng(11)
-    scale_sorted = np.sort(rng.lognormal(0, 2, K))[::-1]
-    x_sorted = bf(rng.standard_normal((rows, K)) * scale_sorted[None, :])
+    x_any = bf(rng.standard_normal((rows, K)) * rng.lognormal(0, 2, K)[None, :])
+    S_any, _ = O.calib_stats(x_any)
+    # put the columns in descending order of their SAMPLED second moments (a column's sum moves with the
+    # column, bit for bit), so the layer is sorted in exactly the sense the criterion uses
+    x_sorted = np.ascontiguousarray(x_any[:, np.argsort(-S_any, kind="stable")])
     w = bf(np.ones((8, K)))                                   # weight side indifferent
     Sa, _ = O.calib_stats(x_sorted)
+    assert (np.diff(Sa) < 0).all()
     Sw, _ = O.calib_stats(w)
     perms = O.select_perm(Sa, rows, Sw, 8, J=5)
     cand = np.concatenate([np.arange(K, dtype=np.int32)[None], perms])
     ex = O.group_error(x_sorted, 1, 3, g, 1.0, cand)
     ew = O.group_error(w, 1, 3, g, 1.0, cand)
-    # sample second moments of a truly sorted layer are sorted too -> candidate = identity
-    if np.array_equal(perms[5], np.arange(K)):
-        _, acc, E = O.accept(ex, 1.0, ew, 0.0, 0.0)
-        assert acc == 0 and E[6] == E[0]                      # equal error: strict '>' rejects
+    # every candidate of a sorted layer is the original order again (the weight-only sort too: equal
+    # keys keep their order), so no candidate can lower the error and the strict '>' rejects
+    assert all(np.array_equal(p_, np.arange(K)) for p_ in perms)
+    _, acc, E = O.accept(ex, 1.0, ew, 0.0, 0.0)
+    assert acc == 0 and (E[1:] == E[0]).all()
     # one 8x channel per group in the original order drowns its three neighbours (their
     # share of a 4-bit grid spanning the large channel is ~1 level); sorting puts the four
     # large channels into one group and gives the small ones grids of their own -> accepted
