@@ -19,6 +19,10 @@
  *   - The producer of App. C (RMSNorm or adaptive LayerNorm with the channel reordering absorbed)
  *     with the NVFP4 quantizer attached: row statistics in fp32 over the original channel order,
  *     summed in the fixed 32-lane order stated at lane_order_sum.
+ *   - PermuQuant-H (App. D): the Hadamard transform x H in fp32 with the stated butterfly order, its
+ *     channels read through the permutation (x H P), then the NVFP4 quantizer.  The paper names the
+ *     transform only; the matrix (Sylvester, times Paley's order-12 matrix for widths 12 * 2^n), the
+ *     order of the additions and the 1/sqrt(K) scaling are readings stated at hadamard_row.
  *
  * Pins: see tests/test_oracle_*.py.  Every function here is pinned by hand-computed values,
  * closed forms, brute force on tiny inputs or an independent library routine, except the
@@ -480,6 +484,111 @@ int pqo_norm_quant_nvfp4(const uint16_t *H, int64_t rows, int64_t K, int64_t ld,
                 codes[t * (K / 2) + (k * 16 + j) / 2] = (uint8_t)(code[j] | (code[j + 1] << 4));
             if (y_bf16)
                 for (int j = 0; j < 16; ++j) y_bf16[t * K + k * 16 + j] = pqo_f32_to_bf16(g[j]);
+        }
+        free(x);
+    }
+    return fail;
+}
+
+/* ------------------------------------------------------------------ PermuQuant-H: Hadamard, reorder, quantize */
+
+/* Legendre symbol modulo 11: 0 for 0, +1 for the non-zero squares {1, 3, 4, 5, 9}, -1 otherwise. */
+static int legendre11(int r) {
+    r = ((r % 11) + 11) % 11;
+    if (r == 0) return 0;
+    for (int t = 1; t < 11; ++t)
+        if ((t * t) % 11 == r) return 1;
+    return -1;
+}
+
+/* The Hadamard matrix of order 12 by Paley's first construction for q = 11 (q = 3 mod 4):
+ * H = I + S with the skew matrix S = [[0, 1...1], [-1...-1 (column), Q]], Q[i][j] = chi(i - j). */
+static int hadamard12_entry(int i, int j) {
+    if (i == j) return 1;
+    if (i == 0) return 1;
+    if (j == 0) return -1;
+    return legendre11((i - 1) - (j - 1));
+}
+
+/* Which widths the transform is defined for here: K = 2^n (m = 1), or K = 12 * 2^n (m = 12). */
+static int hadamard_factor(int64_t K) {
+    if (K <= 0) return 0;
+    if ((K & (K - 1)) == 0) return 1;
+    if (K % 12 == 0 && ((K / 12) & (K / 12 - 1)) == 0) return 12;
+    return 0;
+}
+
+/* One row x[K] (in place): y = x (H_m (x) H_{2^n}) / sqrt(K), i.e. with the channel index written
+ * i = a * 2^n + b the matrix entry is H_m[a][a'] * (-1)^popcount(b & b').  fp32 throughout, in this
+ * order: (1) for m = 12, across the 12 segments: u[a'][b] = sum_a x[a][b] * H12[a][a'], the terms
+ * added one by one in ascending a (the first term is +-x[0][b] itself); (2) inside every segment the
+ * in-place butterflies of the fast Walsh-Hadamard transform, strides 1, 2, 4, ..., 2^(n-1):
+ * (x[i], x[i+h]) <- (x[i] + x[i+h], x[i] - x[i+h]) for every i with bit h clear; (3) one
+ * multiplication by fl(1 / sqrt(K)) (the double-precision value rounded to fp32). */
+static void hadamard_row(float *x, int64_t K, float *tmp) {
+    int m = hadamard_factor(K);
+    int64_t seg = K / m;
+    if (m == 12) {
+        for (int64_t b = 0; b < seg; ++b)
+            for (int ap = 0; ap < 12; ++ap) {
+                float acc = (hadamard12_entry(0, ap) > 0) ? x[b] : -x[b];
+                for (int a = 1; a < 12; ++a) {
+                    float v = x[a * seg + b];
+                    acc = (hadamard12_entry(a, ap) > 0) ? acc + v : acc - v;
+                }
+                tmp[ap * seg + b] = acc;
+            }
+        memcpy(x, tmp, sizeof(float) * (size_t)K);
+    }
+    for (int a = 0; a < m; ++a) {
+        float *s = x + a * seg;
+        for (int64_t h = 1; h < seg; h <<= 1)
+            for (int64_t i = 0; i < seg; ++i)
+                if (!(i & h)) {
+                    float p = s[i], q = s[i + h];
+                    s[i] = p + q;
+                    s[i + h] = p - q;
+                }
+    }
+    float scale = (float)(1.0 / sqrt((double)K));
+    for (int64_t i = 0; i < K; ++i) x[i] = x[i] * scale;
+}
+
+/* PermuQuant-H runtime producer (App. D): the Hadamard transform of every row, its channels read in
+ * the order `perm` (x H P: position j takes transformed channel perm[j]; NULL = transformed order),
+ * then the NVFP4 groups of that, quantized from the fp32 values.  codes / sf may be NULL (transform
+ * only); y_bf16 (optional) receives bf16 of the reordered transformed row, y_f32 (optional) the fp32
+ * values themselves.  Returns 2 for a width the transform is not defined for. */
+int pqo_hadamard_quant_nvfp4(const uint16_t *X, int64_t rows, int64_t K, int64_t ld, const int32_t *perm, float ts,
+                             uint8_t *codes, uint8_t *sf, uint16_t *y_bf16, float *y_f32) {
+    if (!X || rows <= 0 || K <= 0 || K % 16 != 0 || ld < K) return 1;
+    if ((codes == NULL) != (sf == NULL)) return 1;
+    if (!hadamard_factor(K)) return 2;
+    int fail = 0;
+#pragma omp parallel for schedule(static)
+    for (int64_t t = 0; t < rows; ++t) {
+        float *x = (float *)malloc(sizeof(float) * (size_t)K * 2);
+        if (!x) {
+            fail = 1;
+            continue;
+        }
+        for (int64_t i = 0; i < K; ++i) x[i] = pqo_bf16_to_f32(X[t * ld + i]);
+        hadamard_row(x, K, x + K);
+        for (int64_t k = 0; k < K / 16; ++k) {
+            float g[16], d;
+            uint8_t code[16], sf8;
+            for (int j = 0; j < 16; ++j) {
+                int64_t pos = k * 16 + j;
+                g[j] = x[perm ? perm[pos] : pos];
+                if (y_bf16) y_bf16[t * K + pos] = pqo_f32_to_bf16(g[j]);
+                if (y_f32) y_f32[t * K + pos] = g[j];
+            }
+            if (codes) {
+                nvfp4_group(g, 16, ts, &sf8, &d, code);
+                sf[t * (K / 16) + k] = sf8;
+                for (int j = 0; j < 16; j += 2)
+                    codes[t * (K / 2) + (k * 16 + j) / 2] = (uint8_t)(code[j] | (code[j + 1] << 4));
+            }
         }
         free(x);
     }

@@ -52,6 +52,7 @@ def _declare(L):
     L.pqo_quant_nvfp4.argtypes = [_P, _i64, _i64, _i64, _P, C.c_float, _P, _P]
     L.pqo_dequant_nvfp4.argtypes = [_P, _P, C.c_float, _i64, _i64, _P]
     L.pqo_norm_quant_nvfp4.argtypes = [_P, _i64, _i64, _i64, C.c_int, _P, _P, C.c_float, _P, C.c_float, _P, _P, _P]
+    L.pqo_hadamard_quant_nvfp4.argtypes = [_P, _i64, _i64, _i64, _P, C.c_float, _P, _P, _P, _P]
     L.pqo_fakequant_int.argtypes = [_P, _i64, _i64, _i64, C.c_int, C.c_int, _P, _P, _i64]
     L.pqo_gemm_ref_one.restype = C.c_double
     L.pqo_gemm_ref_one.argtypes = [_P, _P, C.c_float, _P, _P, C.c_float, _i64, _i64, _i64]
@@ -235,6 +236,21 @@ def norm_quant_nvfp4(H, kind, a, b, eps, ts, perm=None):
     _check(lib().pqo_norm_quant_nvfp4(_ptr(H), rows, K, K, kind, _ptr(a), _ptr(b), C.c_float(eps), _ptr(perm),
                                       C.c_float(ts), _ptr(codes), _ptr(sf), _ptr(y)), "norm_quant_nvfp4")
     return codes, sf, y
+
+
+def hadamard_quant_nvfp4(X, ts, perm=None, quantize=True):
+    """App. D: rows of X through the Hadamard transform, channels read in the order perm, NVFP4 groups of
+    the fp32 result.  -> (codes, sf, y_bf16 bits, y_f32); codes / sf are None with quantize=False."""
+    X = _bf16(X)
+    rows, K = X.shape
+    perm = _perm(perm, K)
+    codes = np.empty((rows, K // 2), dtype=np.uint8) if quantize else None
+    sf = np.empty((rows, K // 16), dtype=np.uint8) if quantize else None
+    y = np.empty((rows, K), dtype=np.uint16)
+    yf = np.empty((rows, K), dtype=np.float32)
+    _check(lib().pqo_hadamard_quant_nvfp4(_ptr(X), rows, K, K, _ptr(perm), C.c_float(ts), _ptr(codes), _ptr(sf), _ptr(y),
+                                          _ptr(yf)), "hadamard_quant_nvfp4")
+    return codes, sf, y, yf
 
 
 def dequant_nvfp4(codes, sf, ts):
