@@ -343,6 +343,28 @@ pq_status pq_norm_quant_nvfp4(const void *H, int64_t M, int64_t K, int64_t ld, i
                               const float *b, float eps, const int32_t *perm, const float *ts_x,
                               uint8_t *codes, uint8_t *sf, int sf_layout, void *y_out, void *stream);
 
+/* PermuQuant-H producer (App. D: reordering in the Hadamard-transformed basis, x H P): every row of X
+ * goes through the Hadamard transform, the transformed channels are read in the order `perm` (the
+ * transform itself is unchanged, only the order in which its outputs are consumed), and the result is
+ * quantized to NVFP4 exactly as pq_quant_act_nvfp4 quantizes a tensor, except that the quantizer sees
+ * the fp32 values.  The same call transforms weight rows (Wt H, written to y_out in bf16 and then fed
+ * to pq_calib_stats / pq_group_error / pq_quant_weight), since (x H)(Wt H)^T = x Wt^T.
+ *   Transform: K = m * 2^n with m = 1 or m = 12 (2^n >= 8); y = x (H_m (x) H_{2^n}) / sqrt(K), i.e. with
+ *   channel i = a * 2^n + b the matrix entry is H_m[a][a'] * (-1)^popcount(b & b'); H_12 = I + S is Paley's
+ *   matrix for q = 11: S[0][j] = 1, S[i][0] = -1, S[i][j] = chi(i - j) for i, j >= 1, chi the quadratic
+ *   character modulo 11.  (The paper names the transform only; matrix, order and scaling are this
+ *   library's reading.)  fp32 arithmetic in this order: the 12 segments combined first, terms added one
+ *   by one in ascending segment; then inside every segment the butterflies (x[i], x[i+h]) <-
+ *   (x[i] + x[i+h], x[i] - x[i+h]) with strides h = 1, 2, 4, ...; then one multiplication by
+ *   fl(1 / sqrt(K)).  Other widths return PQ_ERR_SHAPE.
+ *   X : bf16 [M, K], ld.  K % 16 == 0, K <= 16384 (K % 64 == 0 for codes in PQ_SF_TCGEN05).
+ *   perm : device int32 [K] or NULL (transformed order).  ts_x : device fp32 scalar (needed with codes).
+ *   codes, sf : as pq_quant_act_nvfp4, or both NULL to transform only (then y_out is required).
+ *   y_out : bf16 [M, K] contiguous or NULL; receives bf16 of the reordered transformed rows. */
+pq_status pq_hadamard_quant_nvfp4(const void *X, int64_t M, int64_t K, int64_t ld, const int32_t *perm,
+                                  const float *ts_x, uint8_t *codes, uint8_t *sf, int sf_layout,
+                                  void *y_out, void *stream);
+
 /* Integer fake-quant of Eq. 1-2 (quantize, dequantize, round to bf16), optional gather.
  *   T : bf16 [rows, K], ld.  out : bf16 [rows, K], ldo.  perm : int32 [K] or NULL.
  *   fmt.kind must be 1; K % fmt.group == 0; K <= 16384 when perm != NULL. */

@@ -64,6 +64,7 @@ _SIGNATURES = {
     "pq_sf_to_linear": (_int, [_vp, _i64, _i64, _vp, _vp]),
     "pq_norm_quant_nvfp4": (_int, [_vp, _i64, _i64, _i64, _int, _vp, _vp, C.c_float, _vp, _vp, _vp, _vp, _int, _vp,
                                    _vp]),
+    "pq_hadamard_quant_nvfp4": (_int, [_vp, _i64, _i64, _i64, _vp, _vp, _vp, _vp, _int, _vp, _vp]),
     "pq_last_error_detail": (C.c_char_p, []),
     "pq_device_status": (_int, [_vp, _vp]),
     "pq_selftest_wait_expiry": (_int, [_vp, _sz, C.c_longlong, _vp, _vp]),
@@ -333,6 +334,19 @@ def pq_norm_quant_nvfp4(H, kind, a, b, eps, perm, ts_x, codes, sf, sf_layout, y_
     assert y_out is None or (y_out.dtype == torch.bfloat16 and y_out.shape == (M, K) and y_out.is_contiguous())
     _check("pq_norm_quant_nvfp4", lib().pq_norm_quant_nvfp4(_p(H), M, K, H.stride(0), kind, _p(a), _p(b), eps, _p(perm),
                                                             _p(ts_x), _p(codes), _p(sf), sf_layout, _p(y_out), _stream()))
+
+
+def pq_hadamard_quant_nvfp4(X, perm, ts_x, codes, sf, sf_layout, y_out=None):
+    """Rows of X through the Hadamard transform, channels read in the order perm, NVFP4 codes and scales of
+    the result (codes = sf = None: transform only, into y_out)."""
+    _bf16(X)
+    M, K = X.shape
+    assert perm is None or (perm.dtype == torch.int32 and perm.numel() == K and perm.is_contiguous())
+    assert (codes is None) == (sf is None)
+    assert codes is None or (codes.dtype == torch.uint8 and sf.dtype == torch.uint8 and ts_x.dtype == torch.float32)
+    assert y_out is None or (y_out.dtype == torch.bfloat16 and y_out.shape == (M, K) and y_out.is_contiguous())
+    _check("pq_hadamard_quant_nvfp4", lib().pq_hadamard_quant_nvfp4(_p(X), M, K, X.stride(0), _p(perm), _p(ts_x),
+                                                                    _p(codes), _p(sf), sf_layout, _p(y_out), _stream()))
 
 
 def pq_device_status(ws):

@@ -97,7 +97,10 @@ constexpr int kTmemCols = 512;
 // iteration it - kStages (stage_free, which the producer waited for before it refilled the stage)
 // in front of the sf_ready wait, so that wait is sound whatever the slot count; the assertion below
 // keeps the original condition as well.
-constexpr int kSfSlots = 2;
+#ifndef PQ_GEMM_SLOTS
+#define PQ_GEMM_SLOTS 2
+#endif
+constexpr int kSfSlots = PQ_GEMM_SLOTS;
 constexpr uint32_t kSfSlotCol0 = BN, kSfSlotCols = 4 * (4 + 8), kSfbOfs = 16;
 static_assert(kSfSlotCol0 + kSfSlots * kSfSlotCols <= 512, "tensor memory columns");
 static_assert(kSfSlots + 2 <= kStages, "a stager set must know that the previous phase of sf_ready has completed");
@@ -334,11 +337,29 @@ constexpr uint32_t kIdesc = (1u << 7) | (1u << 10) | (static_cast<uint32_t>(BN >
 __device__ __forceinline__ uint32_t sf_slot_col(uint32_t t) { return kSfSlotCol0 + t * kSfSlotCols; }
 
 // Two accumulator values times alpha, each rounded to bf16 (nearest even), packed low | high.
+#ifndef PQ_GEMM_EPI_PACKED
+#define PQ_GEMM_EPI_PACKED 1
+#endif
 __device__ __forceinline__ uint32_t pack_bf16(uint32_t lo_bits, uint32_t hi_bits, float alpha) {
+    uint32_t r;
+#if PQ_GEMM_EPI_PACKED
+    // one packed multiply (two IEEE products per issue slot), then the two-way convert
+    asm("{\n"
+        ".reg .b64 v, a;\n"
+        ".reg .f32 lo, hi;\n"
+        "mov.b64 v, {%1, %2};\n"
+        "mov.b64 a, {%3, %3};\n"
+        "mul.rn.f32x2 v, v, a;\n"
+        "mov.b64 {lo, hi}, v;\n"
+        "cvt.rn.bf16x2.f32 %0, hi, lo;\n"
+        "}\n"
+        : "=r"(r)
+        : "r"(lo_bits), "r"(hi_bits), "f"(alpha));
+#else
     const float lo = __fmul_rn(__uint_as_float(lo_bits), alpha);
     const float hi = __fmul_rn(__uint_as_float(hi_bits), alpha);
-    uint32_t r;
     asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+#endif
     return r;
 }
 

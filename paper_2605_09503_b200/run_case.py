@@ -14,7 +14,7 @@ import torch
 
 from . import binding as B
 
-CASES = ["output_error", "norm_quant", "gemm", "quant", "linear", "batched", "stats", "error", "error_perm", "fakequant", "fakequant_perm", "quant_weight",
+CASES = ["hadamard", "output_error", "norm_quant", "gemm", "quant", "linear", "batched", "stats", "error", "error_perm", "fakequant", "fakequant_perm", "quant_weight",
          "quant_weight_perm", "select_perm"]
 
 
@@ -86,6 +86,13 @@ def main():
         bytes_moved = M * K * 2 + M * K // 2 + M * K // 16
         fn = lambda i: B.pq_norm_quant_nvfp4(X[i % R], args.kind, av, bv, 1e-6, pm, ts, xq[i % R], sfx[i % R],
                                              B.PQ_SF_TCGEN05)
+    elif args.case == "hadamard":
+        X = [acts(M) for _ in range(R)]
+        xq = [torch.empty(M, K // 2, dtype=torch.uint8, device=dev) for _ in range(R)]
+        sfx = [torch.empty(B.sf_bytes(M, K, 1), dtype=torch.uint8, device=dev) for _ in range(R)]
+        pm = perms[0].contiguous()
+        bytes_moved = M * K * 2 + M * K // 2 + M * K // 16
+        fn = lambda i: B.pq_hadamard_quant_nvfp4(X[i % R], pm, ts, xq[i % R], sfx[i % R], B.PQ_SF_TCGEN05)
     elif args.case == "quant":
         X = [acts(M) for _ in range(R)]
         xq = [torch.empty(M, K // 2, dtype=torch.uint8, device=dev) for _ in range(R)]

@@ -1,0 +1,115 @@
+"""GPU parity of the PermuQuant-H producer (App. D: Hadamard transform, reordered read-out, NVFP4 quantizer)
+against the oracle: codes, scale bytes and the bf16 output bit for bit; and the layer identity
+(x H P)(Wt H P)^T = x Wt^T through the W4A4 GEMM."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import pq_oracle as O
+from paper_2605_09503_b200 import binding as B
+from paper_2605_09503_b200 import inputs
+from test_gpu_gemm import assert_close, to_tc
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda"
+
+
+def _case(M, K, seed):
+    g = torch.Generator().manual_seed(seed)
+    scale = torch.exp(1.5 * torch.randn(K, generator=g))
+    x = (torch.randn(M, K, generator=g) * scale).to(torch.bfloat16)
+    perm = torch.randperm(K, generator=g).to(torch.int32)
+    return x, perm
+
+
+# widths: powers of two (one pass, two passes, none), 12 * 2^n (FLUX: 3072 and 12288), ragged row counts
+@pytest.mark.parametrize("layout", [B.PQ_SF_LINEAR, B.PQ_SF_TCGEN05])
+@pytest.mark.parametrize("M,K,with_perm", [(37, 3072, True), (130, 3072, False), (9, 12288, True), (300, 1024, True),
+                                           (5, 64, False), (23, 1536, True), (17, 192, True), (3, 16384, True),
+                                           (70, 256, True), (12, 768, True), (1, 4096, True)])
+def test_hadamard_quant_bit_exact(layout, M, K, with_perm):
+    x, perm = _case(M, K, seed=M + K)
+    ts = 0.02
+    codes = torch.empty(M, K // 2, dtype=torch.uint8, device=DEV)
+    sf = torch.full((B.sf_bytes(M, K, layout),), 0xEE, dtype=torch.uint8, device=DEV)
+    y = torch.empty(M, K, dtype=torch.bfloat16, device=DEV)
+    B.pq_hadamard_quant_nvfp4(x.to(DEV), perm.to(DEV) if with_perm else None,
+                              torch.tensor([ts], dtype=torch.float32, device=DEV), codes, sf, layout, y)
+    c_o, s_o, y_o, _ = O.hadamard_quant_nvfp4(inputs.bits(x), ts, perm.numpy() if with_perm else None)
+    assert np.array_equal(inputs.bits(y.cpu()), y_o)
+    assert np.array_equal(codes.cpu().numpy(), c_o)
+    if layout == B.PQ_SF_LINEAR:
+        assert np.array_equal(sf.cpu().numpy().reshape(M, K // 16), s_o)
+    else:
+        assert np.array_equal(sf.cpu().numpy(), to_tc(s_o))      # padding rows hold zero scale bytes
+
+
+def test_transform_only_and_small_widths():
+    for M, K in ((7, 16), (4, 32), (33, 96), (2, 48 * 4)):
+        x, perm = _case(M, K, seed=K)
+        y = torch.empty(M, K, dtype=torch.bfloat16, device=DEV)
+        B.pq_hadamard_quant_nvfp4(x.to(DEV), perm.to(DEV), None, None, None, B.PQ_SF_LINEAR, y)
+        _, _, y_o, _ = O.hadamard_quant_nvfp4(inputs.bits(x), 1.0, perm.numpy(), quantize=False)
+        assert np.array_equal(inputs.bits(y.cpu()), y_o)
+    x, _ = _case(4, 80, seed=1)                                   # 5 * 16: no transform defined for it
+    with pytest.raises(B.PqError):
+        B.pq_hadamard_quant_nvfp4(x.to(DEV), None, None, None, None, B.PQ_SF_LINEAR,
+                                  torch.empty(4, 80, dtype=torch.bfloat16, device=DEV))
+    with pytest.raises(B.PqError):                                # 12 * 4: segments shorter than one 16-byte load
+        B.pq_hadamard_quant_nvfp4(x[:, :48].contiguous().to(DEV), None, None, None, None, B.PQ_SF_LINEAR,
+                                  torch.empty(4, 48, dtype=torch.bfloat16, device=DEV))
+
+
+def test_strided_rows():
+    M, K = 40, 3072
+    x, perm = _case(M, 2 * K, seed=9)
+    xv = x.to(DEV)[:, :K]                                        # leading dimension 2 K
+    codes = torch.empty(M, K // 2, dtype=torch.uint8, device=DEV)
+    sf = torch.empty(M * K // 16, dtype=torch.uint8, device=DEV)
+    p = torch.randperm(K, generator=torch.Generator().manual_seed(3)).to(torch.int32)
+    B.pq_hadamard_quant_nvfp4(xv, p.to(DEV), torch.tensor([0.05], dtype=torch.float32, device=DEV), codes, sf,
+                              B.PQ_SF_LINEAR, None)
+    c_o, s_o, _, _ = O.hadamard_quant_nvfp4(inputs.bits(x[:, :K].contiguous()), 0.05, p.numpy())
+    assert np.array_equal(codes.cpu().numpy(), c_o) and np.array_equal(sf.cpu().numpy().reshape(M, K // 16), s_o)
+
+
+def test_transformed_layer_reproduces_the_plain_product():
+    """PermuQuant-H end to end on a small layer: activations and weight rows go through the same transform
+    and the same order, so the quantized product approximates x Wt^T, and the GEMM on the transformed
+    operands equals the fp64 reference built from the oracle's transformed codes."""
+    cfg = inputs.CONFIGS["tiny"]
+    M, K, N = 256, 512, 384
+    x, perm = _case(M, K, seed=21)
+    w = (0.02 * torch.randn(N, K, generator=torch.Generator().manual_seed(22))).to(torch.bfloat16)
+    d = lambda t: t.to(DEV)
+    # weight side: transform rows, then the ordinary permuted weight quantizer
+    wh = torch.empty(N, K, dtype=torch.bfloat16, device=DEV)
+    B.pq_hadamard_quant_nvfp4(d(w), None, None, None, None, B.PQ_SF_LINEAR, wh)
+    wq = torch.empty(N, K // 2, dtype=torch.uint8, device=DEV)
+    sfw = torch.empty(B.sf_bytes(N, K, 1), dtype=torch.uint8, device=DEV)
+    ts_w = torch.empty(1, dtype=torch.float32, device=DEV)
+    B.pq_quant_weight(wh, d(perm), None, wq, sfw, B.PQ_SF_TCGEN05, ts_w, B.workspace(B.OP_QUANT_WEIGHT, N, K))
+    # activation side: transform + order + quantize in one kernel, tensor scale from the transformed absmax
+    xh = torch.empty(M, K, dtype=torch.bfloat16, device=DEV)
+    B.pq_hadamard_quant_nvfp4(d(x), None, None, None, None, B.PQ_SF_LINEAR, xh)
+    ts_x = (xh.float().abs().max() / 2688.0).reshape(1).contiguous()
+    xq = torch.empty(M, K // 2, dtype=torch.uint8, device=DEV)
+    sfx = torch.empty(B.sf_bytes(M, K, 1), dtype=torch.uint8, device=DEV)
+    B.pq_hadamard_quant_nvfp4(d(x), d(perm), ts_x, xq, sfx, B.PQ_SF_TCGEN05, None)
+    Y = torch.empty(M, N, dtype=torch.bfloat16, device=DEV)
+    ws = B.workspace(B.OP_GEMM, M, K, N)
+    B.pq_gemm_w4a4(xq, sfx, ts_x, wq, sfw, ts_w, Y, ws)
+    assert B.pq_device_status(ws) == B.PQ_OK
+    # oracle route for the same operands
+    _, _, wh_o, _ = O.hadamard_quant_nvfp4(inputs.bits(w), 1.0, quantize=False)
+    assert np.array_equal(inputs.bits(wh.cpu()), wh_o)
+    tsw_o = O.tensor_scale(O.calib_stats(wh_o)[1])
+    wq_o, sfw_o = O.quant_nvfp4(wh_o, tsw_o, perm.numpy())
+    xq_o, sfx_o, _, _ = O.hadamard_quant_nvfp4(inputs.bits(x), float(ts_x.item()), perm.numpy())
+    assert np.array_equal(xq.cpu().numpy(), xq_o) and np.array_equal(wq.cpu().numpy(), wq_o)
+    ref = O.gemm_ref(xq_o, sfx_o, float(ts_x.item()), wq_o, sfw_o, tsw_o)
+    assert_close(Y.float().cpu().numpy().astype(np.float64), ref)
+    # and the transformed, quantized layer is close to the unquantized product (the rotation cancels)
+    plain = x.double().numpy() @ w.double().numpy().T
+    rel = np.linalg.norm(ref - plain) / np.linalg.norm(plain)
+    assert rel < 0.15, rel
