@@ -2,6 +2,7 @@
 import os
 import socket
 
+import pytest
 import torch
 import torch.distributed as dist
 import torch.multiprocessing as mp
@@ -94,3 +95,19 @@ def test_calibration_partials_combine_in_rank_order():
         assert torch.equal(S, S_want) and torch.equal(E, E_want) and torch.equal(A, A_want)
         assert rows == 1000 + 1001 + 1002
     assert not torch.equal(S_want, got[0][1] + (got[1][1] + got[2][1]))   # the case does depend on the order
+
+
+def test_bench_starts_its_own_ranks():
+    """`python bench.py --gpus 2` without a launcher starts two ranks itself (torch.distributed.run on
+    127.0.0.1).  On a machine without a GPU each rank must stop at the explicit "needs a CUDA device"
+    exit (there is no CPU fallback), which shows that both ranks were started and reached the GPU arm."""
+    import subprocess
+    import sys
+    if torch.cuda.is_available():
+        pytest.skip("the two ranks would run the whole benchmark")
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    env = {k: v for k, v in os.environ.items() if k not in ("WORLD_SIZE", "RANK", "LOCAL_RANK")}
+    out = subprocess.run([sys.executable, os.path.join(root, "bench.py"), "--gpus", "2", "--steps", "2", "--warmup", "1"],
+                         env=env, capture_output=True, text=True, timeout=600)
+    assert out.returncode != 0
+    assert (out.stdout + out.stderr).count("bench.py needs a CUDA device") == 2
