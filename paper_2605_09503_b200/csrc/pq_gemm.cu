@@ -47,8 +47,9 @@
 // The 256 B-scale rows of a tile are two whole blocks: 8 columns per K block.
 //
 // Cross-CTA signalling uses plain remote mbarrier arrives and, for the completion of a stage's
-// MMAs, one tcgen05.commit per CTA (the leader's epilogue passes accumulator completions on).  Every wait on an mbarrier is bounded.  If one expires the CTA
-// records PQ_ERR_TIMEOUT in the status word, raises a shared abort flag that every role polls,
+// MMAs and of a tile's accumulator, one tcgen05.commit per CTA (issued by the pair leader's MMA
+// warp onto each CTA's own copy of the barrier).  Every wait on an mbarrier is bounded.  If one
+// expires the CTA records PQ_ERR_TIMEOUT in the status word, raises a shared abort flag that every role polls,
 // and falls through to the common teardown (cluster barrier, tensor-memory release).
 #include <cuda.h>
 
@@ -58,24 +59,29 @@
 
 namespace {
 
-constexpr int BM = 256, BM_CTA = 128, BN = 256, BN_CTA = BN / 2, BK = 256;
-constexpr int kStages = 5;
+constexpr int BM = 256, BM_CTA = 128, BK = 256;
 constexpr int kABytes = BM_CTA * BK / 2;   // 16384
-constexpr int kBBytes = BN_CTA * BK / 2;   // 16384
 constexpr int kSfBlock = 512;              // 128 rows x 4 groups
 constexpr int kSfaBytes = 4 * kSfBlock;    // 4 K-blocks of one 128-row block
-constexpr int kSfbBytes = 2 * kSfaBytes;   // two 128-row blocks
-constexpr int kStageBytes = kABytes + kBBytes + kSfaBytes + kSfbBytes;  // 38912 = 38 * 1024
-constexpr int kEpiBox = 32 * 128;          // 32 rows x 64 bf16, one TMA store
-constexpr int kEpiWarps = 8;               // lane quadrant x column half of the accumulator
-constexpr int kEpiBytes = kEpiWarps * kEpiBox;      // one staging box per epilogue warp: 32 KB
-constexpr int kFirstStager = 2 + kEpiWarps;
-constexpr int kThreads = 32 * (kFirstStager + 8);   // producer, MMA issuer, 8 epilogue and 8 stager warps
 constexpr int kTmemCols = 512;
-// One 256-column accumulator, then the scale slots.  A slot holds the scales of one stage: per
-// 64-channel K block 4 columns of A scales (128 rows) and 8 columns of B scales (256 rows).  Slot
-// it % kSfSlots serves iteration it; it is rewritten only after the MMAs of iteration it - kSfSlots
-// have completed (their commit releases that iteration's stage).
+constexpr long long kWaitCycles = 4000000000ll;  // default limit of a wait: about two seconds of SM clock
+
+constexpr int BN = 256, BN_CTA = BN / 2;
+constexpr int kStages = 5;
+constexpr int kBBytes = BN_CTA * BK / 2;   // 16384
+constexpr int kSfbBytes = 2 * kSfaBytes;   // the two 128-row blocks of the tile's 256 B rows
+constexpr int kStageBytes = kABytes + kBBytes + kSfaBytes + kSfbBytes;  // 38912 = 38 * 1024
+constexpr int kEpiWarps = 8;               // lane quadrant x column half of the accumulator
+constexpr int kBoxCols = 64;               // output staging box: 32 rows x 64 bf16, one TMA store
+constexpr int kEpiBox = 32 * kBoxCols * 2;
+constexpr int kEpiBytes = kEpiWarps * kEpiBox;      // one staging box per epilogue warp: 32 KB
+constexpr int kStagerSets = 2;             // sets of four stager warps taking alternate K iterations
+constexpr int kFirstStager = 2 + kEpiWarps;
+constexpr int kThreads = 32 * (kFirstStager + 4 * kStagerSets);   // producer, MMA issuer, 8 epilogue and 8 stager warps
+// One 256-column accumulator, then the scale slots.  A slot holds the scales of one stage: per 64-channel
+// K block 4 columns of A scales (128 rows) and 8 columns of B scales (256 rows).  Slot it % kSfSlots
+// serves iteration it; it is rewritten only after the MMAs of iteration it - kSfSlots have completed
+// (their commit releases that iteration's stage).
 //
 // Why the slot count is tied to the stage count.  Every wait here is a PARITY wait: it tells "phase n
 // of this barrier has completed" from "it has not" only if the barrier cannot still be in phase n - 1,
@@ -84,31 +90,29 @@ constexpr int kTmemCols = 512;
 // epilogue warp on acc_full) knows it from its own previous wait.  The stagers do not: the stage
 // count is odd and the two stager sets take alternate iterations, so the previous phase of
 // sf_ready(s), iteration it - kStages, was waited for by the OTHER set.  What a set knows when it
-// reaches iteration `it` is what its own iteration it - 2 waited for: the MMAs of it - 2 - kSfSlots
-// have completed.  Those of it - kStages (hence that iteration's scale copies, which its stagers had
-// to see before its MMAs could be issued) are then known complete only if
-//     it - 2 - kSfSlots >= it - kStages,   i.e.  kSfSlots + 2 <= kStages.
-// With 4 slots and 5 stages the condition fails: when the scale copies of it - kStages were still in
-// flight the wait for phase n returned true one phase early, the warp read the previous occupant's
-// scale bytes from shared memory and stored them to tensor memory -- one lane quadrant of one CTA,
-// all columns, wrong by the ratio of two scale factors -- about once in 450 launches of the
+// reaches iteration `it` is what its own iteration it - kStagerSets waited for: the MMAs of
+// it - kStagerSets - kSfSlots have completed.  Those of it - kStages (hence that iteration's scale
+// copies, which its stagers had to see before its MMAs could be issued) are then known complete only if
+//     it - kStagerSets - kSfSlots >= it - kStages,   i.e.  kSfSlots + kStagerSets <= kStages.
+// With 4 slots, 2 sets and 5 stages the condition fails: when the scale copies of it - kStages were
+// still in flight the wait for phase n returned true one phase early, the warp read the previous
+// occupant's scale bytes from shared memory and stored them to tensor memory -- one lane quadrant of
+// one CTA, all columns, wrong by the ratio of two scale factors -- about once in 450 launches of the
 // 4608 x 3072 x 9216 product.  2 and 3 slots, and 4 slots with the stagers held to three stages
-// ahead, satisfy the condition and never failed.  The stagers now also wait for the release of
-// iteration it - kStages (stage_free, which the producer waited for before it refilled the stage)
-// in front of the sf_ready wait, so that wait is sound whatever the slot count; the assertion below
-// keeps the original condition as well.
-#ifndef PQ_GEMM_SLOTS
-#define PQ_GEMM_SLOTS 2
-#endif
-constexpr int kSfSlots = PQ_GEMM_SLOTS;
-constexpr uint32_t kSfSlotCol0 = BN, kSfSlotCols = 4 * (4 + 8), kSfbOfs = 16;
+// ahead, satisfy the condition and never failed.  The stagers also wait for the release of iteration
+// it - kStages (stage_free, which the producer waited for before it refilled the stage) in front of
+// the sf_ready wait, so that wait is sound whatever the slot count; the assertions keep the original
+// condition as well.
+constexpr int kSfSlots = 2;
+constexpr uint32_t kSfSlotCol0 = BN, kSfbColsPerKb = 8, kSfbOfs = 16;
+constexpr uint32_t kSfSlotCols = 4 * (4 + kSfbColsPerKb);   // 48
 static_assert(kSfSlotCol0 + kSfSlots * kSfSlotCols <= 512, "tensor memory columns");
-static_assert(kSfSlots + 2 <= kStages, "a stager set must know that the previous phase of sf_ready has completed");
+static_assert(kSfSlots + kStagerSets <= kStages, "a stager set must know that the previous phase of sf_ready has completed");
 static_assert(kSfSlots <= 2 * kStages - 2, "the stagers' parity waits on stage_free must be unambiguous");
-constexpr long long kWaitCycles = 4000000000ll;  // default limit of a wait: about two seconds of SM clock
 // barriers: stage_full[S] sf_ready[S] stage_free[S] acc_full acc_empty
 constexpr int kNumBars = 3 * kStages + 2;
 constexpr size_t kSmemBytes = kStages * kStageBytes + kEpiBytes + 1024 /*alignment slack*/ + 8 * kNumBars + 64;
+static_assert(kSmemBytes <= 227 * 1024, "shared memory per CTA");
 
 struct GemmParams {
     const uint8_t *sfx, *sfw;
@@ -309,11 +313,6 @@ __device__ __forceinline__ void tc_st4(uint32_t taddr, const uint4 &v) {
 __device__ __forceinline__ void tc_st2(uint32_t taddr, uint32_t a, uint32_t b) {
     asm volatile("tcgen05.st.sync.aligned.32x32b.x2.b32 [%0], {%1, %2};" ::"r"(taddr), "r"(a), "r"(b) : "memory");
 }
-// Eight columns of B scales of one K block: the two 128-row blocks of the tile's 256 rows.
-__device__ __forceinline__ void stage_b_scales(uint32_t taddr, const uint4 &b0, const uint4 &b1) {
-    tc_st4(taddr, b0);
-    tc_st4(taddr + 4, b1);
-}
 __device__ __forceinline__ void tc_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ uint4 lds128(uint32_t addr) {
     uint4 v;
@@ -334,7 +333,6 @@ __device__ __forceinline__ uint64_t operand_desc(uint32_t smem_addr) {
 constexpr uint32_t kIdesc = (1u << 7) | (1u << 10) | (static_cast<uint32_t>(BN >> 3) << 17) | (0u << 23) |
                             (static_cast<uint32_t>(BM >> 4) << 24);
 
-__device__ __forceinline__ uint32_t sf_slot_col(uint32_t t) { return kSfSlotCol0 + t * kSfSlotCols; }
 
 // Two accumulator values times alpha, each rounded to bf16 (nearest even), packed low | high.
 #ifndef PQ_GEMM_EPI_PACKED
@@ -372,6 +370,7 @@ constexpr int kMaxRegs = 96;
 __global__ void __cluster_dims__(2, 1, 1) __maxnreg__(kMaxRegs)
 gemm_w4a4_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                  const __grid_constant__ CUtensorMap map_y, const GemmParams p) {
+    constexpr int kNB = BN / 128;  // 128-row scale blocks of B per tile
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t base = (raw + 1023u) & ~1023u;  // identical in both CTAs of the pair
@@ -384,12 +383,12 @@ gemm_w4a4_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
     auto stage_full_bar = [&](int s) { return bars + 8u * s; };
     auto sf_ready_bar = [&](int s) { return bars + 8u * (kStages + s); };     // scale blocks landed (own CTA)
     auto stage_free_bar = [&](int s) { return bars + 8u * (2 * kStages + s); };  // the stage's MMAs have run
-    const uint32_t acc_full_bar = bars + 8u * (3 * kStages);
+    const uint32_t acc_full_bar = bars + 8u * (3 * kStages);       // one copy per CTA, both signalled by the issuer
     const uint32_t acc_empty_bar = bars + 8u * (3 * kStages + 1);  // leader's copy only
     uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars_ptr + 8 * kNumBars);
     volatile int *abort_flag = reinterpret_cast<volatile int *>(bars_ptr + 8 * kNumBars + 8);
-
     const WaitCtx wctx{abort_flag, p.status, p.wait_cycles};
+    auto sf_slot_col = [](uint32_t t) { return kSfSlotCol0 + t * kSfSlotCols; };
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t rank = cluster_ctarank();  // 0 = pair leader
@@ -440,10 +439,11 @@ gemm_w4a4_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
             const int n0 = n_blk * BN;
             const int ra = min(m0 >> 7, p.m_rowblocks - 1);
             const int nb0 = n0 >> 7;
-            const int rb0 = min(nb0, p.n_rowblocks - 1), rb1 = min(nb0 + 1, p.n_rowblocks - 1);
             const uint8_t *sfa_src = p.sfx + static_cast<int64_t>(ra) * p.kb4 * kSfBlock;
-            const uint8_t *sfb0_src = p.sfw + static_cast<int64_t>(rb0) * p.kb4 * kSfBlock;
-            const uint8_t *sfb1_src = p.sfw + static_cast<int64_t>(rb1) * p.kb4 * kSfBlock;
+            const uint8_t *sfb_src[kNB];
+#pragma unroll
+            for (int j = 0; j < kNB; ++j)
+                sfb_src[j] = p.sfw + static_cast<int64_t>(min(nb0 + j, p.n_rowblocks - 1)) * p.kb4 * kSfBlock;
             for (int kt = 0; kt < p.k_tiles; ++kt, ++it) {
                 const int s = it % kStages;
                 const uint32_t par = (it / kStages) & 1u;
@@ -452,14 +452,16 @@ gemm_w4a4_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
                 const int kb_valid = min(4, p.kb_total - kt * 4);
                 const uint32_t sf_bytes = static_cast<uint32_t>(kb_valid) * kSfBlock;
                 const uint32_t stage = base + s * kStageBytes;
+                const uint32_t sf_stage = stage + kABytes + kBBytes;
                 const uint32_t full_leader = mapa(stage_full_bar(s), 0);
                 const int64_t kofs = static_cast<int64_t>(kt) * 4 * kSfBlock;
                 if (elect_one()) {
                     if (rank == 0) mbar_expect_tx(stage_full_bar(s), 2u * (kABytes + kBBytes));
-                    mbar_expect_tx(sf_ready_bar(s), 3u * sf_bytes);
-                    bulk_load(stage + kABytes + kBBytes, sfa_src + kofs, sf_bytes, sf_ready_bar(s));
-                    bulk_load(stage + kABytes + kBBytes + kSfaBytes, sfb0_src + kofs, sf_bytes, sf_ready_bar(s));
-                    bulk_load(stage + kABytes + kBBytes + 2 * kSfaBytes, sfb1_src + kofs, sf_bytes, sf_ready_bar(s));
+                    mbar_expect_tx(sf_ready_bar(s), (1u + kNB) * sf_bytes);
+                    bulk_load(sf_stage, sfa_src + kofs, sf_bytes, sf_ready_bar(s));
+#pragma unroll
+                    for (int j = 0; j < kNB; ++j)
+                        bulk_load(sf_stage + (1 + j) * kSfaBytes, sfb_src[j] + kofs, sf_bytes, sf_ready_bar(s));
                     tma_load_2d_pair(stage, &map_a, kt * (BK / 2), m0, full_leader);
                     tma_load_2d_pair(stage + kABytes, &map_b, kt * (BK / 2), n0 + static_cast<int>(rank) * BN_CTA,
                                      full_leader);
@@ -497,19 +499,21 @@ gemm_w4a4_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
                     const uint32_t sfa_t = tmem_base + sf_slot_col(t), sfb_t = sfa_t + kSfbOfs;
                     const int kb_valid = min(4, p.kb_total - kt * 4);
                     if (elect_one()) {
-                        if (kb_valid == 4) {
-                            tc_mma_pair(d_tmem, da, db, kIdesc, sfa_t, sfb_t, acc);
-                            tc_mma_pair(d_tmem, da + 2, db + 2, kIdesc, sfa_t + 4, sfb_t + 8, 1u);
-                            tc_mma_pair(d_tmem, da + 4, db + 4, kIdesc, sfa_t + 8, sfb_t + 16, 1u);
-                            tc_mma_pair(d_tmem, da + 6, db + 6, kIdesc, sfa_t + 12, sfb_t + 24, 1u);
-                        } else {
-                            for (int kk = 0; kk < kb_valid; ++kk)
-                                tc_mma_pair(d_tmem, da + 2 * kk, db + 2 * kk, kIdesc, sfa_t + 4 * kk, sfb_t + 8 * kk,
-                                            acc | static_cast<uint32_t>(kk));
+#pragma unroll
+                        for (int kk = 0; kk < 4; ++kk) {
+                            if (kk < kb_valid) {
+                                const uint32_t accumulate = acc | static_cast<uint32_t>(kk);
+                                tc_mma_pair(d_tmem, da + 2 * kk, db + 2 * kk, kIdesc, sfa_t + 4 * kk,
+                                            sfb_t + kSfbColsPerKb * kk, accumulate);
+                            }
                         }
                         // the stage (and its scale slot) is free in both CTAs once these MMAs have run
                         tc_commit_pair(stage_free_bar(s));
                         tc_commit_pair(stage_free_bar(s) + peer);
+                        if (kt == p.k_tiles - 1) {  // ... and with them the tile's accumulator is complete
+                            tc_commit_pair(acc_full_bar);
+                            tc_commit_pair(acc_full_bar + peer);
+                        }
                     }
                     __syncwarp();
                     acc = 1u;
@@ -517,8 +521,6 @@ gemm_w4a4_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
                     ph ^= (s == 0) ? 1u : 0u;
                     t = (t + 1 == kSfSlots) ? 0u : t + 1;
                 }
-                if (ok && elect_one()) tc_commit_pair(acc_full_bar);  // the leader's epilogue passes it on
-                __syncwarp();
             }
         }
     } else if (warp >= kFirstStager) {
@@ -532,7 +534,7 @@ gemm_w4a4_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
         bool ok = true;
         for (int tile = pair; tile < total_tiles && ok; tile += num_pairs) {
             for (int kt = 0; kt < p.k_tiles; ++kt, ++it) {
-                if ((it & 1u) != set) continue;
+                if ((it % kStagerSets) != set) continue;
                 const int s = it % kStages;
                 const uint32_t t = it % kSfSlots;
                 // The stage's previous occupant has been released (which makes the parity wait that
@@ -544,13 +546,13 @@ gemm_w4a4_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
                 const uint32_t sf_s = base + s * kStageBytes + kABytes + kBBytes + lane * 16u;
                 const uint32_t sf_t = tmem_base + lane_ofs + sf_slot_col(t);
                 // the shared-memory reads do not depend on the slot: start them before waiting for it
-                uint4 a[4], b0[4], b1[4];
-                if (kb_valid == 4) {
+                uint4 sa[4], sb[kNB][4];
 #pragma unroll
-                    for (int kk = 0; kk < 4; ++kk) {
-                        a[kk] = lds128(sf_s + kk * kSfBlock);
-                        b0[kk] = lds128(sf_s + kSfaBytes + kk * kSfBlock);
-                        b1[kk] = lds128(sf_s + 2 * kSfaBytes + kk * kSfBlock);
+                for (int kk = 0; kk < 4; ++kk) {
+                    if (kk < kb_valid) {
+                        sa[kk] = lds128(sf_s + kk * kSfBlock);
+#pragma unroll
+                        for (int j = 0; j < kNB; ++j) sb[j][kk] = lds128(sf_s + (1 + j) * kSfaBytes + kk * kSfBlock);
                     }
                 }
                 // the MMAs that read this slot kSfSlots iterations ago have completed (their commit
@@ -559,19 +561,13 @@ gemm_w4a4_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
                     ok = mbar_wait_warp(stage_free_bar((it - kSfSlots) % kStages), ((it - kSfSlots) / kStages) & 1u, wctx);
                 if (!ok) break;
                 tc_fence_after();
-                if (kb_valid == 4) {
 #pragma unroll
-                    for (int kk = 0; kk < 4; ++kk) {
-                        tc_st4(sf_t + 4 * kk, a[kk]);
-                        stage_b_scales(sf_t + kSfbOfs + 8 * kk, b0[kk], b1[kk]);
-                    }
-                } else {
-                    for (int kk = 0; kk < kb_valid; ++kk) {
-                        const uint4 a = lds128(sf_s + kk * kSfBlock);
-                        const uint4 b0 = lds128(sf_s + kSfaBytes + kk * kSfBlock);
-                        const uint4 b1 = lds128(sf_s + 2 * kSfaBytes + kk * kSfBlock);
-                        tc_st4(sf_t + 4 * kk, a);
-                        stage_b_scales(sf_t + kSfbOfs + 8 * kk, b0, b1);
+                for (int kk = 0; kk < 4; ++kk) {
+                    if (kk < kb_valid) {
+                        tc_st4(sf_t + 4 * kk, sa[kk]);
+#pragma unroll
+                        for (int j = 0; j < kNB; ++j)
+                            tc_st4(sf_t + kSfbOfs + kSfbColsPerKb * kk + 4 * j, sb[j][kk]);
                     }
                 }
                 tc_wait_st();
@@ -582,25 +578,26 @@ gemm_w4a4_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
         }
     } else {
         // ------------------------------------------------------------ epilogue
-        // Eight warps: lane quadrant q x column half h.  A warp reads its 32 rows x 128 columns
-        // out of tensor memory, scales and rounds them to bf16 and keeps them packed in 64
-        // registers; the accumulator goes back to the MMA issuer after those four loads (a few
-        // hundred cycles), and the two 64-column boxes leave through one staging box and TMA
-        // stores behind the next tile's main loop.
+        // Eight warps: lane quadrant q x column half h.  A warp reads its 32 rows x 128 columns out of
+        // tensor memory, scales and rounds them to bf16 and keeps them packed in 64 registers; the
+        // accumulator goes back to the MMA issuer after those loads (a few hundred cycles), and the
+        // two 64-column boxes leave through one staging box and TMA stores behind the next tile's
+        // main loop.
+        constexpr int kBoxes = 128 / kBoxCols, kChunks = kBoxCols / 8;  // boxes per warp, 16-byte chunks per box row
         const int q = warp & 3;                // tensor-memory lane quadrant this warp may read
-        const int h = (warp - 2) >> 2;         // column half
+        const int h = (warp - 2) >> 2;         // 128-column part
         const float alpha = __fmul_rn(__ldg(p.ts_x), __ldg(p.ts_w));
         const uint32_t buf = epi + static_cast<uint32_t>(warp - 2) * kEpiBox;
-        const uint32_t row_ofs = static_cast<uint32_t>(lane) * 128u, sw = static_cast<uint32_t>(lane & 7);
+        // 128-byte swizzle of the staging box (what the store's tensor map expects): chunk ^ (row & 7)
+        const uint32_t row_ofs = static_cast<uint32_t>(lane) * (kBoxCols * 2), sw = static_cast<uint32_t>(lane & 7);
         uint32_t tcount = 0;
         for (int tile = pair; tile < total_tiles; tile += num_pairs, ++tcount) {
             const int m_blk = tile % p.m_tiles, n_blk = tile / p.m_tiles;
-            const int m0 = m_blk * BM + static_cast<int>(rank) * BM_CTA + q * 32, n0 = n_blk * BN + h * (BN / 2);
+            const int m0 = m_blk * BM + static_cast<int>(rank) * BM_CTA + q * 32, n0 = n_blk * BN + h * 128;
             const bool got = mbar_wait(acc_full_bar, tcount & 1u, wctx);
             if (!__all_sync(0xFFFFFFFFu, got)) break;
-            if (rank == 0 && warp == 2 && lane == 0) mbar_arrive_remote(acc_full_bar, 1);
             tc_fence_after();
-            const uint32_t acc = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + h * (BN / 2);
+            const uint32_t acc = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + h * 128;
             uint32_t pk[64];  // pk[8 c + i] = columns 16 c + 2 i, 16 c + 2 i + 1 of this lane's row
             // two loads in flight: chunk c + 1 is on its way while chunk c is scaled and packed
             uint32_t va[16], vb[16];
@@ -621,18 +618,18 @@ gemm_w4a4_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
             __syncwarp();
             if (lane == 0) mbar_arrive_leader(acc_empty_bar, rank);
 #pragma unroll
-            for (int c = 0; c < 2; ++c) {
-                // the store that read the box before (previous chunk or previous tile) must be done with it
+            for (int c = 0; c < kBoxes; ++c) {
+                // the store that read the box before (previous box or previous tile) must be done with it
                 if (lane == 0) bulk_wait_read<0>();
                 __syncwarp();
 #pragma unroll
-                for (int i = 0; i < 8; ++i)
-                    sts128(buf + row_ofs + ((static_cast<uint32_t>(i) ^ sw) << 4), pk[32 * c + 4 * i], pk[32 * c + 4 * i + 1],
-                           pk[32 * c + 4 * i + 2], pk[32 * c + 4 * i + 3]);
+                for (int i = 0; i < kChunks; ++i)
+                    sts128(buf + row_ofs + ((static_cast<uint32_t>(i) ^ sw) << 4), pk[4 * kChunks * c + 4 * i],
+                           pk[4 * kChunks * c + 4 * i + 1], pk[4 * kChunks * c + 4 * i + 2], pk[4 * kChunks * c + 4 * i + 3]);
                 fence_async_smem();
                 __syncwarp();
                 if (lane == 0) {
-                    if (m0 < p.M && n0 + c * 64 < p.N) tma_store_2d(&map_y, n0 + c * 64, m0, buf);
+                    if (m0 < p.M && n0 + c * kBoxCols < p.N) tma_store_2d(&map_y, n0 + c * kBoxCols, m0, buf);
                     bulk_commit();
                 }
             }
@@ -764,12 +761,9 @@ int resident_pairs() {
     return n;
 }
 
-}  // namespace
-
-namespace {
 pq_status gemm_launch(const uint8_t *xq, const uint8_t *sfx, const float *ts_x, const uint8_t *wq, const uint8_t *sfw,
                       const float *ts_w, int64_t M, int64_t N, int64_t K, void *Y, int64_t ldy, void *ws,
-                      size_t ws_bytes, void *stream, bool programmatic) {
+                      size_t ws_bytes, void *stream) {
     PQ_REQUIRE(xq && sfx && ts_x && wq && sfw && ts_w && Y, PQ_ERR_NULL);
     PQ_REQUIRE(M > 0 && N > 0 && K >= 64 && K % 64 == 0 && N % 8 == 0 && ldy >= N, PQ_ERR_SHAPE);
     PQ_REQUIRE(M < (1ll << 31) - 256 && N < (1ll << 31) - 256 && K < (1ll << 31), PQ_ERR_SHAPE);
@@ -816,7 +810,6 @@ pq_status gemm_launch(const uint8_t *xq, const uint8_t *sfx, const float *ts_x, 
     attr.val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = &attr;
     cfg.numAttrs = 1;
-    (void)programmatic;
     PQ_CUDA_OK(cudaLaunchKernelEx(&cfg, gemm_w4a4_kernel, map_a, map_b, map_y, p));
     return PQ_OK;
 }
@@ -825,7 +818,7 @@ pq_status gemm_launch(const uint8_t *xq, const uint8_t *sfx, const float *ts_x, 
 extern "C" pq_status pq_gemm_w4a4(const uint8_t *xq, const uint8_t *sfx, const float *ts_x, const uint8_t *wq,
                                   const uint8_t *sfw, const float *ts_w, int64_t M, int64_t N, int64_t K, void *Y,
                                   int64_t ldy, void *ws, size_t ws_bytes, void *stream) {
-    return gemm_launch(xq, sfx, ts_x, wq, sfw, ts_w, M, N, K, Y, ldy, ws, ws_bytes, stream, false);
+    return gemm_launch(xq, sfx, ts_x, wq, sfw, ts_w, M, N, K, Y, ldy, ws, ws_bytes, stream);
 }
 
 extern "C" pq_status pq_linear_w4a4(const void *X, int64_t M, int64_t K, int64_t ld, const float *ts_x, uint8_t *xq,
@@ -833,7 +826,7 @@ extern "C" pq_status pq_linear_w4a4(const void *X, int64_t M, int64_t K, int64_t
                                     void *Y, int64_t ldy, void *ws, size_t ws_bytes, void *stream) {
     const pq_status rc = pq_quant_act_nvfp4(X, M, K, ld, ts_x, xq, sfx, PQ_SF_TCGEN05, stream);
     if (rc != PQ_OK) return rc;
-    return gemm_launch(xq, sfx, ts_x, wq, sfw, ts_w, M, N, K, Y, ldy, ws, ws_bytes, stream, true);
+    return gemm_launch(xq, sfx, ts_x, wq, sfw, ts_w, M, N, K, Y, ldy, ws, ws_bytes, stream);
 }
 
 extern "C" pq_status pq_linear_w4a4_host(const void *X_host, int64_t M, int64_t K, const float *ts_x, void *X_dev,
@@ -921,7 +914,7 @@ extern "C" pq_status pq_linear_w4a4_batched(int n, const void *const *X, int64_t
         }
         for (int i = i0; i < i1 && rc == PQ_OK; ++i) {
             const int s = i % n_sets;
-            rc = gemm_launch(xq[s], sfx[s], ts_x, wq, sfw, ts_w, M, N, K, Y[i], ldy, ws, ws_bytes, pipe->g, i > i0);
+            rc = gemm_launch(xq[s], sfx[s], ts_x, wq, sfw, ts_w, M, N, K, Y[i], ldy, ws, ws_bytes, pipe->g);
             if (rc == PQ_OK && cudaEventRecord(pipe->g_done[s], pipe->g) != cudaSuccess) rc = PQ_ERR_CUDA;
         }
     }
@@ -970,7 +963,7 @@ extern "C" pq_status pq_linear_w4a4_host_batched(int n, const void *const *X_hos
         if (i >= n_sets && !cuda_ok(cudaStreamWaitEvent(run, pipe->down_done[s], 0))) break;
         rc = pq_quant_act_nvfp4(X_dev[s], M, K, K, ts_x, xq, sfx, PQ_SF_TCGEN05, run);
         if (rc != PQ_OK || !cuda_ok(cudaEventRecord(pipe->q_done[s], run))) break;
-        rc = gemm_launch(xq, sfx, ts_x, wq, sfw, ts_w, M, N, K, Y_dev[s], N, ws, ws_bytes, run, true);
+        rc = gemm_launch(xq, sfx, ts_x, wq, sfw, ts_w, M, N, K, Y_dev[s], N, ws, ws_bytes, run);
         if (rc != PQ_OK || !cuda_ok(cudaEventRecord(pipe->g_done[s], run))) break;
         // download
         if (!cuda_ok(cudaStreamWaitEvent(down, pipe->g_done[s], 0))) break;
