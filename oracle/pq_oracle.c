@@ -216,6 +216,29 @@ int pqo_calib_stats(const uint16_t *T, int64_t rows, int64_t K, int64_t ld, doub
     return 0;
 }
 
+/* Per channel i: sum[i] += sum_t x[t,i]: the first moment the variance criterion of the reordering
+ * ablation (Tab. 2(a)) needs beside the second one.  Same row blocking as pqo_calib_stats: fp32
+ * additions in row order inside a chunk, a slab's chunk partials in fp64 from zero, slab sums into
+ * the fp64 total, all in ascending order. */
+int pqo_calib_sum(const uint16_t *T, int64_t rows, int64_t K, int64_t ld, double *sum) {
+    if (!T || !sum || rows <= 0 || K <= 0 || ld < K) return 1;
+    for (int64_t s0 = 0; s0 < rows; s0 += PQO_SLAB) {
+        int64_t s1 = (s0 + PQO_SLAB < rows) ? s0 + PQO_SLAB : rows;
+#pragma omp parallel for schedule(static)
+        for (int64_t i = 0; i < K; ++i) {
+            double slab = 0.0;
+            for (int64_t r0 = s0; r0 < s1; r0 += PQO_CHUNK) {
+                int64_t r1 = (r0 + PQO_CHUNK < s1) ? r0 + PQO_CHUNK : s1;
+                float p = 0.0f;
+                for (int64_t t = r0; t < r1; ++t) p = p + pqo_bf16_to_f32(T[t * ld + i]);
+                slab += (double)p;
+            }
+            sum[i] += slab;
+        }
+    }
+    return 0;
+}
+
 /* Output-side calibration error, the other reading of "the quantization error on the
  * calibration data" of Sec. 3.3 (acceptance rule, Eq. 10): per output column n
  *     err[n] += sum_t (Yref[t,n] - Yq[t,n])^2
@@ -298,6 +321,48 @@ int pqo_order_by_absmax(const float *amax, int64_t K, int32_t *perm) {
     }
     qsort(buf, (size_t)K, sizeof(keyed), keyed_desc);
     for (int64_t i = 0; i < K; ++i) perm[i] = buf[i].idx;
+    free(buf);
+    return 0;
+}
+
+/* The variance criterion of the reordering ablation (Tab. 2(a)): channels by descending
+ * var_i = E[x_i^2] - E[x_i]^2 with E[x_i^2] = sumsq[i] / rows and E[x_i] = sum[i] / rows, all in fp64
+ * (two divisions, one multiplication, one subtraction, no fused operation); equal values by
+ * ascending channel.  The value may come out slightly negative for a constant channel; the order is
+ * that of the signed values. */
+int pqo_order_by_variance(const double *sum, const double *sumsq, int64_t rows, int64_t K, int32_t *perm) {
+    if (!sum || !sumsq || !perm || K <= 0 || rows <= 0) return 1;
+    keyed *buf = (keyed *)malloc(sizeof(keyed) * (size_t)K);
+    if (!buf) return 2;
+    for (int64_t i = 0; i < K; ++i) {
+        double mean = sum[i] / (double)rows;
+        double second = sumsq[i] / (double)rows;
+        double sq = mean * mean;
+        buf[i].key = second - sq;
+        buf[i].idx = (int32_t)i;
+    }
+    qsort(buf, (size_t)K, sizeof(keyed), keyed_desc);
+    for (int64_t i = 0; i < K; ++i) perm[i] = buf[i].idx;
+    free(buf);
+    return 0;
+}
+
+/* The "round-robin" order of the reordering ablation (Tab. 2(a)).  The paper names it without a
+ * definition; the reading taken here: the channels, sorted by descending second moment (equal values by
+ * ascending channel), are dealt to the K/g groups one at a time in turn, so that every group receives
+ * channels of every magnitude (the opposite of clustering).  The channel of sorted rank r goes to group
+ * r mod G at slot r div G, G = K / group:  perm[(r % G) * group + r / G] = sorted[r]. */
+int pqo_order_round_robin(const double *sumsq, int64_t K, int group, int32_t *perm) {
+    if (!sumsq || !perm || K <= 0 || group <= 0 || K % group != 0) return 1;
+    keyed *buf = (keyed *)malloc(sizeof(keyed) * (size_t)K);
+    if (!buf) return 2;
+    for (int64_t i = 0; i < K; ++i) {
+        buf[i].key = sumsq[i];
+        buf[i].idx = (int32_t)i;
+    }
+    qsort(buf, (size_t)K, sizeof(keyed), keyed_desc);
+    int64_t G = K / group;
+    for (int64_t r = 0; r < K; ++r) perm[(r % G) * group + r / G] = buf[r].idx;
     free(buf);
     return 0;
 }

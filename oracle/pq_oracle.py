@@ -44,6 +44,9 @@ def _declare(L):
     L.pqo_select_perm.argtypes = [_P, _i64, _P, _i64, _i64, C.c_int, _P]
     L.pqo_output_error.argtypes = [_P, _i64, _P, _i64, _i64, _i64, _P]
     L.pqo_order_by_absmax.argtypes = [_P, _i64, _P]
+    L.pqo_calib_sum.argtypes = [_P, _i64, _i64, _i64, _P]
+    L.pqo_order_by_variance.argtypes = [_P, _P, _i64, _i64, _P]
+    L.pqo_order_round_robin.argtypes = [_P, _i64, C.c_int, _P]
     L.pqo_group_error.argtypes = [_P, _i64, _i64, _i64, C.c_int, C.c_int, C.c_int, C.c_float, _P,
                                   C.c_int, _P]
     L.pqo_accept.argtypes = [_P, C.c_double, _P, C.c_double, C.c_int, _i64, C.c_double, _P, _P, _P]
@@ -167,6 +170,34 @@ def order_by_absmax(amax):
     amax = np.ascontiguousarray(amax, dtype=np.float32)
     perm = np.empty(amax.size, dtype=np.int32)
     _check(lib().pqo_order_by_absmax(_ptr(amax), amax.size, _ptr(perm)), "order_by_absmax")
+    return perm
+
+
+def calib_sum(T, total=None):
+    """Accumulate the per-channel plain sum (fp64) of one batch: the first moment of the variance criterion."""
+    T = _bf16(T)
+    rows, K = T.shape
+    if total is None:
+        total = np.zeros(K, dtype=np.float64)
+    _check(lib().pqo_calib_sum(_ptr(T), rows, K, K, _ptr(total)), "calib_sum")
+    return total
+
+
+def order_by_variance(total, sumsq, rows):
+    """Tab. 2(a) variance criterion: channels by descending E[x^2] - E[x]^2, ties by ascending channel."""
+    total = np.ascontiguousarray(total, dtype=np.float64)
+    sumsq = np.ascontiguousarray(sumsq, dtype=np.float64)
+    perm = np.empty(sumsq.size, dtype=np.int32)
+    _check(lib().pqo_order_by_variance(_ptr(total), _ptr(sumsq), int(rows), sumsq.size, _ptr(perm)), "order_by_variance")
+    return perm
+
+
+def order_round_robin(sumsq, group):
+    """Tab. 2(a) round-robin order (this build's reading): channels sorted by descending second moment and
+    dealt to the K / group groups in turn."""
+    sumsq = np.ascontiguousarray(sumsq, dtype=np.float64)
+    perm = np.empty(sumsq.size, dtype=np.int32)
+    _check(lib().pqo_order_round_robin(_ptr(sumsq), sumsq.size, int(group), _ptr(perm)), "order_round_robin")
     return perm
 
 

@@ -55,8 +55,9 @@ __device__ __forceinline__ void load_group(const uint16_t *p, uint4 &lo, uint4 &
 #endif
 constexpr int kActRows = PQ_ACT_ROWS;  // rows per thread: their loads are issued together
 
+// 32 registers per thread (eight 256-thread blocks per SM): all 2048 thread slots of an SM carry a load
 template <int SF_LAYOUT, bool WIDE, int kActTileRows>
-__global__ void __launch_bounds__(kActThreads)
+__global__ void __launch_bounds__(kActThreads, 2048 / kActThreads)
 quant_nvfp4_kernel(const uint16_t *__restrict__ X, int64_t rows, int64_t rows_pad, int64_t K,
                    int64_t ld, const float *__restrict__ ts_ptr, uint8_t *__restrict__ codes,
                    uint8_t *__restrict__ sf) {
