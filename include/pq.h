@@ -60,7 +60,7 @@ typedef enum {
 
 /* Quantization format of the error / fake-quant entry points.
  *   kind 0: NVFP4 (bits and group ignored: 4 bits, groups of 16).
- *   kind 1: symmetric integer, Eq. 1-2, Q = 2^(bits-1) - 1; bits in 2..8, group in {16,32,64,128}. */
+ *   kind 1: symmetric integer, Eq. 1-2, Q = 2^(bits-1) - 1; bits in 2..8, group in {16,32,64,128,256}. */
 typedef struct {
     int kind;
     int bits;
@@ -200,6 +200,31 @@ pq_status pq_output_error(const float *Yref, int64_t ld_ref, const void *Yq, int
  *   perm : device int32 [K] out.  ws : pq_workspace_bytes(PQ_OP_SELECT_PERM, 0, K, 0, 1). */
 pq_status pq_order_by_absmax(const float *amax, int64_t K, int32_t *perm, void *ws, size_t ws_bytes,
                              void *stream);
+
+/* Per-channel first moments, the other ingredient of the variance criterion of the reordering ablation
+ * (Tab. 2(a)):  sum[i] += sum_t T[t,i], blocked exactly like the squares of pq_calib_stats (fp32
+ * additions in row order inside a chunk of PQ_CHUNK_ROWS rows; chunks, slabs and the total in fp64).
+ *   T : bf16 [rows, K], ld.  sum : fp64 [K] in/out (the caller zeroes it before the first batch).
+ *   ws : pq_workspace_bytes(PQ_OP_CALIB_STATS, rows, K, 0, 0). */
+pq_status pq_calib_sum(const void *T, int64_t rows, int64_t K, int64_t ld, double *sum, void *ws,
+                       size_t ws_bytes, void *stream);
+
+/* The variance criterion of Tab. 2(a) as one more candidate order: channels by descending
+ * var_i = sumsq[i] / rows - (sum[i] / rows)^2 in fp64 (two divisions, one multiplication, one
+ * subtraction; may come out slightly negative for a constant channel), equal values in ascending
+ * channel order.
+ *   sum, sumsq : device fp64 [K] as accumulated by pq_calib_sum / pq_calib_stats over `rows` rows.
+ *   perm : device int32 [K] out.  K <= 16384.  ws : pq_workspace_bytes(PQ_OP_SELECT_PERM, 0, K, 0, 1). */
+pq_status pq_order_by_variance(const double *sum, const double *sumsq, int64_t rows, int64_t K,
+                               int32_t *perm, void *ws, size_t ws_bytes, void *stream);
+
+/* The "round-robin" order of Tab. 2(a).  The paper names it without defining it; this library's
+ * reading: the channels sorted by descending second moment (equal values in ascending channel order)
+ * are dealt to the K / group groups one at a time in turn, so every group receives channels of every
+ * magnitude: with G = K / group, perm[(r % G) * group + r / G] = channel of sorted rank r.
+ *   sumsq : device fp64 [K].  K % group == 0, K <= 16384.  perm, ws : as for pq_order_by_variance. */
+pq_status pq_order_round_robin(const double *sumsq, int64_t K, int group, int32_t *perm, void *ws,
+                               size_t ws_bytes, void *stream);
 
 /* Relative-error weights for pq_accept: lambda[0] = 1 / sum_i sumsq_a[i], lambda[1] =
  * 1 / sum_i sumsq_w[i] (sequential fp64 sums in channel order).  lambda: device fp64 [2]. */
@@ -367,7 +392,7 @@ pq_status pq_hadamard_quant_nvfp4(const void *X, int64_t M, int64_t K, int64_t l
 
 /* Integer fake-quant of Eq. 1-2 (quantize, dequantize, round to bf16), optional gather.
  *   T : bf16 [rows, K], ld.  out : bf16 [rows, K], ldo.  perm : int32 [K] or NULL.
- *   fmt.kind must be 1; K % fmt.group == 0; K <= 16384 when perm != NULL. */
+ *   fmt.kind must be 1; fmt.group in {16, 32, 64, 128, 256}; K % fmt.group == 0; K <= 16384 when perm != NULL. */
 pq_status pq_fakequant_int(const void *T, int64_t rows, int64_t K, int64_t ld, pq_format fmt,
                            const int32_t *perm, void *out, int64_t ldo, void *stream);
 

@@ -41,6 +41,9 @@ _SIGNATURES = {
     "pq_calib_stats": (_int, [_vp, _i64, _i64, _i64, _vp, _vp, _vp, _sz, _vp]),
     "pq_quant_act_nvfp4_perm": (_int, [_vp, _i64, _i64, _i64, _vp, _vp, _vp, _vp, _int, _vp]),
     "pq_order_by_absmax": (_int, [_vp, _i64, _vp, _vp, _sz, _vp]),
+    "pq_calib_sum": (_int, [_vp, _i64, _i64, _i64, _vp, _vp, _sz, _vp]),
+    "pq_order_by_variance": (_int, [_vp, _vp, _i64, _i64, _vp, _vp, _sz, _vp]),
+    "pq_order_round_robin": (_int, [_vp, _i64, _int, _vp, _vp, _sz, _vp]),
     "pq_output_error": (_int, [_vp, _i64, _vp, _i64, _i64, _i64, _vp, _vp, _sz, _vp]),
     "pq_calib_stats_static": (_int, [_vp, _i64, _i64, _i64, _vp, _vp, _vp]),
     "pq_calib_stats_static_max_bytes": (_sz, []),
@@ -149,6 +152,31 @@ def pq_order_by_absmax(amax, perm, ws):
     assert amax.dtype == torch.float32 and perm.dtype == torch.int32 and perm.numel() == amax.numel()
     w, wb = _ws(ws)
     _check("pq_order_by_absmax", lib().pq_order_by_absmax(_p(amax), amax.numel(), _p(perm), w, wb, _stream()))
+
+
+def pq_calib_sum(T, total, ws):
+    """total[i] += sum over rows of T[:, i] (fp64 [K]); workspace as for pq_calib_stats."""
+    _bf16(T)
+    assert total.dtype == torch.float64 and total.numel() == T.shape[1]
+    w, wb = _ws(ws)
+    _check("pq_calib_sum", lib().pq_calib_sum(_p(T), T.shape[0], T.shape[1], T.stride(0), _p(total), w, wb, _stream()))
+
+
+def pq_order_by_variance(total, sumsq, rows, perm, ws):
+    """perm[pos] = channel with the pos-th largest variance sumsq/rows - (total/rows)^2; int32 [K]."""
+    assert total.dtype == torch.float64 and sumsq.dtype == torch.float64 and perm.dtype == torch.int32
+    assert total.numel() == sumsq.numel() == perm.numel()
+    w, wb = _ws(ws)
+    _check("pq_order_by_variance", lib().pq_order_by_variance(_p(total), _p(sumsq), int(rows), sumsq.numel(), _p(perm),
+                                                              w, wb, _stream()))
+
+
+def pq_order_round_robin(sumsq, group, perm, ws):
+    """Channels sorted by descending second moment, dealt to the K / group groups in turn; int32 [K]."""
+    assert sumsq.dtype == torch.float64 and perm.dtype == torch.int32 and perm.numel() == sumsq.numel()
+    w, wb = _ws(ws)
+    _check("pq_order_round_robin", lib().pq_order_round_robin(_p(sumsq), sumsq.numel(), int(group), _p(perm), w, wb,
+                                                              _stream()))
 
 
 def pq_output_error(Yref, Yq, err, ws):

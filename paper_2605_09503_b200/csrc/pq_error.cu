@@ -316,7 +316,7 @@ extern "C" pq_status pq_group_error(const void *T, int64_t rows, int64_t K, int6
     const int group = fmt.kind == 0 ? 16 : fmt.group;
     if (fmt.kind == 1) {
         PQ_REQUIRE(fmt.bits >= 2 && fmt.bits <= 8, PQ_ERR_FORMAT);
-        PQ_REQUIRE(group == 16 || group == 32 || group == 64 || group == 128, PQ_ERR_FORMAT);
+        PQ_REQUIRE(group == 16 || group == 32 || group == 64 || group == 128 || group == 256, PQ_ERR_FORMAT);
     } else {
         PQ_REQUIRE(ts, PQ_ERR_NULL);
     }
@@ -336,6 +336,7 @@ extern "C" pq_status pq_group_error(const void *T, int64_t rows, int64_t K, int6
         case 16: return launch<1, 2>(t, rows, K, ld, ts, Qf, perms, P, ws, err, st);
         case 32: return launch<1, 4>(t, rows, K, ld, ts, Qf, perms, P, ws, err, st);
         case 64: return launch<1, 8>(t, rows, K, ld, ts, Qf, perms, P, ws, err, st);
-        default: return launch<1, 16>(t, rows, K, ld, ts, Qf, perms, P, ws, err, st);
+        case 128: return launch<1, 16>(t, rows, K, ld, ts, Qf, perms, P, ws, err, st);
+        default: return launch<1, 32>(t, rows, K, ld, ts, Qf, perms, P, ws, err, st);   // 256: a whole warp per group
     }
 }

@@ -6,7 +6,9 @@
 // comparisons of one candidate are a few hundred million integer compares spread over the
 // whole GPU -- latency-trivial next to the calibration passes, free of shared-memory size
 // limits, and the result is unique, hence identical to any comparison sort.
-// Keys are non-negative doubles, which order exactly like their 64-bit patterns.
+// Keys are 64-bit patterns that order like the doubles they stand for: a non-negative double orders
+// like its own bits; a signed one after flipping all bits of a negative value and the sign bit of
+// the others.
 #include "pq_common.cuh"
 
 namespace {
@@ -32,10 +34,29 @@ __global__ void absmax_keys(const float *__restrict__ amax, int64_t K, unsigned 
     if (i < K) keys[i] = static_cast<unsigned long long>(__double_as_longlong(static_cast<double>(fabsf(amax[i]))));
 }
 
+// keys[i] = sortable pattern of var_i = sumsq_i / rows - (sum_i / rows)^2 in fp64 (two divisions, one
+// multiplication, one subtraction); the value may be slightly negative for a constant channel.
+__global__ void variance_keys(const double *__restrict__ sum, const double *__restrict__ sumsq, double rows, int64_t K,
+                              unsigned long long *__restrict__ keys) {
+    const int64_t i = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
+    if (i >= K) return;
+    const double mean = __ddiv_rn(sum[i], rows);
+    const double second = __ddiv_rn(sumsq[i], rows);
+    const double var = __dadd_rn(__dsub_rn(second, __dmul_rn(mean, mean)), 0.0);  // + 0.0: a zero is +0
+    const long long bits = __double_as_longlong(var);
+    keys[i] = bits < 0 ? ~static_cast<unsigned long long>(bits) : static_cast<unsigned long long>(bits) | (1ull << 63);
+}
+
+// keys[i] = bit pattern of a non-negative fp64 value
+__global__ void plain_keys(const double *__restrict__ v, int64_t K, unsigned long long *__restrict__ keys) {
+    const int64_t i = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
+    if (i < K) keys[i] = static_cast<unsigned long long>(__double_as_longlong(fabs(v[i])));
+}
+
 constexpr int kRankThreads = 256;
 
 __global__ void __launch_bounds__(kRankThreads)
-perm_rank(const unsigned long long *__restrict__ keys, int64_t K, int32_t *__restrict__ perms) {
+perm_rank(const unsigned long long *__restrict__ keys, int64_t K, int32_t *__restrict__ perms, int deal_groups, int group) {
     __shared__ unsigned long long tile[kRankThreads];
     const int j = blockIdx.y;
     const unsigned long long *kj = keys + static_cast<int64_t>(j) * K;
@@ -54,7 +75,10 @@ perm_rank(const unsigned long long *__restrict__ keys, int64_t K, int32_t *__res
             rank += (other > mine) || (other == mine && base + u < i);
         }
     }
-    if (i < K) perms[static_cast<int64_t>(j) * K + rank] = static_cast<int32_t>(i);
+    // deal_groups == 0: the channel of rank r is read at position r; otherwise the sorted channels are dealt
+    // to deal_groups groups in turn: rank r goes to group r % deal_groups, slot r / deal_groups
+    const int64_t pos = deal_groups ? static_cast<int64_t>(rank % deal_groups) * group + rank / deal_groups : rank;
+    if (i < K) perms[static_cast<int64_t>(j) * K + pos] = static_cast<int32_t>(i);
 }
 
 // One thread per order p = 0..P sums its error rows; thread 0 then applies Eq. 10.
@@ -98,7 +122,7 @@ extern "C" pq_status pq_select_perm(const double *sumsq_a, int64_t rows_a, const
     perm_keys<<<static_cast<unsigned>(pq_ceil_div(K, 128)), 128, 0, st>>>(
         sumsq_a, static_cast<double>(rows_a), sumsq_w, static_cast<double>(rows_w), K, J, keys);
     dim3 grid(static_cast<unsigned>(pq_ceil_div(K, kRankThreads)), static_cast<unsigned>(J + 1));
-    perm_rank<<<grid, kRankThreads, 0, st>>>(keys, K, perms);
+    perm_rank<<<grid, kRankThreads, 0, st>>>(keys, K, perms, 0, 0);
     return pq_launch_status();
 }
 
@@ -111,7 +135,34 @@ extern "C" pq_status pq_order_by_absmax(const float *amax, int64_t K, int32_t *p
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     unsigned long long *keys = static_cast<unsigned long long *>(ws);
     absmax_keys<<<static_cast<unsigned>(pq_ceil_div(K, 128)), 128, 0, st>>>(amax, K, keys);
-    perm_rank<<<dim3(static_cast<unsigned>(pq_ceil_div(K, kRankThreads)), 1), kRankThreads, 0, st>>>(keys, K, perm);
+    perm_rank<<<dim3(static_cast<unsigned>(pq_ceil_div(K, kRankThreads)), 1), kRankThreads, 0, st>>>(keys, K, perm, 0, 0);
+    return pq_launch_status();
+}
+
+extern "C" pq_status pq_order_by_variance(const double *sum, const double *sumsq, int64_t rows, int64_t K, int32_t *perm,
+                                          void *ws, size_t ws_bytes, void *stream) {
+    PQ_REQUIRE(sum && sumsq && perm, PQ_ERR_NULL);
+    PQ_REQUIRE(K > 0 && K <= 16384 && rows > 0, PQ_ERR_SHAPE);
+    PQ_REQUIRE(ws && ws_bytes >= pq_workspace_bytes(PQ_OP_SELECT_PERM, 0, K, 0, 1), PQ_ERR_WORKSPACE);
+    PQ_REQUIRE(pq_aligned256(ws), PQ_ERR_ALIGN);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    unsigned long long *keys = static_cast<unsigned long long *>(ws);
+    variance_keys<<<static_cast<unsigned>(pq_ceil_div(K, 128)), 128, 0, st>>>(sum, sumsq, static_cast<double>(rows), K, keys);
+    perm_rank<<<dim3(static_cast<unsigned>(pq_ceil_div(K, kRankThreads)), 1), kRankThreads, 0, st>>>(keys, K, perm, 0, 0);
+    return pq_launch_status();
+}
+
+extern "C" pq_status pq_order_round_robin(const double *sumsq, int64_t K, int group, int32_t *perm, void *ws,
+                                          size_t ws_bytes, void *stream) {
+    PQ_REQUIRE(sumsq && perm, PQ_ERR_NULL);
+    PQ_REQUIRE(K > 0 && K <= 16384 && group > 0 && K % group == 0, PQ_ERR_SHAPE);
+    PQ_REQUIRE(ws && ws_bytes >= pq_workspace_bytes(PQ_OP_SELECT_PERM, 0, K, 0, 1), PQ_ERR_WORKSPACE);
+    PQ_REQUIRE(pq_aligned256(ws), PQ_ERR_ALIGN);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    unsigned long long *keys = static_cast<unsigned long long *>(ws);
+    plain_keys<<<static_cast<unsigned>(pq_ceil_div(K, 128)), 128, 0, st>>>(sumsq, K, keys);
+    perm_rank<<<dim3(static_cast<unsigned>(pq_ceil_div(K, kRankThreads)), 1), kRankThreads, 0, st>>>(
+        keys, K, perm, static_cast<int>(K / group), group);
     return pq_launch_status();
 }
 

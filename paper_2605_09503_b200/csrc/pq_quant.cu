@@ -416,7 +416,7 @@ extern "C" pq_status pq_fakequant_int(const void *T, int64_t rows, int64_t K, in
                                       const int32_t *perm, void *out, int64_t ldo, void *stream) {
     PQ_REQUIRE(T && out, PQ_ERR_NULL);
     PQ_REQUIRE(fmt.kind == 1 && fmt.bits >= 2 && fmt.bits <= 8, PQ_ERR_FORMAT);
-    PQ_REQUIRE(fmt.group == 16 || fmt.group == 32 || fmt.group == 64 || fmt.group == 128, PQ_ERR_FORMAT);
+    PQ_REQUIRE(fmt.group == 16 || fmt.group == 32 || fmt.group == 64 || fmt.group == 128 || fmt.group == 256, PQ_ERR_FORMAT);
     PQ_REQUIRE(rows > 0 && K > 0 && K % fmt.group == 0 && ld >= K && ldo >= K, PQ_ERR_SHAPE);
     PQ_REQUIRE(!perm || K <= 16384, PQ_ERR_SHAPE);
     PQ_REQUIRE(pq_aligned16(T) && pq_aligned16(out) && ld % 8 == 0 && ldo % 8 == 0, PQ_ERR_ALIGN);
@@ -439,7 +439,8 @@ extern "C" pq_status pq_fakequant_int(const void *T, int64_t rows, int64_t K, in
         case 16: PQ_FQ_CASE(2) break;
         case 32: PQ_FQ_CASE(4) break;
         case 64: PQ_FQ_CASE(8) break;
-        default: PQ_FQ_CASE(16) break;
+        case 128: PQ_FQ_CASE(16) break;
+        default: PQ_FQ_CASE(32) break;
     }
 #undef PQ_FQ_CASE
     return pq_launch_status();

@@ -81,6 +81,51 @@ calib_stats_slab(const uint16_t *__restrict__ T, int64_t rows, int64_t K, int64_
     }
 }
 
+// First moments (plain column sums) with the same slab / chunk walk: fp32 additions in row order
+// inside a chunk, the slab's eight chunk partials in fp64 from zero.
+__global__ void __launch_bounds__(kStatsThreads)
+calib_sum_slab(const uint16_t *__restrict__ T, int64_t rows, int64_t K, int64_t ld, double *__restrict__ slab_sum) {
+    __shared__ __align__(16) float sum_s[kSlabChunks][kStatsCols];
+    pq::dependents_may_launch();
+    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+    const int64_t col0 = static_cast<int64_t>(blockIdx.y) * kStatsCols;
+    const int64_t col = col0 + lane * 8;
+    const int64_t slab = blockIdx.x;
+    const int64_t r0 = slab * PQ_SLAB_ROWS + w * PQ_CHUNK_ROWS;
+    const int64_t left = rows - r0;
+    const int n = left >= PQ_CHUNK_ROWS ? PQ_CHUNK_ROWS : (left > 0 ? static_cast<int>(left) : 0);
+    float s[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) s[i] = 0.0f;
+    if (col < K) {
+        const uint16_t *p = T + r0 * ld + col;
+        uint4 v[PQ_CHUNK_ROWS];
+#pragma unroll
+        for (int u = 0; u < PQ_CHUNK_ROWS; ++u)
+            v[u] = u < n ? __ldcs(reinterpret_cast<const uint4 *>(p + static_cast<int64_t>(u) * ld)) : make_uint4(0, 0, 0, 0);
+#pragma unroll
+        for (int u = 0; u < PQ_CHUNK_ROWS; ++u) {
+            if (u < n) {  // a row past the end must not even add +0.0: -0.0 + 0.0 would change a sign
+                float x[8];
+                pq::unpack8(v[u], x);
+#pragma unroll
+                for (int i = 0; i < 8; ++i) s[i] = __fadd_rn(s[i], x[i]);
+            }
+        }
+    }
+    float4 *ds = reinterpret_cast<float4 *>(&sum_s[w][lane * 8]);
+    ds[0] = make_float4(s[0], s[1], s[2], s[3]);
+    ds[1] = make_float4(s[4], s[5], s[6], s[7]);
+    __syncthreads();
+    const int c = threadIdx.x;
+    if (col0 + c < K) {
+        double acc = 0.0;
+#pragma unroll
+        for (int k = 0; k < kSlabChunks; ++k) acc = __dadd_rn(acc, static_cast<double>(sum_s[k][c]));
+        slab_sum[slab * K + col0 + c] = acc;
+    }
+}
+
 // Output-side calibration error: the same slab / chunk walk over the fp32 difference of two
 // tensors (fp32 reference, bf16 quantized-layer output): 6 bytes per element, streaming.  A lane
 // owns 8 adjacent columns; eight rows (two 16-byte loads of the reference and one of the output per
@@ -188,6 +233,23 @@ extern "C" pq_status pq_calib_stats(const void *T, int64_t rows, int64_t K, int6
     float *slab_max = reinterpret_cast<float *>(slab_sum + slabs * K);
     calib_stats_slab<<<grid, kStatsThreads, 0, st>>>(static_cast<const uint16_t *>(T), rows, K, ld, slab_sum, slab_max);
     PQ_CUDA_OK((pq::launch_fold<double, 1, true>(slab_sum, slab_max, slabs, K, sumsq, amax, st)));
+    return pq_launch_status();
+}
+
+extern "C" pq_status pq_calib_sum(const void *T, int64_t rows, int64_t K, int64_t ld, double *sum, void *ws,
+                                  size_t ws_bytes, void *stream) {
+    PQ_REQUIRE(T && sum, PQ_ERR_NULL);
+    PQ_REQUIRE(rows > 0 && K > 0 && K % 8 == 0 && ld >= K, PQ_ERR_SHAPE);
+    PQ_REQUIRE(pq_aligned16(T) && ld % 8 == 0, PQ_ERR_ALIGN);
+    PQ_REQUIRE(ws && ws_bytes >= pq_workspace_bytes(PQ_OP_CALIB_STATS, rows, K, 0, 0), PQ_ERR_WORKSPACE);
+    PQ_REQUIRE(pq_aligned256(ws), PQ_ERR_ALIGN);
+    const int64_t slabs = pq_ceil_div(rows, PQ_SLAB_ROWS);
+    PQ_REQUIRE(slabs < (1ll << 31) && K <= 65535ll * kStatsCols, PQ_ERR_SHAPE);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    dim3 grid(static_cast<unsigned>(slabs), static_cast<unsigned>(pq_ceil_div(K, kStatsCols)));
+    double *slab_sum = static_cast<double *>(ws);
+    calib_sum_slab<<<grid, kStatsThreads, 0, st>>>(static_cast<const uint16_t *>(T), rows, K, ld, slab_sum);
+    PQ_CUDA_OK((pq::launch_fold<double, 1, false>(slab_sum, nullptr, slabs, K, sum, nullptr, st)));
     return pq_launch_status();
 }
 
