@@ -2,8 +2,10 @@
 here: every step is one entry point of libpq.so, all enqueued on the current stream without a
 host round trip (the accept decision stays on the device and is consumed by pq_quant_weight).
 
-  calibrate()  offline: statistics -> Eq. 9 candidates -> Eq. 3 errors -> Eq. 10 -> P^T W quantized
-  QuantLinear  runtime: bf16 activations (already permuted) -> NVFP4 -> W4A4 GEMM -> bf16
+  calibrate()    offline: statistics -> Eq. 9 candidates -> Eq. 3 errors -> Eq. 10 -> P^T W quantized
+  QuantLinear    runtime: bf16 activations (already permuted) -> NVFP4 -> W4A4 GEMM -> bf16
+  calibrate_h()  the same offline pass in the Hadamard-transformed basis (PermuQuant-H, App. D)
+  QuantLinearH   runtime of PermuQuant-H: Hadamard + reordering + NVFP4 in one kernel, then the GEMM
 """
 from dataclasses import dataclass
 
@@ -89,6 +91,19 @@ def calibrate(batches, Wt, fmt=NVFP4, J=5, tau=0.0, sf_layout=B.PQ_SF_TCGEN05) -
     return Calibration(sumsq_a, sumsq_w, amax_a, ts_x, ts_w, perms, err_x, err_w, lam, E, select, wq, sfw, rows_a)
 
 
+def calibrate_h(batches, Wt, fmt=NVFP4, J=5, tau=0.0):
+    """PermuQuant-H (App. D): the representation that is quantized is x H, so statistics, candidate
+    orders, errors and the acceptance rule are all taken on the transformed calibration batches and on
+    the transformed weight rows Wt H (the product is unchanged: (x H)(Wt H)^T = x Wt^T).  Returns the
+    Calibration of the transformed layer; its chosen order is applied AFTER the transform at run time."""
+    def transformed(t):
+        out = torch.empty(t.shape[0], t.shape[1], dtype=torch.bfloat16, device=t.device)
+        B.pq_hadamard_quant_nvfp4(t, None, None, None, None, B.PQ_SF_LINEAR, out)
+        return out
+
+    return calibrate([transformed(x) for x in batches], transformed(Wt), fmt=fmt, J=J, tau=tau)
+
+
 def select_by_output_error(batches, refs, Wt, perms, ts_x, tau=0.0):
     """The acceptance rule of Eq. 10 with E read on the layer's output (Sec. 3.3): for the original
     order and every candidate row of `perms` (int32 [P, K]) quantize W and the calibration batches in
@@ -161,3 +176,23 @@ class QuantLinear:
         code = B.pq_device_status(self.ws)
         if code != B.PQ_OK:
             raise B.PqError("pq_gemm_w4a4 (device)", code, B.status_string(code))
+
+
+class QuantLinearH(QuantLinear):
+    """Runtime half of PermuQuant-H: activations arrive in their ORIGINAL basis and order; one kernel
+    applies the Hadamard transform, reads the transformed channels in the calibrated order and
+    quantizes them (pq_hadamard_quant_nvfp4), then the W4A4 GEMM runs against the weight quantized by
+    calibrate_h."""
+
+    def __init__(self, wq, sfw, ts_w, ts_x, M_max, order):
+        super().__init__(wq, sfw, ts_w, ts_x, M_max)
+        self.order = None if order is None else order.to(torch.int32).contiguous()
+
+    def __call__(self, X, Y=None):
+        M = X.shape[0]
+        assert M <= self.M_max and X.shape[1] == self.K
+        if Y is None:
+            Y = torch.empty(M, self.N, dtype=torch.bfloat16, device=X.device)
+        B.pq_hadamard_quant_nvfp4(X, self.order, self.ts_x, self.xq[:M], self.sfx, B.PQ_SF_TCGEN05)
+        B.pq_gemm_w4a4(self.xq[:M], self.sfx, self.ts_x, self.wq, self.sfw, self.ts_w, Y, self.ws)
+        return Y

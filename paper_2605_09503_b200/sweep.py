@@ -1,7 +1,7 @@
 """Sweeps over the two multi-layer workloads, printed as tables (one JSON line per row with --json).
 
     python -m paper_2605_09503_b200.sweep dit_block     # every linear of a double-stream DiT block, M swept
-    python -m paper_2605_09503_b200.sweep int_sweep     # INT3/INT4 x group 32/64/128 acceptance over 16 layers
+    python -m paper_2605_09503_b200.sweep int_sweep     # INT3/INT4 x group 32/64/128/256 acceptance over 16 layers
 
 dit_block: the eight linears (QKV 3072->9216, out 3072->3072, MLP up 3072->12288, down 12288->3072, image
 and text stream) with random-init N(0, 0.02) weights quantized to NVFP4, run at M tokens each through the
@@ -9,7 +9,7 @@ runtime path (activation quantize + W4A4 GEMM, pq_linear_w4a4); per block: time,
 FP4 peak passed with --peak (TFLOP/s).  Timings are CUDA-graph replays of the eight launches of a block.
 
 int_sweep: sixteen seeded layers (X 4608 x 3072 with the QKV activation statistics, W 3072 x 3072); for
-INT3 and INT4 with groups of 32, 64 and 128 the offline pipeline runs with that format driving Eq. 10;
+INT3 and INT4 with groups of 32, 64, 128 and 256 (Tab. 2(d)'s largest) the offline pipeline runs with that format driving Eq. 10;
 reported per format: mean per-group MSE of the activations without and with the chosen order, layers
 accepted, and the throughput of the per-group error reduction.
 """
@@ -87,7 +87,7 @@ def int_sweep(args):
     cfg = inputs.CONFIGS["int_sweep"]
     rows = []
     for bits in (3, 4):
-        for group in (32, 64, 128):
+        for group in (32, 64, 128, 256):
             fmt = (B.KIND_INT, bits, group)
             mse0 = mse1 = 0.0
             accepted = 0

@@ -113,3 +113,44 @@ def test_transformed_layer_reproduces_the_plain_product():
     plain = x.double().numpy() @ w.double().numpy().T
     rel = np.linalg.norm(ref - plain) / np.linalg.norm(plain)
     assert rel < 0.15, rel
+
+
+def test_permuquant_h_pipeline_against_the_oracle_route():
+    """calibrate_h + QuantLinearH on the small layer: every decision equals the oracle's taken on the
+    oracle's own transformed tensors, and the layer output stays within the GEMM tolerance of the fp64
+    reference of the transformed, reordered, quantized operands."""
+    from paper_2605_09503_b200 import pipeline
+    cfg = inputs.CONFIGS["tiny"]
+    seed, fmt = 1, (B.KIND_INT, 4, 32)
+    xs = [inputs.activations(cfg, seed, b) for b in range(2)]
+    w = inputs.weight(cfg, seed)
+    cal = pipeline.calibrate_h([x.to(DEV) for x in xs], w.to(DEV), fmt=fmt)
+    # oracle: transform, then the ordinary offline pass
+    xh = [O.hadamard_quant_nvfp4(inputs.bits(x), 1.0, quantize=False)[2] for x in xs]
+    wh = O.hadamard_quant_nvfp4(inputs.bits(w), 1.0, quantize=False)[2]
+    Sa = Aa = None
+    for x in xh:
+        Sa, Aa = O.calib_stats(x, Sa, Aa)
+    Sw, Aw = O.calib_stats(wh)
+    ts_x, ts_w = O.tensor_scale(Aa), O.tensor_scale(Aw)
+    perms = O.select_perm(Sa, sum(x.shape[0] for x in xh), Sw, wh.shape[0], 5)
+    cand = np.concatenate([np.arange(cfg.K, dtype=np.int32)[None], perms])
+    ex = np.zeros((7, cfg.K // fmt[2]))
+    for x in xh:
+        ex = O.group_error(x, *fmt, ts_x, cand, err=ex)
+    ew = O.group_error(wh, *fmt, ts_w, cand)
+    best, acc, _ = O.accept(ex, O.error_weight(Sa), ew, O.error_weight(Sw), 0.0)
+    assert np.array_equal(cal.sumsq_a.cpu().numpy(), Sa) and np.array_equal(cal.perms.cpu().numpy(), perms)
+    assert np.array_equal(cal.err_x.cpu().numpy(), ex) and cal.select.tolist() == [best, acc]
+    chosen = perms[best - 1] if acc else None
+    wq_o, sfw_o = O.quant_nvfp4(wh, ts_w, chosen)
+    assert np.array_equal(cal.wq.cpu().numpy(), wq_o)
+    # runtime
+    x_rt = inputs.activations(cfg, seed, 1000)
+    order = cal.chosen_perm() if acc else None
+    layer = pipeline.QuantLinearH(cal.wq, cal.sfw, cal.ts_w, cal.ts_x, cfg.M, order)
+    Y = layer(x_rt.to(DEV)).float().cpu().numpy().astype(np.float64)
+    layer.check()
+    xq_o, sfx_o, _, _ = O.hadamard_quant_nvfp4(inputs.bits(x_rt), ts_x, chosen)
+    assert np.array_equal(layer.xq.cpu().numpy(), xq_o)
+    assert_close(Y, O.gemm_ref(xq_o, sfx_o, ts_x, wq_o, sfw_o, ts_w))
