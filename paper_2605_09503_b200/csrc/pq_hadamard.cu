@@ -11,28 +11,39 @@
 // then one multiplication by fl(1 / sqrt(K)).  Within one stride the butterflies are independent, so how
 // they are spread over threads does not change a bit of the result.
 //
-// Work distribution (one thread block = up to 8 rows, each row kept as K fp32 values in shared memory):
+// Work distribution.  A thread block keeps up to 8 rows as K fp32 values each in shared memory and walks
+// over batches of rows (persistent grid):
 //   phase 1  a thread takes one octet position of one row: m 16-byte loads (the same octet of every
 //            segment), the segment combination and the strides 1, 2, 4 in registers, on PAIRS of
-//            neighbouring channels in packed f32x2 instructions (two IEEE results per issue slot; the
-//            stride-1 butterfly of a pair (x, y) is one packed fused multiply-add (x, y) * (1, -1) +
-//            (y, x), exact products, one rounding: the same bits as x + y and x - y);
+//            neighbouring channels in packed f32x2 instructions (two IEEE results per issue slot);
 //   phase 2  the remaining strides in one to three passes over shared memory: a thread owns one channel
-//            pair position and 2^LOG values of it at the pass's strides (up to 32 packed registers);
-//   phase 3  a lane takes one 16-channel group of the OUTPUT order: indices from the permutation,
-//            values gathered from shared memory, scaled, quantized like pq_quant_act_nvfp4 (coalesced
-//            code stores, four scale bytes merged into a word by shuffles).
-// Shared-memory addresses are XOR-swizzled (octet index bits 3-4 with the two bits just above the
-// first pass's window) so that the strided accesses of phase 2 spread over all banks.
+//            pair position and 2^LOG values of it at the pass's strides (up to 32 packed registers),
+//            addressed through eight base pointers and immediate offsets;
+//   phase 3  a lane takes one 16-channel group of the OUTPUT order: its 16 read-out positions (the
+//            permutation with the shared-memory swizzle applied, as 16-bit byte offsets, prepared once
+//            per block) come as two 16-byte loads, the values are gathered from shared memory and
+//            quantized like pq_quant_act_nvfp4 (coalesced code stores, four scale bytes merged into a
+//            word by shuffles).
+// Shared-memory swizzle of a row image (fp32 index i): bits 3-4 are XORed with the two bits just above
+// the first pass's window and bit 2 with bit 5.  The first spreads the strided accesses of phase 2 over
+// all banks, the second lets the eight lanes of a 16-byte store wavefront of phase 1 hit distinct banks.
+#include <algorithm>
 #include <utility>
 
 #include "pq_common.cuh"
 
 namespace {
 
-constexpr int kMaxRows = 8;         // rows per block (fewer when a row needs more than 24 KB of shared memory)
-constexpr int kThreads = 256;
-constexpr size_t kSmemBudget = 196 * 1024;
+#ifndef PQ_HAD_ROWS
+#define PQ_HAD_ROWS 8
+#endif
+constexpr int kMaxRows = PQ_HAD_ROWS;   // rows per block (fewer when a row needs more than 24 KB of shared memory)
+constexpr int kThreads = 32 * kMaxRows;
+#ifndef PQ_HAD_BLOCKS
+#define PQ_HAD_BLOCKS (512 / (32 * PQ_HAD_ROWS))
+#endif
+constexpr int kBlocksPerSm = PQ_HAD_BLOCKS;
+constexpr size_t kSmemBudget = 192 * 1024;
 
 // ---- Paley's Hadamard matrix of order 12 (compile-time)
 constexpr int quadratic_character_11(int r) {
@@ -79,15 +90,15 @@ __device__ __forceinline__ uint64_t fma2(uint64_t a, uint64_t b, uint64_t c) {
     asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r) : "l"(a), "l"(b), "l"(c));
     return r;
 }
-// (x, y) -> (x + y, x - y): (x, y) * (1, -1) + (y, x)
+// (x, y) -> (x + y, x - y)
 __device__ __forceinline__ uint64_t butterfly_in_pair(uint64_t v) {
     float x, y;
     unpack2(v, x, y);
-    return fma2(v, pack2(1.0f, -1.0f), pack2(y, x));
+    return pack2(__fadd_rn(x, y), __fsub_rn(x, y));
 }
 
 // fp32 index of a channel inside its row's shared-memory image
-__device__ __forceinline__ int swz(int idx, int sw) { return idx ^ (((idx >> sw) & 3) << 3); }
+__device__ __forceinline__ int swz(int idx, int sw) { return idx ^ (((idx >> sw) & 3) << 3) ^ (((idx >> 5) & 1) << 2); }
 
 struct HadParams {
     const uint16_t *X;
@@ -117,17 +128,17 @@ __device__ __forceinline__ void combine_segments(uint64_t (&acc)[4], const uint6
 }
 
 // strides 1, 2, 4 on the four channel pairs of an octet, then the octet goes to shared memory
-__device__ __forceinline__ void finish_octet(uint64_t (&v)[4], float *row_s, int idx, int sw, bool second_half_first) {
+__device__ __forceinline__ void finish_octet(uint64_t (&v)[4], float *row_s, int idx, int sw) {
 #pragma unroll
     for (int e = 0; e < 4; ++e) v[e] = butterfly_in_pair(v[e]);
     const uint64_t a0 = add2(v[0], v[1]), a1 = sub2(v[0], v[1]), a2 = add2(v[2], v[3]), a3 = sub2(v[2], v[3]);
     const uint64_t b0 = add2(a0, a2), b1 = add2(a1, a3), b2 = sub2(a0, a2), b3 = sub2(a1, a3);
-    // two 16-byte stores; every other group of four lanes writes its halves in the opposite order, which
-    // keeps the eight lanes of a store wavefront on distinct banks
-    ulonglong2 *dst = reinterpret_cast<ulonglong2 *>(row_s + swz(idx, sw));
-    const ulonglong2 lo = make_ulonglong2(b0, b1), hi = make_ulonglong2(b2, b3);
-    dst[second_half_first ? 1 : 0] = second_half_first ? hi : lo;
-    dst[second_half_first ? 0 : 1] = second_half_first ? lo : hi;
+    // two 16-byte stores; the swizzle swaps the halves of every other group of four octets, which keeps
+    // the eight lanes of a store wavefront on distinct banks
+    const int half = (idx >> 5) & 1;
+    ulonglong2 *dst = reinterpret_cast<ulonglong2 *>(row_s + (idx ^ (((idx >> sw) & 3) << 3)));
+    dst[half] = make_ulonglong2(b0, b1);
+    dst[half ^ 1] = make_ulonglong2(b2, b3);
 }
 
 __device__ __forceinline__ void unpack_pairs(const uint4 &raw, uint64_t (&v)[4]) {
@@ -137,26 +148,32 @@ __device__ __forceinline__ void unpack_pairs(const uint4 &raw, uint64_t (&v)[4])
 }
 
 template <int AP>
-__device__ __forceinline__ void column_12(const uint64_t (&in)[12][4], float *row_s, int seg, int o, int sw, bool flip) {
+__device__ __forceinline__ void column_12(const uint64_t (&in)[12][4], float *row_s, int seg, int o, int sw) {
     uint64_t acc[4];
 #pragma unroll
     for (int e = 0; e < 4; ++e) acc[e] = in[0][e];  // the first row of the matrix is all ones
     combine_segments<AP, 1>(acc, in);
-    finish_octet(acc, row_s, AP * seg + o * 8, sw, flip);
+    finish_octet(acc, row_s, AP * seg + o * 8, sw);
 }
 template <int... APs>
 __device__ __forceinline__ void all_columns_12(std::integer_sequence<int, APs...>, const uint64_t (&in)[12][4], float *row_s,
-                                               int seg, int o, int sw, bool flip) {
-    (column_12<APs>(in, row_s, seg, o, sw, flip), ...);
+                                               int seg, int o, int sw) {
+    (column_12<APs>(in, row_s, seg, o, sw), ...);
 }
 
 // ---- phase 2: 2^LOG values of one channel-pair position, strides 2^S ... 2^(S+LOG-1)
+// The swizzle reads two bits and bit 5 and writes bits 2-4; of the window's bits only the lowest three can
+// be among those, so the address of value j is that of value j % 8 plus an immediate.
 template <int LOG>
 __device__ __forceinline__ void pass_item(float *row_s, int base, int S, int sw, bool last, uint64_t scale2) {
-    constexpr int N = 1 << LOG;
+    constexpr int N = 1 << LOG, NB = N < 8 ? N : 8;
+    uint64_t *slot[NB];
+#pragma unroll
+    for (int m = 0; m < NB; ++m) slot[m] = reinterpret_cast<uint64_t *>(row_s + swz(base + (m << S), sw));
+    const int step = 4 << S;  // 64-bit words between value j and value j + 8
     uint64_t v[N];
 #pragma unroll
-    for (int j = 0; j < N; ++j) v[j] = *reinterpret_cast<const uint64_t *>(row_s + swz(base + (j << S), sw));
+    for (int j = 0; j < N; ++j) v[j] = slot[j % NB][(j / NB) * step];
 #pragma unroll
     for (int l = 0; l < LOG; ++l) {
 #pragma unroll
@@ -172,7 +189,7 @@ __device__ __forceinline__ void pass_item(float *row_s, int base, int S, int sw,
         for (int j = 0; j < N; ++j) v[j] = mul2(v[j], scale2);
     }
 #pragma unroll
-    for (int j = 0; j < N; ++j) *reinterpret_cast<uint64_t *>(row_s + swz(base + (j << S), sw)) = v[j];
+    for (int j = 0; j < N; ++j) slot[j % NB][(j / NB) * step] = v[j];
 }
 
 // One pass over the rows of the block: items = rows x (K / 2) channel pairs / 2^LOG.
@@ -197,111 +214,140 @@ __device__ __forceinline__ void run_pass(float *smem, const HadParams &p, int nr
 }
 
 template <int SF_LAYOUT>
-__global__ void __launch_bounds__(kThreads, 2) hadamard_quant_kernel(const HadParams p) {
-    extern __shared__ __align__(16) float had_smem[];  // [rows_per_block][K]
+__global__ void __launch_bounds__(kThreads, kBlocksPerSm) hadamard_quant_kernel(const HadParams p) {
+    extern __shared__ __align__(16) float had_smem[];  // [rows_per_block][K] fp32, then K 16-bit read-out offsets
     const int kRows = p.rows_per_block;
+    uint16_t *offset_s = reinterpret_cast<uint16_t *>(had_smem + static_cast<size_t>(kRows) * p.K);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int64_t row0 = static_cast<int64_t>(blockIdx.x) * kRows;
-    const int nrows = static_cast<int>(min(static_cast<int64_t>(kRows), max(static_cast<int64_t>(0), p.rows - row0)));
     const int seg = p.K / p.m, octs = seg >> 3;
+    const int gpr = p.K >> 4, chunks = (gpr + 31) >> 5;  // output groups per row, in chunks of one per lane
+    const int64_t batches = (p.rows_pad + kRows - 1) / kRows;
     pq::wait_for_prior_grid();
     pq::dependents_may_launch();
 
-    // ---- phase 1
-    for (int u = threadIdx.x; u < nrows * octs; u += kThreads) {
-        const int r = u / octs, o = u - r * octs;
-        const uint16_t *src = p.X + (row0 + r) * p.ld + o * 8;
-        float *row_s = had_smem + static_cast<size_t>(r) * p.K;
-        const bool flip = (o >> 2) & 1;
-        if (p.m == 12) {
-            uint64_t in[12][4];
-#pragma unroll
-            for (int a = 0; a < 12; ++a) unpack_pairs(__ldcs(reinterpret_cast<const uint4 *>(src + a * seg)), in[a]);
-            all_columns_12(std::make_integer_sequence<int, 12>{}, in, row_s, seg, o, p.sw, flip);
-        } else {
-            uint64_t v[4];
-            unpack_pairs(__ldcs(reinterpret_cast<const uint4 *>(src)), v);
-            finish_octet(v, row_s, o * 8, p.sw, flip);
-        }
-    }
-    __syncthreads();
-    // ---- phase 2 (the scaling rides on the last pass; without any pass it is applied in phase 3)
-    int start = 3;
-#pragma unroll 1
-    for (int k = 0; k < 3 && p.log[k]; ++k) {
-        run_pass(had_smem, p, nrows, start, p.log[k], k == 2 || p.log[k + 1] == 0);
-        start += p.log[k];
-        __syncthreads();
-    }
-    const float late_scale = p.log[0] ? 1.0f : p.scale;  // multiplying by one changes nothing
-
-    // ---- phase 3: one row per warp, one output group per lane
+    // where each output position reads its channel in a row's (swizzled) shared-memory image, as a byte
+    // offset: the same for every row, so it is worked out once per block (K <= 16384: 16 bits)
+    for (int j = threadIdx.x; j < p.K; j += kThreads)
+        offset_s[j] = static_cast<uint16_t>(swz(p.perm ? __ldg(p.perm + j) : j, p.sw) << 2);
     const float ts = p.codes ? __ldg(p.ts) : 1.0f;
-    const int gpr = p.K >> 4;
-    for (int r = warp; r < kRows; r += kThreads / 32) {
-        const int64_t row = row0 + r;
-        if (row >= p.rows_pad) break;
-        const bool live = row < p.rows;
-        const float *row_s = had_smem + static_cast<size_t>(r) * p.K;
-        for (int g0 = 0; g0 < gpr; g0 += 32) {
-            const int g = g0 + lane;
+
+    for (int64_t batch = blockIdx.x; batch < batches; batch += gridDim.x) {
+        const int64_t row0 = batch * kRows;
+        const int nrows = static_cast<int>(min(static_cast<int64_t>(kRows), max(static_cast<int64_t>(0), p.rows - row0)));
+        __syncthreads();  // the previous batch has been read out (and the offsets are in place)
+
+        // ---- phase 1
+        for (int u = threadIdx.x; u < nrows * octs; u += kThreads) {
+            const int r = u / octs, o = u - r * octs;
+            const uint16_t *src = p.X + (row0 + r) * p.ld + o * 8;
+            float *row_s = had_smem + static_cast<size_t>(r) * p.K;
+            if (p.m == 12) {
+                uint64_t in[12][4];
+#pragma unroll
+                for (int a = 0; a < 12; ++a) unpack_pairs(__ldcs(reinterpret_cast<const uint4 *>(src + a * seg)), in[a]);
+                all_columns_12(std::make_integer_sequence<int, 12>{}, in, row_s, seg, o, p.sw);
+            } else {
+                uint64_t v[4];
+                unpack_pairs(__ldcs(reinterpret_cast<const uint4 *>(src)), v);
+                finish_octet(v, row_s, o * 8, p.sw);
+            }
+        }
+        __syncthreads();
+        // ---- phase 2 (the scaling rides on the last pass; without any pass it is applied in phase 3)
+        int start = 3;
+#pragma unroll 1
+        for (int k = 0; k < 3 && p.log[k]; ++k) {
+            run_pass(had_smem, p, nrows, start, p.log[k], k == 2 || p.log[k + 1] == 0);
+            start += p.log[k];
+            __syncthreads();
+        }
+
+        // ---- phase 3: a warp takes a chunk of 32 output groups of TWO rows at a time, one group per lane:
+        // the read-out offsets are fetched once for both rows and the two quantizer chains interleave
+        const int rows_here = static_cast<int>(min(static_cast<int64_t>(kRows), p.rows_pad - row0));
+        const int row_pairs = (rows_here + 1) >> 1;
+        for (int c = warp; c < row_pairs * chunks; c += kThreads / 32) {
+            const int rp = c / chunks, g = (c - rp * chunks) * 32 + lane;
             const bool have = g < gpr;
-            float out[16];
+            uint32_t iw[8];
+            if (have) {
+                const uint4 i0 = reinterpret_cast<const uint4 *>(offset_s)[2 * g], i1 = reinterpret_cast<const uint4 *>(offset_s)[2 * g + 1];
+                iw[0] = i0.x, iw[1] = i0.y, iw[2] = i0.z, iw[3] = i0.w, iw[4] = i1.x, iw[5] = i1.y, iw[6] = i1.z, iw[7] = i1.w;
+            } else {
 #pragma unroll
-            for (int j = 0; j < 16; ++j) out[j] = 0.0f;
-            if (live && have) {
+                for (int j = 0; j < 8; ++j) iw[j] = 0;
+            }
+            float out[2][16];
+            bool live[2], present[2];
+            int64_t row[2];
 #pragma unroll
-                for (int h = 0; h < 4; ++h) {
-                    const int j0 = 16 * g + 4 * h;
-                    int4 idx = make_int4(j0, j0 + 1, j0 + 2, j0 + 3);
-                    if (p.perm) idx = __ldg(reinterpret_cast<const int4 *>(p.perm) + 4 * g + h);
-                    out[4 * h + 0] = __fmul_rn(row_s[swz(idx.x, p.sw)], late_scale);
-                    out[4 * h + 1] = __fmul_rn(row_s[swz(idx.y, p.sw)], late_scale);
-                    out[4 * h + 2] = __fmul_rn(row_s[swz(idx.z, p.sw)], late_scale);
-                    out[4 * h + 3] = __fmul_rn(row_s[swz(idx.w, p.sw)], late_scale);
-                }
-                if (p.y_out) {
-                    uint32_t yw[8];
+            for (int h = 0; h < 2; ++h) {
+                const int r = 2 * rp + h;
+                row[h] = row0 + r;
+                present[h] = r < rows_here;
+                live[h] = row[h] < p.rows;
+                const char *row_b = reinterpret_cast<const char *>(had_smem + static_cast<size_t>(r) * p.K);
 #pragma unroll
-                    for (int j = 0; j < 8; ++j)
-                        yw[j] = __bfloat16_as_ushort(__float2bfloat16_rn(out[2 * j])) |
-                                (static_cast<uint32_t>(__bfloat16_as_ushort(__float2bfloat16_rn(out[2 * j + 1]))) << 16);
-                    uint4 *ydst = reinterpret_cast<uint4 *>(p.y_out + row * p.K) + 2 * g;
-                    ydst[0] = make_uint4(yw[0], yw[1], yw[2], yw[3]);
-                    ydst[1] = make_uint4(yw[4], yw[5], yw[6], yw[7]);
+                for (int j = 0; j < 16; ++j) out[h][j] = 0.0f;
+                if (live[h] && have) {
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) {
+                        out[h][2 * j] = *reinterpret_cast<const float *>(row_b + (iw[j] & 0xFFFFu));
+                        out[h][2 * j + 1] = *reinterpret_cast<const float *>(row_b + (iw[j] >> 16));
+                    }
+                    if (!p.log[0]) {  // no pass of phase 2 carried the scaling
+#pragma unroll
+                        for (int j = 0; j < 16; ++j) out[h][j] = __fmul_rn(out[h][j], p.scale);
+                    }
+                    if (p.y_out) {
+                        uint32_t yw[8];
+#pragma unroll
+                        for (int j = 0; j < 8; ++j)
+                            yw[j] = __bfloat16_as_ushort(__float2bfloat16_rn(out[h][2 * j])) |
+                                    (static_cast<uint32_t>(__bfloat16_as_ushort(__float2bfloat16_rn(out[h][2 * j + 1]))) << 16);
+                        uint4 *ydst = reinterpret_cast<uint4 *>(p.y_out + row[h] * p.K) + 2 * g;
+                        ydst[0] = make_uint4(yw[0], yw[1], yw[2], yw[3]);
+                        ydst[1] = make_uint4(yw[4], yw[5], yw[6], yw[7]);
+                    }
                 }
             }
             if (!p.codes) continue;
-            float amax = 0.0f;
+            uint32_t sf8[2];
+            float rcp[2];
 #pragma unroll
-            for (int j = 0; j < 16; ++j) amax = fmaxf(amax, fabsf(out[j]));
-            uint32_t sf8;
-            float d, rcp;
-            pq::nvfp4_scale(amax, ts, sf8, d, rcp);
-            if (live && have) {
-                float y[8];
-                uint2 cw;
+            for (int h = 0; h < 2; ++h) {
+                float amax = 0.0f, d;
 #pragma unroll
-                for (int j = 0; j < 8; ++j) y[j] = __fmul_rn(out[j], rcp);
-                cw.x = pq::f32x8_to_e2m1(y);
-#pragma unroll
-                for (int j = 0; j < 8; ++j) y[j] = __fmul_rn(out[8 + j], rcp);
-                cw.y = pq::f32x8_to_e2m1(y);
-                *reinterpret_cast<uint2 *>(p.codes + row * (p.K >> 1) + g * 8) = cw;
+                for (int j = 0; j < 16; ++j) amax = fmaxf(amax, fabsf(out[h][j]));
+                pq::nvfp4_scale(amax, ts, sf8[h], d, rcp[h]);
             }
-            // scale bytes: four neighbouring groups sit in neighbouring lanes (padding rows write zeros)
-            uint32_t word = sf8;
-            word |= __shfl_down_sync(0xFFFFFFFFu, sf8, 1) << 8;
-            word |= __shfl_down_sync(0xFFFFFFFFu, sf8, 2) << 16;
-            word |= __shfl_down_sync(0xFFFFFFFFu, sf8, 3) << 24;
-            if (!have) continue;
-            if (SF_LAYOUT == PQ_SF_TCGEN05) {
-                if ((g & 3) == 0) *reinterpret_cast<uint32_t *>(p.sf + pq::sf_tc_offset(row, g, gpr >> 2)) = word;
-            } else if (live) {
-                if ((gpr & 3) == 0) {
-                    if ((g & 3) == 0) *reinterpret_cast<uint32_t *>(p.sf + row * gpr + g) = word;
-                } else {
-                    p.sf[row * gpr + g] = static_cast<uint8_t>(sf8);
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+                if (live[h] && have) {
+                    const uint64_t rcp2 = pack2(rcp[h], rcp[h]);
+                    float ylo[8], yhi[8];
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        unpack2(mul2(pack2(out[h][2 * j], out[h][2 * j + 1]), rcp2), ylo[2 * j], ylo[2 * j + 1]);
+                        unpack2(mul2(pack2(out[h][8 + 2 * j], out[h][9 + 2 * j]), rcp2), yhi[2 * j], yhi[2 * j + 1]);
+                    }
+                    *reinterpret_cast<uint2 *>(p.codes + row[h] * (p.K >> 1) + g * 8) =
+                        make_uint2(pq::f32x8_to_e2m1(ylo), pq::f32x8_to_e2m1(yhi));
+                }
+                // scale bytes: four neighbouring groups sit in neighbouring lanes (padding rows write zeros)
+                uint32_t word = sf8[h];
+                word |= __shfl_down_sync(0xFFFFFFFFu, sf8[h], 1) << 8;
+                word |= __shfl_down_sync(0xFFFFFFFFu, sf8[h], 2) << 16;
+                word |= __shfl_down_sync(0xFFFFFFFFu, sf8[h], 3) << 24;
+                if (!have || !present[h]) continue;
+                if (SF_LAYOUT == PQ_SF_TCGEN05) {
+                    if ((g & 3) == 0) *reinterpret_cast<uint32_t *>(p.sf + pq::sf_tc_offset(row[h], g, gpr >> 2)) = word;
+                } else if (live[h]) {
+                    if ((gpr & 3) == 0) {
+                        if ((g & 3) == 0) *reinterpret_cast<uint32_t *>(p.sf + row[h] * gpr + g) = word;
+                    } else {
+                        p.sf[row[h] * gpr + g] = static_cast<uint8_t>(sf8[h]);
+                    }
                 }
             }
         }
@@ -355,10 +401,14 @@ extern "C" pq_status pq_hadamard_quant_nvfp4(const void *X, int64_t M, int64_t K
     const size_t row_bytes = static_cast<size_t>(K) * sizeof(float);
     p.rows_per_block = static_cast<int>(kSmemBudget / row_bytes < kMaxRows ? kSmemBudget / row_bytes : kMaxRows);
     const int kRows = p.rows_per_block;
-    const size_t smem = static_cast<size_t>(kRows) * row_bytes;
+    const size_t smem = static_cast<size_t>(kRows) * row_bytes + static_cast<size_t>(K) * sizeof(uint16_t);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    const int64_t blocks = pq_ceil_div(p.rows_pad, kRows);
-    PQ_REQUIRE(blocks < (1ll << 31), PQ_ERR_SHAPE);
+    // persistent grid: as many blocks as fit on the device at once, walking over the batches of rows
+    int dev = 0, sms = 148;
+    if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    const int per_sm = static_cast<int>(std::min<size_t>(kBlocksPerSm, (227 * 1024) / (smem + 1024)));
+    const int64_t batches = pq_ceil_div(p.rows_pad, kRows);
+    const int64_t blocks = std::min<int64_t>(batches, static_cast<int64_t>(sms) * (per_sm > 0 ? per_sm : 1));
     auto launch = [&](auto kern) -> pq_status {
         if (smem > 48 * 1024)
             PQ_CUDA_OK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)));
