@@ -153,3 +153,32 @@ def test_repeated_launches_give_the_same_bits():
             wrong += int(not torch.equal(layer(x).view(torch.int16), r.view(torch.int16)))
     layer.check()
     assert wrong == 0
+
+
+def test_hadamard_producer_and_new_statistics_on_a_full_batch():
+    """The bench's stage sizes for the kernels added after the first set: the PermuQuant-H producer on the whole
+    4608 x 3072 batch (codes, scales in the tensor-core layout, bf16 output), the first-moment pass and the
+    group-256 error, all bit for bit."""
+    from test_gpu_gemm import to_tc
+    cfg = inputs.CONFIGS["qkv"]
+    x = inputs.activations(cfg, 0, 3)
+    xb, xd = inputs.bits(x), x.to(DEV)
+    g = torch.Generator().manual_seed(11)
+    perm = torch.randperm(cfg.K, generator=g).to(torch.int32)
+    _, _, yh, _ = O.hadamard_quant_nvfp4(xb, 1.0, quantize=False)
+    ts = O.tensor_scale(O.calib_stats(yh)[1])
+    tsd = torch.tensor([ts], dtype=torch.float32, device=DEV)
+    xq = torch.empty(cfg.M, cfg.K // 2, dtype=torch.uint8, device=DEV)
+    sf = torch.empty(B.sf_bytes(cfg.M, cfg.K, B.PQ_SF_TCGEN05), dtype=torch.uint8, device=DEV)
+    y = torch.empty(cfg.M, cfg.K, dtype=torch.bfloat16, device=DEV)
+    B.pq_hadamard_quant_nvfp4(xd, perm.to(DEV), tsd, xq, sf, B.PQ_SF_TCGEN05, y)
+    c_o, s_o, y_o, _ = O.hadamard_quant_nvfp4(xb, ts, perm.numpy())
+    assert np.array_equal(xq.cpu().numpy(), c_o)
+    assert np.array_equal(sf.cpu().numpy(), to_tc(s_o))
+    assert np.array_equal(inputs.bits(y.cpu()), y_o)
+    T = torch.zeros(cfg.K, dtype=torch.float64, device=DEV)
+    B.pq_calib_sum(xd, T, B.workspace(B.OP_CALIB_STATS, cfg.M, cfg.K))
+    assert np.array_equal(T.cpu().numpy(), O.calib_sum(xb))
+    err = torch.zeros(1, cfg.K // 256, dtype=torch.float64, device=DEV)
+    B.pq_group_error(xd, (B.KIND_INT, 4, 256), None, None, err, B.workspace(B.OP_GROUP_ERROR, cfg.M, cfg.K, 0, 1))
+    assert np.array_equal(err.cpu().numpy(), O.group_error(xb, 1, 4, 256))

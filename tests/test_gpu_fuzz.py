@@ -140,3 +140,48 @@ def test_weight_quantizer_and_gemm_on_random_shapes(case):
     assert np.array_equal(xq.cpu().numpy(), xq_o)
     ref = O.gemm_ref(xq_o, sfx_o, ts_x, wq_o, sfw_o, ts_w.item())
     assert_close(Y.view(M, N).float().cpu().numpy().astype(np.float64), ref, min_exact=0.95)
+
+
+@pytest.mark.parametrize("case", list(range(10)))
+def test_hadamard_producer_and_orders_on_random_shapes(case):
+    """Random row counts, widths (powers of two and 12 * 2^n), leading dimensions and scale layouts through
+    the PermuQuant-H producer, plus the first-moment pass and the variance / round-robin orders, with guard
+    bytes behind every output."""
+    rng = np.random.default_rng(5000 + case)
+    rows = int(rng.integers(1, 300))
+    K = int(rng.choice([64, 96, 128, 192, 384, 512, 768, 1536, 2048, 3072, 6144]))
+    ld = K + 8 * int(rng.integers(0, 5))
+    xd, xb = strided_input(rng, rows, K, ld)
+    ts = float(np.float32(rng.uniform(0.003, 0.05)))
+    tsd = torch.tensor([ts], dtype=torch.float32, device=DEV)
+    perm = rng.permutation(K).astype(np.int32)
+    layout = B.PQ_SF_TCGEN05 if K % 64 == 0 and rng.random() < 0.5 else B.PQ_SF_LINEAR
+    cbuf, codes = guarded(rows * K // 2)
+    nsf = B.sf_bytes(rows, K, layout)
+    sbuf, sf = guarded(nsf)
+    ybuf, y = guarded(rows * K * 2, torch.bfloat16)
+    B.pq_hadamard_quant_nvfp4(xd, torch.from_numpy(perm).to(DEV), tsd, codes.view(rows, K // 2), sf, layout, y.view(rows, K))
+    c_o, s_o, y_o, _ = O.hadamard_quant_nvfp4(xb, ts, perm)
+    assert np.array_equal(codes.view(rows, K // 2).cpu().numpy(), c_o)
+    assert np.array_equal(inputs.bits(y.view(rows, K).cpu()), y_o)
+    want_sf = to_tc(s_o) if layout == B.PQ_SF_TCGEN05 else s_o.reshape(-1)
+    assert np.array_equal(sf.cpu().numpy(), want_sf)
+    assert intact(cbuf, rows * K // 2) and intact(sbuf, nsf) and intact(ybuf, rows * K * 2)
+
+    T0 = rng.standard_normal(K)
+    T = torch.from_numpy(T0.copy()).to(DEV)
+    need = B.workspace_bytes(B.OP_CALIB_STATS, rows, K)
+    wbuf, ws = guarded(need)
+    B.pq_calib_sum(xd, T, ws)
+    To = O.calib_sum(xb, T0.copy())
+    assert np.array_equal(T.cpu().numpy(), To) and intact(wbuf, need)
+    So, _ = O.calib_stats(xb)
+    need = B.workspace_bytes(B.OP_SELECT_PERM, 0, K, 0, 1)
+    wbuf, ws = guarded(need)
+    pbuf, p = guarded(K * 4, torch.int32)
+    Sd = torch.from_numpy(So).to(DEV)
+    B.pq_order_by_variance(T, Sd, rows, p, ws)
+    assert np.array_equal(p.cpu().numpy(), O.order_by_variance(To, So, rows)) and intact(pbuf, K * 4)
+    group = int(rng.choice([16, 32, 64]))
+    B.pq_order_round_robin(Sd, group, p, ws)
+    assert np.array_equal(p.cpu().numpy(), O.order_round_robin(So, group)) and intact(pbuf, K * 4) and intact(wbuf, need)

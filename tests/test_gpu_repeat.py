@@ -64,6 +64,10 @@ def test_streaming_entry_points_repeat_bit_for_bit():
                        [xq, sfx]) == 0
     fq = torch.empty(M, K, dtype=torch.bfloat16, device=DEV)
     assert _repeat(lambda: B.pq_fakequant_int(x, (B.KIND_INT, 4, 64), None, fq), [fq]) == 0
+    # PermuQuant-H producer (persistent blocks, three phases over shared memory) and the first moments
+    assert _repeat(lambda: B.pq_hadamard_quant_nvfp4(x, perms[2], ts, xq, sfx, B.PQ_SF_TCGEN05, fq), [xq, sfx, fq]) == 0
+    T = torch.zeros(K, dtype=torch.float64, device=DEV)
+    assert _repeat(lambda: B.pq_calib_sum(x, T, ws), [T]) == 0
 
     N = 1024
     yref = torch.randn(M, N, device=DEV, generator=g)
