@@ -34,7 +34,7 @@ REPEAT_PAUSE_S = 0.25
 XROT = 10          # activation buffers the stand-alone streaming loops rotate over (283 MB)
 ORACLE_ROWS_MAX = 2048   # largest row sample of the workload the oracle legs use
 FP4_OVER_BF16 = 4.0  # nominal dense tensor ratio (9 vs 2.25 PFLOP/s)
-GEMM_DRAM_BYTES_PER_LAUNCH = 54.36e6   # ncu, 23.92 MB read + 30.44 MB written per launch of the bench workload (mean of two launches)
+GEMM_DRAM_BYTES_PER_LAUNCH = 53.60e6   # ncu, 23.92 MB read + 29.68 MB written per launch of the bench workload (mean of two launches)
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
 
