@@ -163,6 +163,29 @@ __device__ __forceinline__ uint32_t nvfp4_codes(const float (&x)[8], float r) {
     return f32x8_to_e2m1(y);
 }
 
+__device__ __forceinline__ uint32_t max_bf16x2(uint32_t a, uint32_t b) {
+    uint32_t r;
+    asm("max.bf16x2 %0, %1, %2;" : "=r"(r) : "r"(a), "r"(b));
+    return r;
+}
+
+// NVFP4 codes of eight bf16 values (four packed pairs) given the group's reciprocal decode scale: widen,
+// multiply in fp32 two at a time (packed f32x2: two IEEE products per instruction), convert.
+__device__ __forceinline__ uint32_t nvfp4_codes_packed(const uint4 &v, float r) {
+    const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+    uint64_t r2;
+    asm("mov.b64 %0, {%1, %1};" : "=l"(r2) : "f"(r));
+    float y[8];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        uint64_t x2, p;
+        asm("mov.b64 %0, {%1, %2};" : "=l"(x2) : "r"(w[i] << 16), "r"(w[i] & 0xFFFF0000u));
+        asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(p) : "l"(x2), "l"(r2));
+        asm("mov.b64 {%0, %1}, %2;" : "=f"(y[2 * i]), "=f"(y[2 * i + 1]) : "l"(p));
+    }
+    return f32x8_to_e2m1(y);
+}
+
 // Integer quantizer of Eq. 1-2: s = amax / Q, z = clamp(rint(x * (1/s)), -Q, Q).
 __device__ __forceinline__ void int_scale(float amax, float Qf, float &s, float &r) {
     s = __fdiv_rn(amax, Qf);

@@ -1,12 +1,11 @@
 // NVFP4 quantizers (runtime activations, offline permuted weights) and the integer fake-quant
 // of Eq. 1-2.
 //
-// All three are streaming kernels bound by HBM bandwidth: a thread owns 8 adjacent channels
-// (one 16-byte load), the TEAM = group/8 lanes that share a group reduce the absmax with
-// xor-shuffles, every lane then derives the group scale redundantly and converts its own
-// eight values.  A warp reads 512 contiguous bytes per load instruction and writes 128
-// contiguous bytes of codes; the scale bytes of four adjacent groups are merged into one
-// 32-bit store (the four bytes are adjacent in both scale layouts).
+// All three are streaming kernels bound by HBM bandwidth.  The activation quantizer gives a thread a
+// whole 16-channel group (one 32-byte load, no shuffles; a warp reads 1 KB of a row per instruction
+// and writes 256 contiguous bytes of codes).  The fake-quant kernels give a thread 8 adjacent
+// channels (one 16-byte load); the TEAM = group/8 lanes that share a group reduce the absmax with
+// xor-shuffles, every lane then derives the group scale redundantly and converts its own values.
 //
 // The permuted variants (weights, fake-quant with a gather) stage each row in shared memory
 // with coalesced 16-byte loads and gather from there, so global memory is still read once.
@@ -33,9 +32,8 @@ inline dim3 tile_grid(int64_t col_chunks, int64_t row_blocks) {
 
 // ---------------------------------------------------------------- activations (no gather)
 // One thread per 16-channel group: a 32-byte load (one 256-bit instruction when the tensor is
-// 32-byte aligned), the group's absmax, scale and codes in registers, an 8-byte store of codes.
-// The scale bytes of four adjacent groups are collected with shuffles into one 32-bit store
-// (adjacent in both scale layouts).  The index space covers the rows padded to a multiple of 128
+// 32-byte aligned), the group's absmax (on the bf16 pairs), scale and codes in registers (packed fp32
+// multiplies), an 8-byte store of codes and a one-byte store of the scale.  The index space covers the rows padded to a multiple of 128
 // in the tensor-core layout; padding rows only write zero scale bytes.  A block owns 8 (or 4) rows x 32
 // consecutive groups (a warp = 1 KB of one row), so no thread divides anything.
 template <bool WIDE>
@@ -84,30 +82,21 @@ quant_nvfp4_kernel(const uint16_t *__restrict__ X, int64_t rows, int64_t rows_pa
     for (int i = 0; i < kActRows; ++i) {
         const int64_t row = row0 + i * kActTileRows;
         const bool in_range = row < rows_pad && g < gpr, live = row < rows && g < gpr;
-        float x[8], y[8];
-        pq::unpack8(lo[i], x);
-        pq::unpack8(hi[i], y);
-        const float amax = fmaxf(pq::absmax8(x), pq::absmax8(y));
+        // group absmax on the bf16 pairs (a maximum of magnitudes selects one of its inputs: exact)
+        const uint32_t m = 0x7FFF7FFFu;
+        const uint32_t mx = pq::max_bf16x2(pq::max_bf16x2(pq::max_bf16x2(lo[i].x & m, lo[i].y & m), pq::max_bf16x2(lo[i].z & m, lo[i].w & m)),
+                                           pq::max_bf16x2(pq::max_bf16x2(hi[i].x & m, hi[i].y & m), pq::max_bf16x2(hi[i].z & m, hi[i].w & m)));
+        const float amax = fmaxf(__uint_as_float(mx << 16), __uint_as_float(mx & 0xFFFF0000u));
         uint32_t sf8;
         float d, r;
         pq::nvfp4_scale(amax, ts, sf8, d, r);
-        const uint32_t c0 = pq::nvfp4_codes(x, r), c1 = pq::nvfp4_codes(y, r);
+        const uint32_t c0 = pq::nvfp4_codes_packed(lo[i], r), c1 = pq::nvfp4_codes_packed(hi[i], r);
         if (live) __stcs(reinterpret_cast<uint2 *>(codes + row * (K >> 1) + static_cast<int64_t>(g) * 8), make_uint2(c0, c1));
-        // scale bytes of groups g .. g+3 (same row when the row holds a multiple of 4 groups)
-        uint32_t word = sf8;
-        word |= __shfl_down_sync(0xFFFFFFFFu, sf8, 1) << 8;
-        word |= __shfl_down_sync(0xFFFFFFFFu, sf8, 2) << 16;
-        word |= __shfl_down_sync(0xFFFFFFFFu, sf8, 3) << 24;
+        // one scale byte per thread: the lanes of a warp write runs of four adjacent bytes (adjacent in both
+        // layouts) in one instruction; padding rows of the tensor-core layout get zeros
         if (!in_range) continue;
-        if (SF_LAYOUT == PQ_SF_TCGEN05) {
-            if ((g & 3u) == 0) *reinterpret_cast<uint32_t *>(sf + pq::sf_tc_offset(row, g, gpr >> 2)) = word;
-        } else if (live) {
-            if ((gpr & 3u) == 0) {
-                if ((g & 3u) == 0) *reinterpret_cast<uint32_t *>(sf + row * gpr + g) = word;
-            } else {
-                sf[row * gpr + g] = static_cast<uint8_t>(sf8);
-            }
-        }
+        if (SF_LAYOUT == PQ_SF_TCGEN05) sf[pq::sf_tc_offset(row, g, gpr >> 2)] = static_cast<uint8_t>(sf8);
+        else if (live) sf[row * gpr + g] = static_cast<uint8_t>(sf8);
     }
 }
 
