@@ -71,6 +71,16 @@ def test_argument_errors_are_caught_on_the_host(L):
     assert L.pq_select_perm(p, 8, p, 8, 64, 5, p, None, 0, None) == 5                # the sort keys need a workspace
     assert L.pq_select_perm(p, 8, p, 8, 64, 5, p, odd, 1 << 20, None) == 3           # ... 256-byte aligned
     assert L.pq_order_by_absmax(p, 64, p, None, 0, None) == 5
+    assert L.pq_hadamard_quant_nvfp4(None, 8, 64, 64, None, p, p, p, 0, None, None) == 1          # NULL input
+    assert L.pq_hadamard_quant_nvfp4(p, 8, 64, 64, None, p, p, None, 0, None, None) == 1           # codes without scales
+    assert L.pq_hadamard_quant_nvfp4(p, 8, 64, 64, None, None, None, None, 0, None, None) == 1     # nothing to write
+    assert L.pq_hadamard_quant_nvfp4(p, 8, 80, 80, None, p, p, p, 0, None, None) == 2              # 5 * 16: no transform
+    assert L.pq_hadamard_quant_nvfp4(p, 8, 48, 48, None, p, p, p, 0, None, None) == 2              # segments of 4
+    assert L.pq_hadamard_quant_nvfp4(p, 8, 96, 96, None, p, p, p, 1, None, None) == 2              # K % 64 for the TC layout
+    assert L.pq_hadamard_quant_nvfp4(p, 8, 64, 64, odd, p, p, p, 0, None, None) == 3               # misaligned order
+    assert L.pq_calib_sum(p, 8, 64, 64, p, None, 0, None) == 5
+    assert L.pq_order_by_variance(p, p, 0, 64, p, p, 1 << 20, None) == 2                           # rows
+    assert L.pq_order_round_robin(p, 64, 24, p, p, 1 << 20, None) == 2                             # K % group
     assert L.pq_selftest_wait_expiry(None, 4, 1000, p, None) == 1
     assert L.pq_selftest_wait_expiry(p, 4, 0, p, None) == 2                           # limit out of range
     assert L.pq_selftest_wait_expiry(p, 4, 10 ** 12, p, None) == 2
