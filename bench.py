@@ -487,6 +487,12 @@ def run_ours(args):
                                                                           xq_rot[i % XROT], sfx_rot[i % XROT],
                                                                           B.PQ_SF_TCGEN05), it),
                   quant_bytes, bound="instruction issue / latency (one wave of 16 warps per SM; 16-21 instructions per element)")
+            # the same producer when the channels arrive already in output order (reordering absorbed upstream):
+            # no gather, a row never leaves the registers
+            stage(name + "_preordered",
+                  graph_loop(torch, lambda i: B.pq_norm_quant_nvfp4(xs[i % XROT], kind, av, bv, 1e-6, None, cal.ts_x,
+                                                                    xq_rot[i % XROT], sfx_rot[i % XROT], B.PQ_SF_TCGEN05), it),
+                  quant_bytes, bound="instruction issue (about 15 instructions per element), not the gather")
         # PermuQuant-H producer: Hadamard transform + reordering + quantizer (same bytes as the plain quantizer)
         stage("hadamard_quant", graph_loop(torch, lambda i: B.pq_hadamard_quant_nvfp4(xs[i % XROT], order, cal.ts_x,
                                                                                       xq_rot[i % XROT], sfx_rot[i % XROT],

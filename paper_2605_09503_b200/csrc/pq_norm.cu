@@ -12,8 +12,9 @@
 // one 32-bit store).  The normalized values exist only in registers, in fp32.  Optionally the
 // reordered bf16 tensor of the unfused kernel is written too.
 //
-// Two kernels: rows of up to 6400 channels go four per warp (below, second kernel); wider rows one
-// per warp, eight positions per lane (first kernel).
+// Three kernels: rows of up to 6400 channels go four per warp (below, second kernel); wider rows one
+// per warp, eight positions per lane (first kernel); and without a permutation (channels already in
+// output order) rows of up to 4096 channels never leave the registers (third kernel).
 #include "pq_common.cuh"
 
 namespace {
@@ -434,10 +435,133 @@ norm_quant_grouped_kernel(const uint16_t *__restrict__ H, int64_t rows, int64_t 
     }
 }
 
+// ---- channels already in output order --------------------------------------------------------------
+// When the reordering has been absorbed upstream (the previous linear layer writes its output columns in the
+// new order and the norm's parameters are stored reordered, App. C), the producer needs no gather: perm ==
+// NULL.  A warp then keeps its row in registers from the load to the codes: lane l owns the octets l, l + 32,
+// ... (the walk the statistics are defined on), the two octets of a 16-channel group sit in neighbouring
+// lanes (one shuffle for the group's absmax), every lane converts its own eight values and stores four bytes of
+// codes (128 contiguous bytes per warp instruction).  No shared memory, nothing but streaming.
+constexpr int kDirectMaxOcts = 16;  // octets per lane: rows of up to 4096 channels
+constexpr int kDirectThreads = 128;
+
+template <int KIND, int SF_LAYOUT, int NOCT>  // NOCT = octets per lane the registers are sized for
+__global__ void __launch_bounds__(kDirectThreads)
+norm_quant_ordered_kernel(const uint16_t *__restrict__ H, int64_t rows, int64_t rows_pad, int K, int64_t ld,
+                          const float *__restrict__ a, const float *__restrict__ b, float eps,
+                          const float *__restrict__ ts_ptr, uint8_t *__restrict__ codes, uint8_t *__restrict__ sf,
+                          uint16_t *__restrict__ y_out) {
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int64_t row = static_cast<int64_t>(blockIdx.x) * (blockDim.x >> 5) + warp;
+    if (row >= rows_pad) return;  // whole warps only
+    const bool live = row < rows;
+    const int octs = K >> 3, gpr = K >> 4;
+    const float ts = __ldg(ts_ptr);
+    uint4 raw[NOCT];
+#pragma unroll
+    for (int u = 0; u < NOCT; ++u) {
+        const int o = lane + 32 * u;
+        raw[u] = (live && o < octs) ? __ldcs(reinterpret_cast<const uint4 *>(H + row * ld + o * 8)) : make_uint4(0, 0, 0, 0);
+    }
+    // statistics in the lane walk: this lane's octets in ascending order, then the butterfly over the lanes
+    float p = 0.0f;
+#pragma unroll
+    for (int u = 0; u < NOCT; ++u) {
+        if (lane + 32 * u < octs) {
+            float x[8];
+            pq::unpack8(raw[u], x);
+#pragma unroll
+            for (int e = 0; e < 8; ++e) p = KIND == 0 ? __fmaf_rn(x[e], x[e], p) : __fadd_rn(p, x[e]);
+        }
+    }
+    p = lane_butterfly(p);
+    float inv, mu = 0.0f;
+    if (KIND == 0) {
+        inv = __fdiv_rn(1.0f, __fsqrt_rn(__fadd_rn(__fdiv_rn(p, static_cast<float>(K)), eps)));
+    } else {
+        mu = __fdiv_rn(p, static_cast<float>(K));
+        float q = 0.0f;
+#pragma unroll
+        for (int u = 0; u < NOCT; ++u) {
+            if (lane + 32 * u < octs) {
+                float x[8];
+                pq::unpack8(raw[u], x);
+#pragma unroll
+                for (int e = 0; e < 8; ++e) {
+                    const float d0 = __fsub_rn(x[e], mu);
+                    q = __fmaf_rn(d0, d0, q);
+                }
+            }
+        }
+        q = lane_butterfly(q);
+        inv = __fdiv_rn(1.0f, __fsqrt_rn(__fadd_rn(__fdiv_rn(q, static_cast<float>(K)), eps)));
+    }
+    if (!live) inv = 0.0f, mu = 0.0f;
+    // normalize, quantize, store: octet o = lane + 32 u, group o / 2 (its other octet is in lane ^ 1)
+#pragma unroll
+    for (int u = 0; u < NOCT; ++u) {
+        const int o = lane + 32 * u;
+        if (32 * u >= octs) break;  // uniform over the warp
+        const bool have = o < octs;
+        float out[8];
+#pragma unroll
+        for (int e = 0; e < 8; ++e) out[e] = 0.0f;
+        if (live && have) {
+            float x[8];
+            pq::unpack8(raw[u], x);
+            const float4 a0 = __ldg(reinterpret_cast<const float4 *>(a) + 2 * o), a1 = __ldg(reinterpret_cast<const float4 *>(a) + 2 * o + 1);
+            const float w[8] = {a0.x, a0.y, a0.z, a0.w, a1.x, a1.y, a1.z, a1.w};
+            if (KIND == 0) {
+#pragma unroll
+                for (int e = 0; e < 8; ++e) out[e] = __fmul_rn(__fmul_rn(x[e], inv), w[e]);
+            } else {
+                const float4 b0 = __ldg(reinterpret_cast<const float4 *>(b) + 2 * o), b1 = __ldg(reinterpret_cast<const float4 *>(b) + 2 * o + 1);
+                const float sh[8] = {b0.x, b0.y, b0.z, b0.w, b1.x, b1.y, b1.z, b1.w};
+#pragma unroll
+                for (int e = 0; e < 8; ++e)
+                    out[e] = __fmaf_rn(__fmul_rn(__fsub_rn(x[e], mu), inv), __fadd_rn(1.0f, w[e]), sh[e]);
+            }
+        }
+        float amax = pq::absmax8(out);
+        amax = fmaxf(amax, __shfl_xor_sync(0xFFFFFFFFu, amax, 1));
+        uint32_t sf8;
+        float d, rcp;
+        pq::nvfp4_scale(amax, ts, sf8, d, rcp);
+        if (live && have) {
+            *reinterpret_cast<uint32_t *>(codes + row * (K >> 1) + o * 4) = pq::nvfp4_codes(out, rcp);
+            if (y_out) {
+                uint32_t yw[4];
+#pragma unroll
+                for (int j = 0; j < 4; ++j)
+                    yw[j] = __bfloat16_as_ushort(__float2bfloat16_rn(out[2 * j])) |
+                            (static_cast<uint32_t>(__bfloat16_as_ushort(__float2bfloat16_rn(out[2 * j + 1]))) << 16);
+                reinterpret_cast<uint4 *>(y_out + row * K)[o] = make_uint4(yw[0], yw[1], yw[2], yw[3]);
+            }
+        }
+        // the scale byte of a group: written by the lane that holds its first octet (padding rows write zeros)
+        if (!have || (o & 1)) continue;
+        const int g = o >> 1;
+        if (SF_LAYOUT == PQ_SF_TCGEN05) sf[pq::sf_tc_offset(row, g, gpr >> 2)] = static_cast<uint8_t>(sf8);
+        else if (live) sf[row * gpr + g] = static_cast<uint8_t>(sf8);
+    }
+}
+
 template <int KIND, int SF_LAYOUT>
 pq_status launch(const uint16_t *H, int64_t M, int64_t rows_pad, int K, int64_t ld, const float *a, const float *b,
                  float eps, const int32_t *perm, const float *ts, uint8_t *codes, uint8_t *sf, uint16_t *y_out,
                  cudaStream_t st) {
+    // no reordering to apply and a row fits a warp's registers: the streaming kernel
+    if (!perm && K <= 256 * kDirectMaxOcts) {
+        const int64_t blocks = pq_ceil_div(rows_pad, kDirectThreads / 32);
+        PQ_REQUIRE(blocks < (1ll << 31), PQ_ERR_SHAPE);
+        const unsigned grid = static_cast<unsigned>(blocks);
+        const int noct = static_cast<int>(pq_ceil_div(K, 256));
+        if (noct <= 4) norm_quant_ordered_kernel<KIND, SF_LAYOUT, 4><<<grid, kDirectThreads, 0, st>>>(H, M, rows_pad, K, ld, a, b, eps, ts, codes, sf, y_out);
+        else if (noct <= 8) norm_quant_ordered_kernel<KIND, SF_LAYOUT, 8><<<grid, kDirectThreads, 0, st>>>(H, M, rows_pad, K, ld, a, b, eps, ts, codes, sf, y_out);
+        else if (noct <= 12) norm_quant_ordered_kernel<KIND, SF_LAYOUT, 12><<<grid, kDirectThreads, 0, st>>>(H, M, rows_pad, K, ld, a, b, eps, ts, codes, sf, y_out);
+        else norm_quant_ordered_kernel<KIND, SF_LAYOUT, 16><<<grid, kDirectThreads, 0, st>>>(H, M, rows_pad, K, ld, a, b, eps, ts, codes, sf, y_out);
+        return pq_launch_status();
+    }
     // up to 6400 channels: four rows per warp, four warps per block (two blocks per SM at 3072 channels)
     const size_t group_smem = static_cast<size_t>(kGroupWarps) * kGroupRows * K * 2;
     if (group_smem <= kSmemBudget) {

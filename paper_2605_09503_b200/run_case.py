@@ -31,6 +31,7 @@ def main():
     ap.add_argument("--iters", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--rot", type=int, default=4)
+    ap.add_argument("--ordered", action="store_true", help="norm_quant: channels already in output order (no permutation)")
     ap.add_argument("--graph", action="store_true",
                     help="capture the timed launches in one CUDA graph (takes the host's launch rate out of the number)")
     args = ap.parse_args()
@@ -82,7 +83,7 @@ def main():
         sfx = [torch.empty(B.sf_bytes(M, K, 1), dtype=torch.uint8, device=dev) for _ in range(R)]
         av = torch.randn(K, device=dev, generator=g) * 0.2
         bv = torch.randn(K, device=dev, generator=g)
-        pm = perms[0].contiguous()
+        pm = None if args.ordered else perms[0].contiguous()
         bytes_moved = M * K * 2 + M * K // 2 + M * K // 16
         fn = lambda i: B.pq_norm_quant_nvfp4(X[i % R], args.kind, av, bv, 1e-6, pm, ts, xq[i % R], sfx[i % R],
                                              B.PQ_SF_TCGEN05)
