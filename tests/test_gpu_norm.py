@@ -26,7 +26,11 @@ def _case(M, K, seed):
 @pytest.mark.parametrize("kind", [B.NORM_RMS, B.NORM_ADALN])
 @pytest.mark.parametrize("layout", [B.PQ_SF_LINEAR, B.PQ_SF_TCGEN05])
 @pytest.mark.parametrize("M,K,with_perm", [(130, 512, True), (37, 3072, True), (64, 3072, False), (5, 12288, True),
-                                           (300, 1024, True), (1, 64, False), (23, 1536, True), (18, 6400, True)])
+                                           (300, 1024, True), (1, 64, False), (23, 1536, True), (18, 6400, True),
+                                           # channels already in output order: the register-resident kernel at each of
+                                           # its four register sizes, and the fall-back for rows wider than 4096
+                                           (150, 1024, False), (33, 2048, False), (20, 4096, False), (7, 6400, False),
+                                           (129, 2560, False)])
 def test_norm_quant_bit_exact(kind, layout, M, K, with_perm):
     h, a, b, perm = _case(M, K, seed=M + K + kind)
     ts, eps = 0.011, 1e-6
