@@ -521,7 +521,7 @@ def run_ours(args):
         stage("quant_act_nvfp4_candidate_order",
               graph_loop(torch, lambda i: B.pq_quant_act_nvfp4_perm(xs[i % XROT], order, cal.ts_x, xq_rot[i % XROT],
                                                                     sfx_rot[i % XROT], B.PQ_SF_TCGEN05), it),
-              quant_bytes, note="calibration-time gather quantizer, one block per row")
+              quant_bytes, note="calibration-time gather quantizer: four rows per warp share indices and gathers")
         del yrefs, yqs
 
     # ---- end to end: host tensors in, host tensor out, through the C ABI

@@ -266,9 +266,12 @@ pq_status pq_quant_act_nvfp4(const void *X, int64_t M, int64_t K, int64_t ld, co
 
 /* The same quantizer with a channel order applied on the way in (codes and scales of X P): the
  * calibration-time form, used to evaluate a candidate order on the layer output (pq_output_error)
- * before any producer has been rewritten to emit permuted activations.  One block per row stages
- * the row in shared memory and gathers from there; perm == NULL is pq_quant_act_nvfp4.
- *   perm : device int32 [K].  K <= 16384.  Other arguments as for pq_quant_act_nvfp4. */
+ * before any producer has been rewritten to emit permuted activations.  Rows are staged in shared
+ * memory and gathered from there (rows of up to 6400 channels four per warp, sharing indices and
+ * gathers, when perm is 16-byte aligned; otherwise one block per row; same results);
+ * perm == NULL is pq_quant_act_nvfp4.
+ *   perm : device int32 [K], values in [0, K) (not checked).  K <= 16384.  Other arguments as for
+ *   pq_quant_act_nvfp4. */
 pq_status pq_quant_act_nvfp4_perm(const void *X, int64_t M, int64_t K, int64_t ld, const int32_t *perm,
                                   const float *ts_x, uint8_t *codes, uint8_t *sf, int sf_layout,
                                   void *stream);

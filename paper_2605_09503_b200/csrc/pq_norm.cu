@@ -296,14 +296,20 @@ norm_quant_grouped_kernel(const uint16_t *__restrict__ H, int64_t rows, int64_t 
                 for (int r = 0; r < R; ++r) {
                     float x[8];
                     pq::unpack8(v[u][r], x);
+                    if (KIND != 2) {
 #pragma unroll
-                    for (int e = 0; e < 8; ++e) p[r] = KIND == 0 ? __fmaf_rn(x[e], x[e], p[r]) : __fadd_rn(p[r], x[e]);
+                        for (int e = 0; e < 8; ++e) p[r] = KIND == 0 ? __fmaf_rn(x[e], x[e], p[r]) : __fadd_rn(p[r], x[e]);
+                    }
                 }
             }
         }
+        if (KIND != 2) {
 #pragma unroll
-        for (int r = 0; r < R; ++r) p[r] = lane_butterfly(p[r]);
-        if (KIND == 0) {
+            for (int r = 0; r < R; ++r) p[r] = lane_butterfly(p[r]);
+        }
+        if (KIND == 2) {
+            // no normalization: the values themselves are quantized
+        } else if (KIND == 0) {
 #pragma unroll
             for (int r = 0; r < R; ++r)
                 if (r < nlive) inv[r] = __fdiv_rn(1.0f, __fsqrt_rn(__fadd_rn(__fdiv_rn(p[r], static_cast<float>(K)), eps)));
@@ -366,8 +372,10 @@ norm_quant_grouped_kernel(const uint16_t *__restrict__ H, int64_t rows, int64_t 
                 if (perm) idx = __ldg(reinterpret_cast<const int4 *>(perm) + (POS / 4) * q + h);
                 g[4 * h + 0] = channel_rows<R>(xs, idx.x), g[4 * h + 1] = channel_rows<R>(xs, idx.y);
                 g[4 * h + 2] = channel_rows<R>(xs, idx.z), g[4 * h + 3] = channel_rows<R>(xs, idx.w);
-                const float4 a4 = __ldg(reinterpret_cast<const float4 *>(a) + (POS / 4) * q + h);
-                w[4 * h + 0] = a4.x, w[4 * h + 1] = a4.y, w[4 * h + 2] = a4.z, w[4 * h + 3] = a4.w;
+                if (KIND != 2) {
+                    const float4 a4 = __ldg(reinterpret_cast<const float4 *>(a) + (POS / 4) * q + h);
+                    w[4 * h + 0] = a4.x, w[4 * h + 1] = a4.y, w[4 * h + 2] = a4.z, w[4 * h + 3] = a4.w;
+                }
                 if (KIND == 1) {
                     const float4 b4 = __ldg(reinterpret_cast<const float4 *>(b) + (POS / 4) * q + h);
                     sh[4 * h + 0] = b4.x, sh[4 * h + 1] = b4.y, sh[4 * h + 2] = b4.z, sh[4 * h + 3] = b4.w;
@@ -387,8 +395,9 @@ norm_quant_grouped_kernel(const uint16_t *__restrict__ H, int64_t rows, int64_t 
 #pragma unroll
             for (int j = 0; j < POS; ++j) {
                 const float v = row_value(g[j], r);
-                out[j] = KIND == 0 ? __fmul_rn(__fmul_rn(v, inv[r]), w[j])
-                                   : __fmaf_rn(__fmul_rn(__fsub_rn(v, mu[r]), inv[r]), w[j], sh[j]);
+                out[j] = KIND == 2   ? v
+                         : KIND == 0 ? __fmul_rn(__fmul_rn(v, inv[r]), w[j])
+                                     : __fmaf_rn(__fmul_rn(__fsub_rn(v, mu[r]), inv[r]), w[j], sh[j]);
                 amax = fmaxf(amax, fabsf(out[j]));
             }
             if (!(live && have)) amax = 0.0f;  // nothing of such a row or group is stored but a zero scale byte
@@ -589,7 +598,36 @@ pq_status launch(const uint16_t *H, int64_t M, int64_t rows_pad, int K, int64_t 
     return pq_launch_status();
 }
 
+template <int SF_LAYOUT>
+pq_status launch_gather_only(const uint16_t *X, int64_t M, int64_t rows_pad, int K, int64_t ld, const int32_t *perm,
+                             const float *ts, uint8_t *codes, uint8_t *sf, cudaStream_t st) {
+    const size_t group_smem = static_cast<size_t>(kGroupWarps) * kGroupRows * K * 2;
+    if (group_smem > 40 * 1024)
+        PQ_CUDA_OK(cudaFuncSetAttribute(norm_quant_grouped_kernel<2, SF_LAYOUT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                        static_cast<int>(group_smem)));
+    const int64_t blocks = pq_ceil_div(rows_pad, kGroupWarps * kGroupRows);
+    PQ_REQUIRE(blocks < (1ll << 31), PQ_ERR_SHAPE);
+    norm_quant_grouped_kernel<2, SF_LAYOUT><<<static_cast<unsigned>(blocks), kGroupWarps * kSplit * 32, group_smem, st>>>(
+        X, M, rows_pad, K, ld, nullptr, nullptr, 0.0f, perm, ts, codes, sf, nullptr);
+    return pq_launch_status();
+}
+
 }  // namespace
+
+// The gather quantizer of pq_quant_act_nvfp4_perm for rows the four-rows-per-warp kernel can hold: that kernel
+// with the normalization left out (the gathered values themselves are quantized).
+bool pq_gather_quant_grouped_fits(int64_t K) {
+    return K > 0 && static_cast<size_t>(kGroupWarps) * kGroupRows * static_cast<size_t>(K) * 2 <= kSmemBudget;
+}
+pq_status pq_gather_quant_grouped(const void *X, int64_t M, int64_t K, int64_t ld, const int32_t *perm, const float *ts_x,
+                                  uint8_t *codes, uint8_t *sf, int sf_layout, void *stream) {
+    const int64_t rows_pad = sf_layout == PQ_SF_TCGEN05 ? pq_ceil_div(M, 128) * 128 : M;
+    const uint16_t *x = static_cast<const uint16_t *>(X);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    return sf_layout == PQ_SF_TCGEN05
+               ? launch_gather_only<PQ_SF_TCGEN05>(x, M, rows_pad, static_cast<int>(K), ld, perm, ts_x, codes, sf, st)
+               : launch_gather_only<PQ_SF_LINEAR>(x, M, rows_pad, static_cast<int>(K), ld, perm, ts_x, codes, sf, st);
+}
 
 extern "C" pq_status pq_norm_quant_nvfp4(const void *H, int64_t M, int64_t K, int64_t ld, int kind, const float *a,
                                          const float *b, float eps, const int32_t *perm, const float *ts_x,

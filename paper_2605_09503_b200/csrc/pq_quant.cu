@@ -366,6 +366,11 @@ extern "C" pq_status pq_quant_act_nvfp4_perm(const void *X, int64_t M, int64_t K
     PQ_REQUIRE(M > 0 && K > 0 && K % 16 == 0 && K <= 16384 && ld >= K, PQ_ERR_SHAPE);
     PQ_REQUIRE(sf_layout == PQ_SF_LINEAR || K % 64 == 0, PQ_ERR_SHAPE);
     PQ_REQUIRE(pq_aligned16(X) && ld % 8 == 0 && pq_aligned16(codes) && pq_aligned16(sf), PQ_ERR_ALIGN);
+    // rows of up to 6400 channels: four rows per warp share the indices and one gather (the fused producer's
+    // kernel without its normalization); wider rows, or an index vector it cannot load 16 bytes at a time: one
+    // block per row
+    if (pq_gather_quant_grouped_fits(K) && pq_aligned16(perm))
+        return pq_gather_quant_grouped(X, M, K, ld, perm, ts_x, codes, sf, sf_layout, stream);
     return launch_gather(static_cast<const uint16_t *>(X), M, K, ld, perm, nullptr, ts_x, codes, sf, sf_layout,
                          static_cast<cudaStream_t>(stream));
 }

@@ -55,7 +55,7 @@ def test_output_error_full_size_output_of_the_bench_layer():
 
 
 @pytest.mark.parametrize("layout", [B.PQ_SF_LINEAR, B.PQ_SF_TCGEN05])
-@pytest.mark.parametrize("M,K", [(130, 512), (37, 3072), (5, 16384)])
+@pytest.mark.parametrize("M,K", [(130, 512), (37, 3072), (5, 16384), (129, 6400), (3, 6464), (2, 64)])
 def test_quant_act_with_an_order_is_bit_exact(layout, M, K):
     g = torch.Generator().manual_seed(M + K)
     x = (torch.randn(M, K, generator=g) * torch.exp(torch.randn(K, generator=g))).to(torch.bfloat16)
@@ -72,6 +72,29 @@ def test_quant_act_with_an_order_is_bit_exact(layout, M, K):
         lin = torch.empty(M * K // 16, dtype=torch.uint8, device=DEV)
         B.pq_sf_to_linear(sf, M, K, lin)
         assert np.array_equal(lin.cpu().numpy().reshape(M, K // 16), s_o)
+
+
+def test_quant_act_with_an_order_whose_index_vector_is_only_4_byte_aligned():
+    """The four-rows-per-warp kernel loads indices 16 bytes at a time; an index vector that is not 16-byte
+    aligned takes the one-block-per-row kernel.  Same codes and scales either way."""
+    M, K = 70, 3072
+    g = torch.Generator().manual_seed(5)
+    x = (torch.randn(M, K, generator=g) * torch.exp(torch.randn(K, generator=g))).to(torch.bfloat16)
+    perm = torch.randperm(K, generator=g).to(torch.int32)
+    ts = torch.tensor([float(x.float().abs().max()) / 2688.0], dtype=torch.float32, device=DEV)
+    buf = torch.zeros(K + 4, dtype=torch.int32, device=DEV)
+    buf[1:K + 1] = perm.to(DEV)
+    shifted = buf[1:K + 1]
+    assert shifted.data_ptr() % 16 == 4
+    out = []
+    for pm in (perm.to(DEV), shifted):
+        codes = torch.empty(M, K // 2, dtype=torch.uint8, device=DEV)
+        sf = torch.full((B.sf_bytes(M, K, B.PQ_SF_TCGEN05),), 0xEE, dtype=torch.uint8, device=DEV)
+        B.pq_quant_act_nvfp4_perm(x.to(DEV), pm, ts, codes, sf, B.PQ_SF_TCGEN05)
+        out.append((codes.cpu().numpy(), sf.cpu().numpy()))
+    c_o, _ = O.quant_nvfp4(inputs.bits(x), float(ts.item()), perm.numpy())
+    assert np.array_equal(out[0][0], c_o) and np.array_equal(out[1][0], c_o)
+    assert np.array_equal(out[0][1], out[1][1])
 
 
 def test_selection_by_output_error_matches_the_oracle_route():
