@@ -509,7 +509,7 @@ def run_ours(args):
         ws_qw = B.workspace(B.OP_QUANT_WEIGHT, N, K)
         stage("quant_weight", graph_loop(torch, lambda i: B.pq_quant_weight(Wt, cal.perms, cal.select, wq2, sfw2, 1, tsw2,
                                                                             ws_qw), max(5, it // 4)),
-              2 * N * K * 2 + N * K // 2 + N * K // 16, note="two reads of W (absmax, then gather + quantize)")
+              2 * N * K * 2 + N * K // 2 + N * K // 16, note="two reads of W (absmax, then gather + quantize, four rows per warp)")
 
         # output-side calibration error: fp32 reference and bf16 layer output of one batch (6 B per element)
         yrefs = [torch.randn(M, N, device=dev) for _ in range(2)]

@@ -62,11 +62,13 @@ static inline int pq_device_slot() {
 pq_status pq_quant_act_nvfp4_shaped(const void *X, int64_t M, int64_t K, int64_t ld, const float *ts_x, uint8_t *codes,
                                     uint8_t *sf, int sf_layout, int small_blocks, void *stream);
 
-// pq_quant_act_nvfp4_perm through the four-rows-per-warp producer kernel without a normalization
-// (library-internal; defined in pq_norm.cu).  Arguments already validated by the caller.
+// The gather quantizers (pq_quant_act_nvfp4_perm, pq_quant_weight) through the four-rows-per-warp producer
+// kernel without a normalization (library-internal; defined in pq_norm.cu).  perm / perm_select as for
+// pq_quant_weight; perm 16-byte aligned; arguments already validated by the caller.
 bool pq_gather_quant_grouped_fits(int64_t K);
-pq_status pq_gather_quant_grouped(const void *X, int64_t M, int64_t K, int64_t ld, const int32_t *perm, const float *ts_x,
-                                  uint8_t *codes, uint8_t *sf, int sf_layout, void *stream);
+pq_status pq_gather_quant_grouped(const void *X, int64_t M, int64_t K, int64_t ld, const int32_t *perm,
+                                  const int32_t *perm_select, const float *ts_x, uint8_t *codes, uint8_t *sf,
+                                  int sf_layout, void *stream);
 
 #ifdef __CUDACC__
 

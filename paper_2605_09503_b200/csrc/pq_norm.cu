@@ -236,8 +236,12 @@ template <int KIND, int SF_LAYOUT>
 __global__ void __launch_bounds__(32 * kGroupWarps * kSplit, 2)
 norm_quant_grouped_kernel(const uint16_t *__restrict__ H, int64_t rows, int64_t rows_pad, int K, int64_t ld,
                         const float *__restrict__ a, const float *__restrict__ b, float eps,
-                        const int32_t *__restrict__ perm, const float *__restrict__ ts_ptr,
-                        uint8_t *__restrict__ codes, uint8_t *__restrict__ sf, uint16_t *__restrict__ y_out) {
+                        const int32_t *__restrict__ perm, const int32_t *__restrict__ perm_select,
+                        const float *__restrict__ ts_ptr, uint8_t *__restrict__ codes, uint8_t *__restrict__ sf,
+                        uint16_t *__restrict__ y_out) {
+    // perm_select given: perm is a table of candidate orders [., K] and {best, accept} on the device name the
+    // row best - 1, or the original order (the offline weight quantizer, whose decision never visits the host)
+    if (perm_select) perm = perm_select[1] ? perm + static_cast<int64_t>(perm_select[0] - 1) * K : nullptr;
     extern __shared__ __align__(16) uint16_t row_s[];  // [row groups][K][R rows] bf16 bit patterns
     __shared__ float stat_s[kGroupWarps][2 * kGroupRows];
     constexpr int R = kGroupRows;
@@ -580,7 +584,7 @@ pq_status launch(const uint16_t *H, int64_t M, int64_t rows_pad, int K, int64_t 
         const int64_t blocks = pq_ceil_div(rows_pad, kGroupWarps * kGroupRows);
         PQ_REQUIRE(blocks < (1ll << 31), PQ_ERR_SHAPE);
         norm_quant_grouped_kernel<KIND, SF_LAYOUT><<<static_cast<unsigned>(blocks), kGroupWarps * kSplit * 32, group_smem, st>>>(
-            H, M, rows_pad, K, ld, a, b, eps, perm, ts, codes, sf, y_out);
+            H, M, rows_pad, K, ld, a, b, eps, perm, nullptr, ts, codes, sf, y_out);
         return pq_launch_status();
     }
     // wider rows: one warp per row, the row as bf16 in shared memory: 8 rows per block up to 12800 channels
@@ -600,7 +604,7 @@ pq_status launch(const uint16_t *H, int64_t M, int64_t rows_pad, int K, int64_t 
 
 template <int SF_LAYOUT>
 pq_status launch_gather_only(const uint16_t *X, int64_t M, int64_t rows_pad, int K, int64_t ld, const int32_t *perm,
-                             const float *ts, uint8_t *codes, uint8_t *sf, cudaStream_t st) {
+                             const int32_t *perm_select, const float *ts, uint8_t *codes, uint8_t *sf, cudaStream_t st) {
     const size_t group_smem = static_cast<size_t>(kGroupWarps) * kGroupRows * K * 2;
     if (group_smem > 40 * 1024)
         PQ_CUDA_OK(cudaFuncSetAttribute(norm_quant_grouped_kernel<2, SF_LAYOUT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -608,25 +612,26 @@ pq_status launch_gather_only(const uint16_t *X, int64_t M, int64_t rows_pad, int
     const int64_t blocks = pq_ceil_div(rows_pad, kGroupWarps * kGroupRows);
     PQ_REQUIRE(blocks < (1ll << 31), PQ_ERR_SHAPE);
     norm_quant_grouped_kernel<2, SF_LAYOUT><<<static_cast<unsigned>(blocks), kGroupWarps * kSplit * 32, group_smem, st>>>(
-        X, M, rows_pad, K, ld, nullptr, nullptr, 0.0f, perm, ts, codes, sf, nullptr);
+        X, M, rows_pad, K, ld, nullptr, nullptr, 0.0f, perm, perm_select, ts, codes, sf, nullptr);
     return pq_launch_status();
 }
 
 }  // namespace
 
-// The gather quantizer of pq_quant_act_nvfp4_perm for rows the four-rows-per-warp kernel can hold: that kernel
-// with the normalization left out (the gathered values themselves are quantized).
+// The gather quantizer of pq_quant_act_nvfp4_perm and pq_quant_weight for rows the four-rows-per-warp kernel can
+// hold: that kernel with the normalization left out (the gathered values themselves are quantized).
 bool pq_gather_quant_grouped_fits(int64_t K) {
     return K > 0 && static_cast<size_t>(kGroupWarps) * kGroupRows * static_cast<size_t>(K) * 2 <= kSmemBudget;
 }
-pq_status pq_gather_quant_grouped(const void *X, int64_t M, int64_t K, int64_t ld, const int32_t *perm, const float *ts_x,
-                                  uint8_t *codes, uint8_t *sf, int sf_layout, void *stream) {
+pq_status pq_gather_quant_grouped(const void *X, int64_t M, int64_t K, int64_t ld, const int32_t *perm,
+                                  const int32_t *perm_select, const float *ts_x, uint8_t *codes, uint8_t *sf,
+                                  int sf_layout, void *stream) {
     const int64_t rows_pad = sf_layout == PQ_SF_TCGEN05 ? pq_ceil_div(M, 128) * 128 : M;
     const uint16_t *x = static_cast<const uint16_t *>(X);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     return sf_layout == PQ_SF_TCGEN05
-               ? launch_gather_only<PQ_SF_TCGEN05>(x, M, rows_pad, static_cast<int>(K), ld, perm, ts_x, codes, sf, st)
-               : launch_gather_only<PQ_SF_LINEAR>(x, M, rows_pad, static_cast<int>(K), ld, perm, ts_x, codes, sf, st);
+               ? launch_gather_only<PQ_SF_TCGEN05>(x, M, rows_pad, static_cast<int>(K), ld, perm, perm_select, ts_x, codes, sf, st)
+               : launch_gather_only<PQ_SF_LINEAR>(x, M, rows_pad, static_cast<int>(K), ld, perm, perm_select, ts_x, codes, sf, st);
 }
 
 extern "C" pq_status pq_norm_quant_nvfp4(const void *H, int64_t M, int64_t K, int64_t ld, int kind, const float *a,

@@ -8,7 +8,9 @@
 // xor-shuffles, every lane then derives the group scale redundantly and converts its own values.
 //
 // The permuted variants (weights, fake-quant with a gather) stage each row in shared memory
-// with coalesced 16-byte loads and gather from there, so global memory is still read once.
+// with coalesced 16-byte loads and gather from there, so global memory is still read once.  For
+// NVFP4 and rows of up to 6400 channels the gather runs in the fused producer's kernel (pq_norm.cu,
+// four rows per warp sharing indices and gathers) with its normalization compiled out.
 #include "pq_common.cuh"
 
 namespace {
@@ -370,7 +372,7 @@ extern "C" pq_status pq_quant_act_nvfp4_perm(const void *X, int64_t M, int64_t K
     // kernel without its normalization); wider rows, or an index vector it cannot load 16 bytes at a time: one
     // block per row
     if (pq_gather_quant_grouped_fits(K) && pq_aligned16(perm))
-        return pq_gather_quant_grouped(X, M, K, ld, perm, ts_x, codes, sf, sf_layout, stream);
+        return pq_gather_quant_grouped(X, M, K, ld, perm, nullptr, ts_x, codes, sf, sf_layout, stream);
     return launch_gather(static_cast<const uint16_t *>(X), M, K, ld, perm, nullptr, ts_x, codes, sf, sf_layout,
                          static_cast<cudaStream_t>(stream));
 }
@@ -402,7 +404,9 @@ extern "C" pq_status pq_quant_weight(const void *Wt, int64_t N, int64_t K, int64
     }
     weight_scale_kernel<<<1, 1, 0, st>>>(amax_bits, ts_w);
     if (!perm) return pq_quant_act_nvfp4(Wt, N, K, ld, ts_w, codes, sf, sf_layout, stream);
-
+    // rows of up to 6400 channels: four rows per warp share the indices and one gather
+    if (pq_gather_quant_grouped_fits(K) && pq_aligned16(perm))
+        return pq_gather_quant_grouped(Wt, N, K, ld, perm, perm_select, ts_w, codes, sf, sf_layout, stream);
     return launch_gather(w, N, K, ld, perm, perm_select, ts_w, codes, sf, sf_layout, st);
 }
 

@@ -175,9 +175,9 @@ def test_quant_weight_bit_exact(layout, N, K, with_perm):
         assert np.array_equal(sf.cpu().numpy().reshape(N, K // 16), so)
 
 
-def test_quant_weight_device_side_decision():
+@pytest.mark.parametrize("N,K", [(64, 256), (5, 8192)])  # four rows per warp / one block per row
+def test_quant_weight_device_side_decision(N, K):
     """perm_select = {best, accept} on the device picks the candidate row or the original order."""
-    N, K = 64, 256
     w = inputs.weight(small_cfg(N, K), 6, N=N)
     rng = np.random.default_rng(9)
     table = np.stack([rng.permutation(K) for _ in range(6)]).astype(np.int32)
