@@ -14,7 +14,9 @@
 //
 // Three kernels: rows of up to 6400 channels go four per warp (below, second kernel); wider rows one
 // per warp, eight positions per lane (first kernel); and without a permutation (channels already in
-// output order) rows of up to 4096 channels never leave the registers (third kernel).
+// output order) rows of up to 4096 channels never leave the registers (third kernel).  KIND 0 is RMSNorm,
+// 1 adaptive LayerNorm; the four-row kernel also exists as KIND 2, no normalization at all: the gather
+// quantizers of the offline path (a candidate order applied to activations or to the weight) run through it.
 #include "pq_common.cuh"
 
 namespace {
