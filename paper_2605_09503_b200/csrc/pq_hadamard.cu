@@ -193,11 +193,12 @@ __device__ __forceinline__ void pass_item(float *row_s, int base, int S, int sw,
 }
 
 // One pass over the rows of the block: items = rows x (K / 2) channel pairs / 2^LOG.
+template <int THREADS>
 __device__ __forceinline__ void run_pass(float *smem, const HadParams &p, int nrows, int S, int LOG, bool last) {
     const uint64_t scale2 = pack2(p.scale, p.scale);
     const int per_row = (p.K >> 1) >> LOG;  // items per row
     const int low_mask = (1 << (S - 1)) - 1;  // pair-index bits below the window (a pair index is channel >> 1)
-    for (int u = threadIdx.x; u < nrows * per_row; u += kThreads) {
+    for (int u = threadIdx.x; u < nrows * per_row; u += THREADS) {
         const int r = u / per_row, w = u - r * per_row;
         // w enumerates the pair positions with the window bits removed: low part below the window, the rest above
         const int pair = (w & low_mask) | ((w & ~low_mask) << LOG);
@@ -213,8 +214,10 @@ __device__ __forceinline__ void run_pass(float *smem, const HadParams &p, int nr
     }
 }
 
-template <int SF_LAYOUT>
-__global__ void __launch_bounds__(kThreads, kBlocksPerSm) hadamard_quant_kernel(const HadParams p) {
+// THREADS: 256 (two blocks per SM) while a block holds eight rows; 512 (one block) when rows wider than 6144
+// channels leave room for fewer, so that an SM still has 16 warps at work on them
+template <int SF_LAYOUT, int THREADS>
+__global__ void __launch_bounds__(THREADS, 512 / THREADS) hadamard_quant_kernel(const HadParams p) {
     extern __shared__ __align__(16) float had_smem[];  // [rows_per_block][K] fp32, then K 16-bit read-out offsets
     const int kRows = p.rows_per_block;
     uint16_t *offset_s = reinterpret_cast<uint16_t *>(had_smem + static_cast<size_t>(kRows) * p.K);
@@ -227,7 +230,7 @@ __global__ void __launch_bounds__(kThreads, kBlocksPerSm) hadamard_quant_kernel(
 
     // where each output position reads its channel in a row's (swizzled) shared-memory image, as a byte
     // offset: the same for every row, so it is worked out once per block (K <= 16384: 16 bits)
-    for (int j = threadIdx.x; j < p.K; j += kThreads)
+    for (int j = threadIdx.x; j < p.K; j += THREADS)
         offset_s[j] = static_cast<uint16_t>(swz(p.perm ? __ldg(p.perm + j) : j, p.sw) << 2);
     const float ts = p.codes ? __ldg(p.ts) : 1.0f;
 
@@ -237,7 +240,7 @@ __global__ void __launch_bounds__(kThreads, kBlocksPerSm) hadamard_quant_kernel(
         __syncthreads();  // the previous batch has been read out (and the offsets are in place)
 
         // ---- phase 1
-        for (int u = threadIdx.x; u < nrows * octs; u += kThreads) {
+        for (int u = threadIdx.x; u < nrows * octs; u += THREADS) {
             const int r = u / octs, o = u - r * octs;
             const uint16_t *src = p.X + (row0 + r) * p.ld + o * 8;
             float *row_s = had_smem + static_cast<size_t>(r) * p.K;
@@ -257,7 +260,7 @@ __global__ void __launch_bounds__(kThreads, kBlocksPerSm) hadamard_quant_kernel(
         int start = 3;
 #pragma unroll 1
         for (int k = 0; k < 3 && p.log[k]; ++k) {
-            run_pass(had_smem, p, nrows, start, p.log[k], k == 2 || p.log[k + 1] == 0);
+            run_pass<THREADS>(had_smem, p, nrows, start, p.log[k], k == 2 || p.log[k + 1] == 0);
             start += p.log[k];
             __syncthreads();
         }
@@ -266,7 +269,7 @@ __global__ void __launch_bounds__(kThreads, kBlocksPerSm) hadamard_quant_kernel(
         // the read-out offsets are fetched once for both rows and the two quantizer chains interleave
         const int rows_here = static_cast<int>(min(static_cast<int64_t>(kRows), p.rows_pad - row0));
         const int row_pairs = (rows_here + 1) >> 1;
-        for (int c = warp; c < row_pairs * chunks; c += kThreads / 32) {
+        for (int c = warp; c < row_pairs * chunks; c += THREADS / 32) {
             const int rp = c / chunks, g = (c - rp * chunks) * 32 + lane;
             const bool have = g < gpr;
             uint32_t iw[8];
@@ -285,7 +288,9 @@ __global__ void __launch_bounds__(kThreads, kBlocksPerSm) hadamard_quant_kernel(
                 const int r = 2 * rp + h;
                 row[h] = row0 + r;
                 present[h] = r < rows_here;
-                live[h] = row[h] < p.rows;
+                // the second row of the last pair does not exist when the block holds an odd number of rows (three
+                // at 16384 channels): that index is the first row of the NEXT batch and lies past this image
+                live[h] = present[h] && row[h] < p.rows;
                 const char *row_b = reinterpret_cast<const char *>(had_smem + static_cast<size_t>(r) * p.K);
 #pragma unroll
                 for (int j = 0; j < 16; ++j) out[h][j] = 0.0f;
@@ -406,15 +411,20 @@ extern "C" pq_status pq_hadamard_quant_nvfp4(const void *X, int64_t M, int64_t K
     // persistent grid: as many blocks as fit on the device at once, walking over the batches of rows
     int dev = 0, sms = 148;
     if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-    const int per_sm = static_cast<int>(std::min<size_t>(kBlocksPerSm, (227 * 1024) / (smem + 1024)));
+    const bool wide_block = kRows < kMaxRows;  // fewer rows per block: twice the threads on them, one block per SM
+    const int per_sm = static_cast<int>(std::min<size_t>(wide_block ? 1 : kBlocksPerSm, (227 * 1024) / (smem + 1024)));
     const int64_t batches = pq_ceil_div(p.rows_pad, kRows);
     const int64_t blocks = std::min<int64_t>(batches, static_cast<int64_t>(sms) * (per_sm > 0 ? per_sm : 1));
     auto launch = [&](auto kern) -> pq_status {
         if (smem > 48 * 1024)
             PQ_CUDA_OK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)));
-        PQ_CUDA_OK(pq::launch_dependent(kern, dim3(static_cast<unsigned>(blocks)), dim3(kThreads), smem, st, p));
+        PQ_CUDA_OK(pq::launch_dependent(kern, dim3(static_cast<unsigned>(blocks)), dim3(wide_block ? 2 * kThreads : kThreads),
+                                        smem, st, p));
         return pq_launch_status();
     };
-    return sf_layout == PQ_SF_TCGEN05 ? launch(hadamard_quant_kernel<PQ_SF_TCGEN05>)
-                                      : launch(hadamard_quant_kernel<PQ_SF_LINEAR>);
+    if (wide_block)
+        return sf_layout == PQ_SF_TCGEN05 ? launch(hadamard_quant_kernel<PQ_SF_TCGEN05, 2 * kThreads>)
+                                          : launch(hadamard_quant_kernel<PQ_SF_LINEAR, 2 * kThreads>);
+    return sf_layout == PQ_SF_TCGEN05 ? launch(hadamard_quant_kernel<PQ_SF_TCGEN05, kThreads>)
+                                      : launch(hadamard_quant_kernel<PQ_SF_LINEAR, kThreads>);
 }

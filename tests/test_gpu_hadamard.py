@@ -26,7 +26,9 @@ def _case(M, K, seed):
 @pytest.mark.parametrize("layout", [B.PQ_SF_LINEAR, B.PQ_SF_TCGEN05])
 @pytest.mark.parametrize("M,K,with_perm", [(37, 3072, True), (130, 3072, False), (9, 12288, True), (300, 1024, True),
                                            (5, 64, False), (23, 1536, True), (17, 192, True), (3, 16384, True),
-                                           (70, 256, True), (12, 768, True), (1, 4096, True)])
+                                           (70, 256, True), (12, 768, True), (1, 4096, True),
+                                           # blocks of three rows (16384 channels) and of six (8192), more than one batch
+                                           (8, 16384, True), (13, 8192, True)])
 def test_hadamard_quant_bit_exact(layout, M, K, with_perm):
     x, perm = _case(M, K, seed=M + K)
     ts = 0.02
