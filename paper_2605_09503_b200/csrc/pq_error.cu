@@ -11,32 +11,15 @@
 //     eight rows at a time and walks them in order; a block covers the eight chunks of a slab.  The pass streams the tensor once from HBM;
 //     its cost per element is arithmetic (about ten instructions), so it sits between the HBM and
 //     the ALU roof.
-//   candidate orders: one block per (chunk, order); rows are staged in shared memory a few at a
-//     time (coalesced) and the lanes gather their eight channels from there, so the tensor is
+//   candidate orders: one block per (chunk, order); the chunk's rows are staged in shared memory four
+//     at a time, interleaved per channel, and a thread gathers the 16 channels of its run for four rows
+//     with 64-bit loads, then runs the original-order kernel's error routine on them; the tensor is
 //     fetched from HBM once per chunk and served from L2 to the other orders' blocks.
 #include "pq_common.cuh"
 
 namespace {
 
 constexpr int kErrThreads = 256;
-
-// Gather path: a TEAM of group/8 adjacent lanes owns a group, 8 channels per lane.
-template <int KIND, int TEAM>
-__device__ __forceinline__ float group_sse_lane(const float (&x)[8], float ts, float Qf) {
-    const float amax = pq::team_max<TEAM>(pq::absmax8(x));
-    float q[8], d;
-    if (KIND == 0) {
-        uint32_t sf8;
-        float r;
-        pq::nvfp4_scale(amax, ts, sf8, d, r);
-        pq::nvfp4_levels_abs(x, r, q);
-    } else {
-        float r;
-        pq::int_scale(amax, Qf, d, r);
-        pq::int_levels_abs(x, r, Qf, q);
-    }
-    return pq::team_sum<TEAM>(pq::run_sse_abs(x, q, d));
-}
 
 // ---------------------------------------------------------------- original order
 constexpr int kDirectThreads = 128;
@@ -207,71 +190,98 @@ group_error_direct(const uint16_t *__restrict__ T, int64_t rows, int64_t K, int6
 }
 
 // ---------------------------------------------------------------- candidate orders
-constexpr int kMaxOctPerThread = 8;  // 256 threads x 8 octets x 8 channels = 16384 channels
+// One block per (chunk of 16 rows, candidate order).  The chunk goes through shared memory four rows at a
+// time, interleaved per channel (8 bytes per channel: one 64-bit load gathers a channel for four rows, so a
+// random order costs a quarter of the shared-memory wavefronts of a row-by-row gather); the 16-byte pieces of
+// an octet are XOR-swizzled by bits of the octet index, which makes the transposing stores conflict-free.  A
+// thread owns whole 16-channel runs (GPT of them, blockDim apart), keeps their 16 channel positions packed
+// in registers for the whole chunk, and for every row rebuilds the two 16-byte words the original-order
+// kernel loads, so the error of a run is computed by the same routine, in row order.
+constexpr int kMaxGpt = 4;  // 256 threads x 4 runs x 16 channels = 16384 channels
 
-template <int KIND, int TEAM>
+__device__ __forceinline__ int quad_piece(int o, int k) { return 4 * o + (k ^ ((o >> 1) & 3)); }   // 16-byte piece k of octet o
+__device__ __forceinline__ uint32_t quad_channel(uint32_t c) { return c ^ (((c >> 4) & 3u) << 1); }  // 8-byte slot of channel c
+
+template <int KIND, int TEAM16, int GPT>
 __global__ void __launch_bounds__(kErrThreads)
 group_error_gather(const uint16_t *__restrict__ T, int64_t rows, int64_t K, int64_t ld,
                    const float *__restrict__ ts_ptr, float Qf, const int32_t *__restrict__ perms, int P,
-                   int sub_rows, float *__restrict__ part /*[chunks, P, K/g]*/) {
-    extern __shared__ __align__(16) uint16_t rows_s[];  // [sub_rows][K]
+                   float *__restrict__ part /*[chunks, P, K/g]*/) {
+    extern __shared__ __align__(16) uint16_t quad_s[];  // [K][4 rows]
+    __shared__ float2 scale_table[KIND == 0 ? 256 : 1];
     pq::dependents_may_launch();
     const int64_t chunk = blockIdx.x;
     const int p = blockIdx.y;
     const int32_t *perm = perms + static_cast<int64_t>(p) * K;
-    const int oct_per_row = static_cast<int>(K >> 3);
+    const int octs = static_cast<int>(K >> 3), runs = static_cast<int>(K >> 4);
     const int64_t r0 = chunk * PQ_CHUNK_ROWS;
-    const int n = static_cast<int>(min(static_cast<int64_t>(PQ_CHUNK_ROWS), rows - r0));
     const float ts = (KIND == 0) ? __ldg(ts_ptr) : 1.0f;
+    const float c6 = __fmul_rn(6.0f, ts);
+    if (KIND == 0) build_scale_table(scale_table, ts);  // the first barrier below publishes it
 
-    // this thread's octets: o = threadIdx.x + i * kErrThreads; channel indices packed 2 x 16 bit
-    uint32_t ch[kMaxOctPerThread][4];
-    float acc[kMaxOctPerThread];
+    // positions of this thread's channels in the interleaved image, two per register
+    uint32_t ch[GPT][8];
+    float acc[GPT];
 #pragma unroll
-    for (int i = 0; i < kMaxOctPerThread; ++i) {
-        acc[i] = 0.0f;
-        const int o = threadIdx.x + i * kErrThreads;
+    for (int t = 0; t < GPT; ++t) {
+        acc[t] = 0.0f;
+        const int q = threadIdx.x + t * blockDim.x;
 #pragma unroll
-        for (int w = 0; w < 4; ++w) {
+        for (int w = 0; w < 8; ++w) {
             uint32_t lo = 0, hi = 0;
-            if (o < oct_per_row) {
-                lo = static_cast<uint32_t>(perm[o * 8 + 2 * w]);
-                hi = static_cast<uint32_t>(perm[o * 8 + 2 * w + 1]);
+            if (q < runs) {
+                lo = quad_channel(static_cast<uint32_t>(perm[q * 16 + 2 * w]));
+                hi = quad_channel(static_cast<uint32_t>(perm[q * 16 + 2 * w + 1]));
             }
-            ch[i][w] = lo | (hi << 16);
+            ch[t][w] = lo | (hi << 16);
         }
     }
 
-    for (int s0 = 0; s0 < n; s0 += sub_rows) {
-        const int ns = min(sub_rows, n - s0);
-        __syncthreads();
-        for (int idx = threadIdx.x; idx < ns * oct_per_row; idx += kErrThreads) {
-            const int rr = idx / oct_per_row, o = idx - rr * oct_per_row;
-            reinterpret_cast<uint4 *>(rows_s)[idx] =
-                __ldg(reinterpret_cast<const uint4 *>(T + (r0 + s0 + rr) * ld) + o);
+    uint4 *quad4 = reinterpret_cast<uint4 *>(quad_s);
+    const uint2 *quad2 = reinterpret_cast<const uint2 *>(quad_s);
+#pragma unroll 1
+    for (int quad = 0; quad < PQ_CHUNK_ROWS / 4; ++quad) {
+        const int64_t row = r0 + 4 * quad;
+        __syncthreads();  // the previous four rows have been used
+        for (int o = threadIdx.x; o < octs; o += blockDim.x) {
+            uint4 v[4];
+#pragma unroll
+            for (int r = 0; r < 4; ++r)  // rows past the end are zeros: their error is +0.0 and adding it changes nothing
+                v[r] = row + r < rows ? __ldg(reinterpret_cast<const uint4 *>(T + (row + r) * ld) + o) : make_uint4(0, 0, 0, 0);
+            const uint32_t *w0 = &v[0].x, *w1 = &v[1].x, *w2 = &v[2].x, *w3 = &v[3].x;
+#pragma unroll
+            for (int k = 0; k < 4; ++k)
+                quad4[quad_piece(o, k)] = make_uint4(__byte_perm(w0[k], w1[k], 0x5410), __byte_perm(w2[k], w3[k], 0x5410),
+                                                     __byte_perm(w0[k], w1[k], 0x7632), __byte_perm(w2[k], w3[k], 0x7632));
         }
         __syncthreads();
-        for (int rr = 0; rr < ns; ++rr) {
-            const uint16_t *row = rows_s + static_cast<int64_t>(rr) * K;
 #pragma unroll
-            for (int i = 0; i < kMaxOctPerThread; ++i) {
-                if (i * kErrThreads >= oct_per_row) break;  // uniform over the block
-                const bool live = threadIdx.x + i * kErrThreads < oct_per_row;
-                float x[8];
+        for (int t = 0; t < GPT; ++t) {
+            if (t * static_cast<int>(blockDim.x) >= runs) break;  // uniform over the block
+            uint2 g[16];
 #pragma unroll
-                for (int w = 0; w < 4; ++w) {
-                    x[2 * w] = live ? pq::bf16_bits_to_f32(row[ch[i][w] & 0xFFFFu]) : 0.0f;
-                    x[2 * w + 1] = live ? pq::bf16_bits_to_f32(row[ch[i][w] >> 16]) : 0.0f;
+            for (int w = 0; w < 8; ++w) {
+                g[2 * w] = quad2[ch[t][w] & 0xFFFFu];
+                g[2 * w + 1] = quad2[ch[t][w] >> 16];
+            }
+#pragma unroll
+            for (int r = 0; r < 4; ++r) {
+                uint32_t pr[8];
+#pragma unroll
+                for (int w = 0; w < 8; ++w) {
+                    const uint32_t a = r < 2 ? g[2 * w].x : g[2 * w].y, b = r < 2 ? g[2 * w + 1].x : g[2 * w + 1].y;
+                    pr[w] = __byte_perm(a, b, (r & 1) ? 0x7632 : 0x5410);
                 }
-                acc[i] = __fadd_rn(acc[i], group_sse_lane<KIND, TEAM>(x, ts, Qf));
+                acc[t] = __fadd_rn(acc[t], row_sse16<KIND, TEAM16>(make_uint4(pr[0], pr[1], pr[2], pr[3]),
+                                                                   make_uint4(pr[4], pr[5], pr[6], pr[7]), c6, scale_table, Qf));
             }
         }
     }
-    const int64_t Kg = K / (8 * TEAM);
+    const int64_t Kg = runs / TEAM16;
 #pragma unroll
-    for (int i = 0; i < kMaxOctPerThread; ++i) {
-        const int o = threadIdx.x + i * kErrThreads;
-        if (o < oct_per_row && (o % TEAM) == 0) part[(chunk * P + p) * Kg + o / TEAM] = acc[i];
+    for (int t = 0; t < GPT; ++t) {
+        const int q = threadIdx.x + t * blockDim.x;
+        if (q < runs && (q % TEAM16) == 0) part[(chunk * P + p) * Kg + q / TEAM16] = acc[t];
     }
 }
 
@@ -292,16 +302,23 @@ pq_status launch(const uint16_t *T, int64_t rows, int64_t K, int64_t ld, const f
         if (pq_launch_status() != PQ_OK) return PQ_ERR_CUDA;
         return fold<double, 1>(ws, slabs, Kg, err, st);
     }
-    int sub_rows = static_cast<int>((96 * 1024) / (K * 2));
-    if (sub_rows > 16) sub_rows = 16;
-    if (sub_rows < 1) sub_rows = 1;
-    const size_t smem = static_cast<size_t>(sub_rows) * K * 2;
-    if (smem > 48 * 1024)
-        PQ_CUDA_OK(cudaFuncSetAttribute(group_error_gather<KIND, TEAM>,
-                                        cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)));
+    const int runs = static_cast<int>(K >> 4);
+    const int threads = runs >= kErrThreads ? kErrThreads : ((runs + 31) / 32) * 32;
+    const int gpt = static_cast<int>(pq_ceil_div(runs, threads));
+    if (gpt > kMaxGpt) return PQ_ERR_SHAPE;
+    const size_t smem = static_cast<size_t>(K) * 8;  // four rows, interleaved per channel
     dim3 grid(static_cast<unsigned>(chunks), static_cast<unsigned>(P));
-    group_error_gather<KIND, TEAM><<<grid, kErrThreads, smem, st>>>(T, rows, K, ld, ts, Qf, perms, P, sub_rows,
-                                                                 static_cast<float *>(ws));
+    auto run = [&](auto kern) -> pq_status {
+        if (smem > 40 * 1024)  // the kernel's static shared memory counts towards the 48 KB default limit
+            PQ_CUDA_OK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)));
+        kern<<<grid, threads, smem, st>>>(T, rows, K, ld, ts, Qf, perms, P, static_cast<float *>(ws));
+        return PQ_OK;
+    };
+    constexpr int TEAM16 = TEAM / 2;
+    const pq_status rl = gpt == 1   ? run(group_error_gather<KIND, TEAM16, 1>)
+                         : gpt == 2 ? run(group_error_gather<KIND, TEAM16, 2>)
+                                    : run(group_error_gather<KIND, TEAM16, 4>);
+    if (rl != PQ_OK) return rl;
     if (pq_launch_status() != PQ_OK) return PQ_ERR_CUDA;
     return fold<float, kSlabChunks>(ws, chunks, static_cast<int64_t>(P) * Kg, err, st);
 }
