@@ -100,7 +100,7 @@ def test_calibration_partials_combine_in_rank_order():
 def test_bench_starts_its_own_ranks():
     """`python bench.py --gpus 2` without a launcher starts two ranks itself (torch.distributed.run on
     127.0.0.1).  On a machine without a GPU each rank must stop at the explicit "needs a CUDA device"
-    exit (there is no CPU fallback), which shows that both ranks were started and reached the GPU arm."""
+    exit (there is no CPU fallback), which shows that the ranks were started and reached the GPU arm."""
     import subprocess
     import sys
     if torch.cuda.is_available():
@@ -110,4 +110,8 @@ def test_bench_starts_its_own_ranks():
     out = subprocess.run([sys.executable, os.path.join(root, "bench.py"), "--gpus", "2", "--steps", "2", "--warmup", "1"],
                          env=env, capture_output=True, text=True, timeout=600)
     assert out.returncode != 0
-    assert (out.stdout + out.stderr).count("bench.py needs a CUDA device") == 2
+    text = out.stdout + out.stderr
+    # the launcher ends the other rank as soon as one has failed, so one or two ranks get to say it
+    assert 1 <= text.count("bench.py needs a CUDA device") <= 2
+    # the launcher prints this notice only when it starts more than one process per node
+    assert "OMP_NUM_THREADS environment variable for each process" in text
