@@ -30,7 +30,9 @@ def _case(M, K, seed):
                                            # channels already in output order: the register-resident kernel at each of
                                            # its four register sizes, and the fall-back for rows wider than 4096
                                            (150, 1024, False), (33, 2048, False), (20, 4096, False), (7, 6400, False),
-                                           (129, 2560, False)])
+                                           (129, 2560, False),
+                                           # the widest rows (three and six warps per block), several blocks
+                                           (29, 16384, True), (10, 32768, True), (10, 32768, False)])
 def test_norm_quant_bit_exact(kind, layout, M, K, with_perm):
     h, a, b, perm = _case(M, K, seed=M + K + kind)
     ts, eps = 0.011, 1e-6

@@ -99,7 +99,8 @@ def test_group_error_original_order_bit_exact(fmt, rows, K):
 
 
 @pytest.mark.parametrize("fmt", FORMATS)
-@pytest.mark.parametrize("rows,K,P", [(130, 512, 7), (70, 3072, 3), (5, 4096, 1), (64, 12288, 2)])
+@pytest.mark.parametrize("rows,K,P", [(130, 512, 7), (70, 3072, 3), (5, 4096, 1), (64, 12288, 2),
+                                      (33, 8192, 2), (40, 16384, 2), (21, 48 * 16, 8)])   # two and four runs per thread
 def test_group_error_candidates_bit_exact(fmt, rows, K, P):
     x = inputs.activations(small_cfg(rows, K), 3, 0)
     rng = np.random.default_rng(K + P)
@@ -194,7 +195,7 @@ def test_quant_weight_device_side_decision(N, K):
 
 
 @pytest.mark.parametrize("bits,group", [(3, 32), (3, 64), (3, 128), (4, 32), (4, 64), (4, 128), (4, 16), (8, 32)])
-@pytest.mark.parametrize("rows,K,with_perm", [(130, 512, False), (33, 3072, True), (4, 16384, True)])
+@pytest.mark.parametrize("rows,K,with_perm", [(130, 512, False), (33, 3072, True), (4, 16384, True), (40, 16384, True)])
 def test_fakequant_int_bit_exact(bits, group, rows, K, with_perm):
     x = inputs.activations(small_cfg(rows, K), 7, 0)
     perm = np.random.default_rng(K).permutation(K).astype(np.int32) if with_perm else None

@@ -55,7 +55,7 @@ def test_output_error_full_size_output_of_the_bench_layer():
 
 
 @pytest.mark.parametrize("layout", [B.PQ_SF_LINEAR, B.PQ_SF_TCGEN05])
-@pytest.mark.parametrize("M,K", [(130, 512), (37, 3072), (5, 16384), (129, 6400), (3, 6464), (2, 64)])
+@pytest.mark.parametrize("M,K", [(130, 512), (37, 3072), (5, 16384), (129, 6400), (3, 6464), (2, 64), (40, 8192)])
 def test_quant_act_with_an_order_is_bit_exact(layout, M, K):
     g = torch.Generator().manual_seed(M + K)
     x = (torch.randn(M, K, generator=g) * torch.exp(torch.randn(K, generator=g))).to(torch.bfloat16)
