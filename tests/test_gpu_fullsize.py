@@ -182,3 +182,40 @@ def test_hadamard_producer_and_new_statistics_on_a_full_batch():
     err = torch.zeros(1, cfg.K // 256, dtype=torch.float64, device=DEV)
     B.pq_group_error(xd, (B.KIND_INT, 4, 256), None, None, err, B.workspace(B.OP_GROUP_ERROR, cfg.M, cfg.K, 0, 1))
     assert np.array_equal(err.cpu().numpy(), O.group_error(xb, 1, 4, 256))
+
+
+def test_a_full_batch_through_the_kernels_that_apply_a_channel_order():
+    """The bench's stage sizes for the kernels that gather through a permutation, whole 4608 x 3072 tensors bit for
+    bit: the fused adaptive-LayerNorm producer (tensor-core scale layout), the quantizer with a candidate order,
+    the error of six candidate orders in one call, and the integer fake-quant with an order."""
+    from test_gpu_gemm import to_tc
+    cfg = inputs.CONFIGS["qkv"]
+    M, K = cfg.M, cfg.K
+    x = inputs.activations(cfg, 0, 5)
+    xb, xd = inputs.bits(x), x.to(DEV)
+    g = torch.Generator().manual_seed(23)
+    perms = torch.stack([torch.randperm(K, generator=g) for _ in range(6)]).to(torch.int32)
+    perm = perms[2].contiguous()
+    ts = O.tensor_scale(O.calib_stats(xb)[1])
+    tsd = torch.tensor([ts], dtype=torch.float32, device=DEV)
+    xq = torch.empty(M, K // 2, dtype=torch.uint8, device=DEV)
+    sf = torch.empty(B.sf_bytes(M, K, B.PQ_SF_TCGEN05), dtype=torch.uint8, device=DEV)
+    # quantizer with a candidate order
+    B.pq_quant_act_nvfp4_perm(xd, perm.to(DEV), tsd, xq, sf, B.PQ_SF_TCGEN05)
+    c_o, s_o = O.quant_nvfp4(xb, ts, perm.numpy())
+    assert np.array_equal(xq.cpu().numpy(), c_o) and np.array_equal(sf.cpu().numpy(), to_tc(s_o))
+    # fused producer
+    a = (0.3 * torch.randn(K, generator=g)).float()
+    b = torch.randn(K, generator=g).float()
+    ts_n = torch.tensor([0.011], dtype=torch.float32, device=DEV)
+    B.pq_norm_quant_nvfp4(xd, B.NORM_ADALN, a.to(DEV), b.to(DEV), 1e-6, perm.to(DEV), ts_n, xq, sf, B.PQ_SF_TCGEN05, None)
+    c_o, s_o, _ = O.norm_quant_nvfp4(xb, 1, a.numpy(), b.numpy(), 1e-6, 0.011, perm.numpy())
+    assert np.array_equal(xq.cpu().numpy(), c_o) and np.array_equal(sf.cpu().numpy(), to_tc(s_o))
+    # six candidate orders in one error pass
+    err = torch.zeros(6, K // 16, dtype=torch.float64, device=DEV)
+    B.pq_group_error(xd, (B.KIND_NVFP4, 4, 16), tsd, perms.to(DEV), err, B.workspace(B.OP_GROUP_ERROR, M, K, 0, 6))
+    assert np.array_equal(err.cpu().numpy(), O.group_error(xb, 0, 4, 16, ts=ts, perms=perms.numpy()))
+    # integer fake-quant with an order
+    out = torch.empty(M, K, dtype=torch.bfloat16, device=DEV)
+    B.pq_fakequant_int(xd, (B.KIND_INT, 4, 64), perm.to(DEV), out)
+    assert np.array_equal(inputs.bits(out.cpu()), O.fakequant_int(xb, 4, 64, perm.numpy()))
