@@ -224,6 +224,35 @@ def graph_loop(torch, fn, iters, warmup=3, replays=3):
     return a.elapsed_time(b) / (iters * replays)
 
 
+def burst_loop(torch, fn, iters, repeats=5, pause_s=0.25):
+    """graph_loop in the regime of the headline loop: `iters` calls in one CUDA graph, replayed once per
+    repeat after an idle pause and three warm-up calls; median milliseconds per call.  A kernel timed this
+    way has not been running long enough for the board's power cap to lower the clock, which is the
+    condition the burst peak was measured under."""
+    for i in range(3):
+        fn(i)
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        for i in range(iters):
+            fn(i)
+    graph.replay()
+    torch.cuda.synchronize()
+    times = []
+    for _ in range(repeats):
+        time.sleep(pause_s)
+        for i in range(3):
+            fn(i)
+        torch.cuda.synchronize()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        graph.replay()
+        b.record()
+        torch.cuda.synchronize()
+        times.append(a.elapsed_time(b) / iters)
+    return sorted(times)[len(times) // 2]
+
+
 def run_ours(args):
     import torch
     import torch.distributed as dist
@@ -303,6 +332,18 @@ def run_ours(args):
     sampler = ClockSampler(local)
     for i in range(max(args.warmup, 3)):
         step(i)
+    # The K steps of a repeat go out as ONE CUDA-graph launch (captured here, through the same public call):
+    # the timed region then holds exactly the K steps' kernels back to back, as a serving loop would run them,
+    # and not the host's start-up latency of the first launch after the synchronize, which weighs on a short
+    # loop (K = 20: about 1 us per step).  Very long loops are launched directly.
+    step_graph = None
+    if args.steps <= 2000:
+        torch.cuda.synchronize()
+        step_graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(step_graph):
+            for i in range(args.steps):
+                step(i)
+        torch.cuda.synchronize()
     repeats = []
     sampler.start()
     for _ in range(REPEATS):
@@ -317,8 +358,11 @@ def run_ours(args):
         barrier()
         a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         a.record()
-        for i in range(args.steps):
-            step(i)
+        if step_graph is not None:
+            step_graph.replay()
+        else:
+            for i in range(args.steps):
+                step(i)
         b.record()
         sampler.sample()                   # the queue is still draining here
         barrier()
@@ -329,6 +373,12 @@ def run_ours(args):
         L.check()
     flops = 2.0 * M * N * K
     value = world * flops / (ms_step * 1e-3) / 1e12
+
+    # ---- the two kernels of the step on their own (same launch configuration, same rotation), in the same
+    # regime as the headline loop: short graph launches with idle pauses, before the long loop below heats the board
+    iters = max(20, min(args.steps, 200))
+    ms_gemm = burst_loop(torch, gemm_only, iters, REPEATS, REPEAT_PAUSE_S)
+    ms_quant = burst_loop(torch, quant_only, iters, REPEATS, REPEAT_PAUSE_S)
 
     # ---- the same loop held for about 1.5 s: the 1 kW power cap engages after a few hundred steps and
     # the SM clock settles near 1.6 GHz; this figure goes with the sustained peak, the headline (a few
@@ -349,10 +399,8 @@ def run_ours(args):
         barrier()
         ms_sustained = max_over_ranks(a2.elapsed_time(b2) / sustained_steps)
 
-    # ---- the two kernels of the step on their own (same launch configuration, same rotation)
-    iters = max(20, min(args.steps, 200))
-    ms_gemm = graph_loop(torch, gemm_only, iters)
-    ms_quant = graph_loop(torch, quant_only, iters)
+    # ---- the GEMM again right behind the long loop: the power-capped figure that goes with the sustained peak
+    ms_gemm_capped = graph_loop(torch, gemm_only, iters) if sustained_steps else None
     fp4_peak = peaks["bf16_tflops"] * FP4_OVER_BF16
     gemm_tflops = flops / (ms_gemm * 1e-3) / 1e12
     quant_bytes = M * K * 2 + M * K // 2 + M * K // 16
@@ -362,7 +410,11 @@ def run_ours(args):
                                   "workload (profiles/gemm_w4a4_kernel_qkv_4608x3072x9216.md); algorithmic bytes 108.8e6",
                 "peak_source": f"{peaks['source']} bf16 burst {peaks['bf16_tflops']} TFLOP/s x {FP4_OVER_BF16:g} "
                                f"(nominal fp4:bf16 ratio)",
-                "frac_of_sustained": gemm_tflops / (peaks["bf16_tflops_sustained"] * FP4_OVER_BF16),
+                "regime": "burst: CUDA-graph launches of a few milliseconds with idle pauses, like the measured peak",
+                "after_sustained_loop": None if ms_gemm_capped is None else {
+                    "ms_per_launch": ms_gemm_capped, "achieved": flops / (ms_gemm_capped * 1e-3) / 1e12,
+                    "frac_of_sustained_peak": flops / (ms_gemm_capped * 1e-3) / 1e12
+                                              / (peaks["bf16_tflops_sustained"] * FP4_OVER_BF16)},
                 "frac_of_nominal_9000": gemm_tflops / 9000.0,
                 "ms_per_launch": ms_gemm, "flops_per_launch": flops}
     quant_gbs = quant_bytes / (ms_quant * 1e-3) / 1e9
@@ -370,7 +422,7 @@ def run_ours(args):
     # written), timed the same way; the peak the fractions use is a copy of 4 GB, where launch, ramp and tail vanish
     copy_src = [torch.empty(quant_bytes // 2, dtype=torch.uint8, device=dev) for _ in range(XROT)]
     copy_dst = [torch.empty(quant_bytes // 2, dtype=torch.uint8, device=dev) for _ in range(XROT)]
-    ms_copy = graph_loop(torch, lambda i: copy_dst[i % XROT].copy_(copy_src[i % XROT]), iters)
+    ms_copy = burst_loop(torch, lambda i: copy_dst[i % XROT].copy_(copy_src[i % XROT]), iters, REPEATS, REPEAT_PAUSE_S)
     del copy_src, copy_dst
     stages = {"quant_act_nvfp4": {"ms": ms_quant, "GB/s": quant_gbs, "frac_hbm": quant_gbs / peaks["hbm_gbs"],
                                   "frac_hbm_nominal_8000": quant_gbs / 8000.0, "bytes": quant_bytes,
@@ -578,7 +630,9 @@ def run_ours(args):
                        "l2": f"timed loop rotates over {NSETS} complete buffer sets ({NSETS * set_bytes / 1e6:.0f} MB "
                              f"> 126 MB L2); stand-alone kernel loops are CUDA-graph replays rotating over {XROT} "
                              f"inputs of 28 MB or 2 of 226 MB",
-                       "timing": f"value = median of {REPEATS} repeats of the {args.steps}-step loop, {REPEAT_PAUSE_S} s idle and 3 "
+                       "timing": f"value = median of {REPEATS} repeats of the {args.steps}-step loop"
+                                 f"{' (one CUDA-graph launch of the public call per repeat)' if step_graph is not None else ''}, "
+                                 f"{REPEAT_PAUSE_S} s idle and 3 "
                                  f"warm-up steps before each (burst regime); stages.linear_incl_quant_sustained holds the "
                                  f"loop for about a second (power-capped regime)",
                        "accepted_permutation": bool(cal.select[1].item())},
