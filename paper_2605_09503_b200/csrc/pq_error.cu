@@ -202,8 +202,9 @@ constexpr int kMaxGpt = 4;  // 256 threads x 4 runs x 16 channels = 16384 channe
 __device__ __forceinline__ int quad_piece(int o, int k) { return 4 * o + (k ^ ((o >> 1) & 3)); }   // 16-byte piece k of octet o
 __device__ __forceinline__ uint32_t quad_channel(uint32_t c) { return c ^ (((c >> 4) & 3u) << 1); }  // 8-byte slot of channel c
 
+// one run per thread (up to 4096 channels): held to 64 registers, five 192-thread blocks per SM instead of four
 template <int KIND, int TEAM16, int GPT>
-__global__ void __launch_bounds__(kErrThreads)
+__global__ void __launch_bounds__(kErrThreads, GPT == 1 ? 4 : 1)
 group_error_gather(const uint16_t *__restrict__ T, int64_t rows, int64_t K, int64_t ld,
                    const float *__restrict__ ts_ptr, float Qf, const int32_t *__restrict__ perms, int P,
                    float *__restrict__ part /*[chunks, P, K/g]*/) {
