@@ -109,17 +109,34 @@ quant_nvfp4_kernel(const uint16_t *__restrict__ X, int64_t rows, int64_t rows_pa
 __global__ void amax_all_kernel(const uint16_t *__restrict__ W, int64_t rows, int64_t K, int64_t ld,
                                 unsigned int *__restrict__ amax_bits) {
     const int64_t oct = static_cast<int64_t>(blockIdx.x) * 32 + threadIdx.x;
-    float a = 0.0f;
+    // a maximum of magnitudes selects one of its inputs, so it is taken on the bf16 pairs and in any order:
+    // four rows in flight per step
+    uint32_t mx = 0;
     if (oct * 8 < K) {
-        for (int64_t row = static_cast<int64_t>(blockIdx.y) * kTileRows + threadIdx.y; row < rows;
-             row += static_cast<int64_t>(gridDim.y) * kTileRows) {
-            float x[8];
-            pq::unpack8(__ldg(reinterpret_cast<const uint4 *>(W + row * ld + oct * 8)), x);
-            a = fmaxf(a, pq::absmax8(x));
+        const int64_t step = static_cast<int64_t>(gridDim.y) * kTileRows;
+        for (int64_t row = static_cast<int64_t>(blockIdx.y) * kTileRows + threadIdx.y; row < rows; row += 4 * step) {
+            uint4 v[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u)
+                v[u] = row + u * step < rows ? __ldg(reinterpret_cast<const uint4 *>(W + (row + u * step) * ld + oct * 8))
+                                             : make_uint4(0, 0, 0, 0);
+            const uint32_t m = 0x7FFF7FFFu;
+#pragma unroll
+            for (int u = 0; u < 4; ++u)
+                mx = pq::max_bf16x2(mx, pq::max_bf16x2(pq::max_bf16x2(v[u].x & m, v[u].y & m), pq::max_bf16x2(v[u].z & m, v[u].w & m)));
         }
     }
+    float a = fmaxf(__uint_as_float(mx << 16), __uint_as_float(mx & 0xFFFF0000u));
     for (int m = 16; m; m >>= 1) a = fmaxf(a, __shfl_xor_sync(0xFFFFFFFFu, a, m));
-    if (threadIdx.x == 0 && a > 0.0f) atomicMax(amax_bits, __float_as_uint(a));
+    // one atomic per block (all of them hit the same word)
+    __shared__ float warp_max[kTileRows];
+    if (threadIdx.x == 0) warp_max[threadIdx.y] = a;
+    __syncthreads();
+    if (threadIdx.x == 0 && threadIdx.y == 0) {
+#pragma unroll
+        for (int w = 1; w < kTileRows; ++w) a = fmaxf(a, warp_max[w]);
+        if (a > 0.0f) atomicMax(amax_bits, __float_as_uint(a));
+    }
 }
 
 __global__ void weight_scale_kernel(const unsigned int *__restrict__ amax_bits, float *ts) {
