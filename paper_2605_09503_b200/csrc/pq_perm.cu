@@ -55,12 +55,17 @@ __global__ void plain_keys(const double *__restrict__ v, int64_t K, unsigned lon
 
 constexpr int kRankThreads = 256;
 
+// Four neighbouring lanes share a channel: each counts the keys of a quarter of every tile that precede the
+// channel's, the four counts are added by shuffles (integers: any order).  A block ranks 64 channels.
+constexpr int kRankShare = 4, kRankChannels = kRankThreads / kRankShare;
+
 __global__ void __launch_bounds__(kRankThreads)
 perm_rank(const unsigned long long *__restrict__ keys, int64_t K, int32_t *__restrict__ perms, int deal_groups, int group) {
     __shared__ unsigned long long tile[kRankThreads];
     const int j = blockIdx.y;
     const unsigned long long *kj = keys + static_cast<int64_t>(j) * K;
-    const int64_t i = static_cast<int64_t>(blockIdx.x) * kRankThreads + threadIdx.x;
+    const int sub = threadIdx.x % kRankShare;
+    const int64_t i = static_cast<int64_t>(blockIdx.x) * kRankChannels + threadIdx.x / kRankShare;
     const unsigned long long mine = (i < K) ? kj[i] : 0ull;
     int rank = 0;
     for (int64_t base = 0; base < K; base += kRankThreads) {
@@ -68,17 +73,20 @@ perm_rank(const unsigned long long *__restrict__ keys, int64_t K, int32_t *__res
         __syncthreads();
         tile[threadIdx.x] = (l < K) ? kj[l] : 0ull;
         __syncthreads();
-        const int n = static_cast<int>(min(static_cast<int64_t>(kRankThreads), K - base));
-        for (int u = 0; u < n; ++u) {
+        // the whole tile, unrolled: a slot past the end holds key 0 at an index above every channel, which
+        // precedes nothing ("other precedes mine": larger key, or equal key and lower channel index)
+#pragma unroll 16
+        for (int u = sub; u < kRankThreads; u += kRankShare) {
             const unsigned long long other = tile[u];
-            // "other precedes mine": larger key, or equal key and lower channel index
             rank += (other > mine) || (other == mine && base + u < i);
         }
     }
+#pragma unroll
+    for (int m = 1; m < kRankShare; m <<= 1) rank += __shfl_xor_sync(0xFFFFFFFFu, rank, m);
     // deal_groups == 0: the channel of rank r is read at position r; otherwise the sorted channels are dealt
     // to deal_groups groups in turn: rank r goes to group r % deal_groups, slot r / deal_groups
     const int64_t pos = deal_groups ? static_cast<int64_t>(rank % deal_groups) * group + rank / deal_groups : rank;
-    if (i < K) perms[static_cast<int64_t>(j) * K + pos] = static_cast<int32_t>(i);
+    if (i < K && sub == 0) perms[static_cast<int64_t>(j) * K + pos] = static_cast<int32_t>(i);
 }
 
 // One thread per order p = 0..P sums its error rows; thread 0 then applies Eq. 10.
@@ -121,7 +129,7 @@ extern "C" pq_status pq_select_perm(const double *sumsq_a, int64_t rows_a, const
     unsigned long long *keys = static_cast<unsigned long long *>(ws);
     perm_keys<<<static_cast<unsigned>(pq_ceil_div(K, 128)), 128, 0, st>>>(
         sumsq_a, static_cast<double>(rows_a), sumsq_w, static_cast<double>(rows_w), K, J, keys);
-    dim3 grid(static_cast<unsigned>(pq_ceil_div(K, kRankThreads)), static_cast<unsigned>(J + 1));
+    dim3 grid(static_cast<unsigned>(pq_ceil_div(K, kRankChannels)), static_cast<unsigned>(J + 1));
     perm_rank<<<grid, kRankThreads, 0, st>>>(keys, K, perms, 0, 0);
     return pq_launch_status();
 }
@@ -135,7 +143,7 @@ extern "C" pq_status pq_order_by_absmax(const float *amax, int64_t K, int32_t *p
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     unsigned long long *keys = static_cast<unsigned long long *>(ws);
     absmax_keys<<<static_cast<unsigned>(pq_ceil_div(K, 128)), 128, 0, st>>>(amax, K, keys);
-    perm_rank<<<dim3(static_cast<unsigned>(pq_ceil_div(K, kRankThreads)), 1), kRankThreads, 0, st>>>(keys, K, perm, 0, 0);
+    perm_rank<<<dim3(static_cast<unsigned>(pq_ceil_div(K, kRankChannels)), 1), kRankThreads, 0, st>>>(keys, K, perm, 0, 0);
     return pq_launch_status();
 }
 
@@ -148,7 +156,7 @@ extern "C" pq_status pq_order_by_variance(const double *sum, const double *sumsq
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     unsigned long long *keys = static_cast<unsigned long long *>(ws);
     variance_keys<<<static_cast<unsigned>(pq_ceil_div(K, 128)), 128, 0, st>>>(sum, sumsq, static_cast<double>(rows), K, keys);
-    perm_rank<<<dim3(static_cast<unsigned>(pq_ceil_div(K, kRankThreads)), 1), kRankThreads, 0, st>>>(keys, K, perm, 0, 0);
+    perm_rank<<<dim3(static_cast<unsigned>(pq_ceil_div(K, kRankChannels)), 1), kRankThreads, 0, st>>>(keys, K, perm, 0, 0);
     return pq_launch_status();
 }
 
@@ -161,7 +169,7 @@ extern "C" pq_status pq_order_round_robin(const double *sumsq, int64_t K, int gr
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     unsigned long long *keys = static_cast<unsigned long long *>(ws);
     plain_keys<<<static_cast<unsigned>(pq_ceil_div(K, 128)), 128, 0, st>>>(sumsq, K, keys);
-    perm_rank<<<dim3(static_cast<unsigned>(pq_ceil_div(K, kRankThreads)), 1), kRankThreads, 0, st>>>(
+    perm_rank<<<dim3(static_cast<unsigned>(pq_ceil_div(K, kRankChannels)), 1), kRankThreads, 0, st>>>(
         keys, K, perm, static_cast<int>(K / group), group);
     return pq_launch_status();
 }

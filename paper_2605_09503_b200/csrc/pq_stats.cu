@@ -205,13 +205,23 @@ __global__ void tensor_scale_kernel(const float *__restrict__ amax, int64_t K, f
     }
 }
 
-// lambda[s] = 1 / (sequential fp64 sum of side s), one thread per side.
-__global__ void error_weights_kernel(const double *__restrict__ sa, const double *__restrict__ sw,
-                                     int64_t K, double *lambda) {
-    const double *src = threadIdx.x == 0 ? sa : sw;
+// lambda[s] = 1 / (sequential fp64 sum of side s in ascending channel order), one warp per side: the lanes
+// fetch 1024 values at a time into shared memory (coalesced), lane 0 adds them in order.
+__global__ void __launch_bounds__(64) error_weights_kernel(const double *__restrict__ sa, const double *__restrict__ sw,
+                                                           int64_t K, double *lambda) {
+    __shared__ double stage[2][1024];
+    const int side = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const double *src = side == 0 ? sa : sw;
     double s = 0.0;
-    for (int64_t i = 0; i < K; ++i) s = __dadd_rn(s, src[i]);
-    lambda[threadIdx.x] = __ddiv_rn(1.0, s);
+    for (int64_t i0 = 0; i0 < K; i0 += 1024) {
+        const int n = static_cast<int>(K - i0 < 1024 ? K - i0 : 1024);
+        for (int j = lane; j < n; j += 32) stage[side][j] = src[i0 + j];
+        __syncwarp();
+        if (lane == 0)
+            for (int j = 0; j < n; ++j) s = __dadd_rn(s, stage[side][j]);
+        __syncwarp();
+    }
+    if (lane == 0) lambda[side] = __ddiv_rn(1.0, s);
 }
 
 }  // namespace
@@ -283,7 +293,7 @@ extern "C" pq_status pq_error_weights(const double *sumsq_a, const double *sumsq
                                       double *lambda, void *stream) {
     PQ_REQUIRE(sumsq_a && sumsq_w && lambda, PQ_ERR_NULL);
     PQ_REQUIRE(K > 0, PQ_ERR_SHAPE);
-    error_weights_kernel<<<1, 2, 0, static_cast<cudaStream_t>(stream)>>>(sumsq_a, sumsq_w, K, lambda);
+    error_weights_kernel<<<1, 64, 0, static_cast<cudaStream_t>(stream)>>>(sumsq_a, sumsq_w, K, lambda);
     return pq_launch_status();
 }
 
